@@ -1,0 +1,198 @@
+/*
+ * percache.h — C ABI of the reuse-prefill library (one model, one GPU per handle).
+ *
+ * The operation is the one PerCache's QKV-cache tier performs at query time
+ * (paper Section 3.2.2 "QKV Cache Reuse", Appendix B.1 "Inference implementation
+ * details"): a prompt is an ordered list of knowledge chunks followed by the
+ * user's query tokens; tensors of chunks already in the cache are loaded and
+ * concatenated in order, the rows they cover are dropped from every block's
+ * attention input, projection and position encoding run on the remaining rows
+ * only (each at its true position in the full sequence), the computed tensors are
+ * concatenated with the loaded ones and the rest of the block proceeds normally.
+ * Tensors computed for chunks that were not cached are sliced per chunk and kept
+ * (Section 3.2.1, cache slicer).
+ *
+ * Deliberate differences from the paper's prototype, all documented in the design
+ * notes: only K and V are cached (bf16, 16-token pages, K stored before rotation
+ * and rotated to its slot's position when gathered); a chunk may hit at any place
+ * of the list, not only as part of a prefix; only the new rows (missed chunks and
+ * query tokens) continue through the blocks and are returned.
+ *
+ * General rules
+ *  - Every function returns 0 (PERCACHE_OK) or a negative PERCACHE_E_* code; nothing
+ *    throws or aborts across this boundary.  percache_strerror() names a code.
+ *  - A handle is not thread-safe.  All device work of a handle runs on the stream
+ *    given at creation; calls return after that work has finished.
+ *  - A call that fails leaves the store exactly as it was.
+ *  - The library never frees or keeps caller memory: every caller buffer may be
+ *    released as soon as the call returns.
+ *  - There is no CPU fallback: without a CUDA device every call that needs one fails
+ *    with PERCACHE_E_CUDA.
+ */
+#ifndef PERCACHE_H_
+#define PERCACHE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define PERCACHE_OK                 0
+#define PERCACHE_E_INVAL           -1   /* bad argument (NULL, negative size, unsupported shape)        */
+#define PERCACHE_E_NOMEM           -2   /* host or device allocation failed                            */
+#define PERCACHE_E_NOSPACE         -3   /* the paged store has too few free pages                      */
+#define PERCACHE_E_EXISTS          -4   /* chunk id already stored                                     */
+#define PERCACHE_E_LEN_MISMATCH    -5   /* chunk id stored with a different token count                */
+#define PERCACHE_E_MISS_NO_INPUT   -6   /* chunk is not stored and no hidden states were given for it  */
+#define PERCACHE_E_CAPACITY        -7   /* prompt / batch exceeds a limit fixed at creation            */
+#define PERCACHE_E_DEVICE_TIMEOUT  -8   /* a bounded wait inside a kernel ran out; results are invalid */
+#define PERCACHE_E_CUDA            -9   /* a CUDA runtime / driver call failed                         */
+#define PERCACHE_E_NOTFOUND        -10  /* chunk id not stored (has / drop)                            */
+
+#define PERCACHE_PAGE_TOKENS 16
+
+/* percache_config_t.flags */
+#define PERCACHE_FLAG_REFERENCE_KERNELS  1u  /* debugging aid: run every GEMM and the attention with the plain
+                                                one-thread-per-output CUDA kernels instead of the tcgen05 ones */
+#define PERCACHE_FLAG_PHASE_TIMING       2u  /* record CUDA events around every kernel class (see stats)       */
+
+typedef struct percache percache_t;   /* opaque */
+
+typedef struct {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn;
+  float   rope_theta, rms_eps;
+  int32_t page_tokens;              /* must be PERCACHE_PAGE_TOKENS                                         */
+  int64_t pool_pages;               /* capacity of the paged store, in pages (each page: 16 tokens, all
+                                       layers, K and V)                                                    */
+  int32_t max_prompt_tokens;        /* longest prompt (chunks + query); also the largest RoPE position + 1  */
+  int32_t max_batch_prompts;        /* most prompts in one percache_prefill call                            */
+  int64_t max_batch_ctx_tokens;     /* most context tokens (sum of prompt lengths) in one call              */
+  int64_t max_batch_new_rows;       /* most new rows (missed-chunk tokens + query tokens) in one call       */
+  int32_t device;                   /* CUDA device ordinal                                                  */
+  void*   stream;                   /* cudaStream_t of the caller, or NULL for the default stream           */
+  uint32_t flags;                   /* PERCACHE_FLAG_*                                                      */
+} percache_config_t;
+
+/* One layer's parameters: bf16, row-major [out_features][in_features] (norm gains: [d_model]).
+ * Host or device pointers (see weights_on_device); copied during percache_create. */
+typedef struct {
+  const void *attn_norm, *wq, *wk, *wv, *wo, *ffn_norm, *w_gate, *w_up, *w_down;
+} percache_layer_weights_t;
+
+/* Create a handle: allocates the paged store, work buffers and a private copy of the weights on
+ * cfg->device.  Supported shapes: head_dim 128; d_model, d_ffn multiples of 64; n_q_heads a multiple of
+ * n_kv_heads.  Device allocation failure -> PERCACHE_E_NOMEM; the handle is not created. */
+int percache_create(const percache_config_t* cfg, const percache_layer_weights_t* layers /*[n_layers]*/,
+                    int32_t weights_on_device, percache_t** out);
+
+/* Free everything the handle owns.  NULL is accepted. */
+int percache_destroy(percache_t* h);
+
+/* Insert a chunk's unrotated K and V for all layers (what a prefill of that chunk collected; paper
+ * Section 3.2.1).  k, v: bf16 [n_layers][n_tokens][n_kv_heads][head_dim], host or device memory as
+ * ptr_is_device says.  Copied into ceil(n_tokens/16) pages before return.  An id that is already stored
+ * is not overwritten: PERCACHE_E_EXISTS. */
+int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens,
+                          const void* k, const void* v, int32_t ptr_is_device);
+
+/* A prompt: ordered chunk list plus query tokens (paper Section 3, system overview). */
+typedef struct {
+  int32_t n_chunks;
+  const uint64_t* chunk_ids;            /* host [n_chunks]                                                 */
+  const int32_t*  chunk_len;            /* host [n_chunks], tokens per chunk (> 0)                          */
+  const void* const* chunk_hidden;      /* host [n_chunks] of pointers to bf16 [len][d_model] layer-0 input;
+                                           an entry (or the whole array) may be NULL for a chunk expected to
+                                           hit; NULL for a chunk that misses -> PERCACHE_E_MISS_NO_INPUT    */
+  int32_t n_query;                      /* >= 0                                                             */
+  const void* query_hidden;             /* bf16 [n_query][d_model]                                          */
+  int32_t hidden_on_device;             /* 1: chunk_hidden[i] and query_hidden point to device memory       */
+} percache_prompt_t;
+
+typedef struct {
+  float*   out_hidden;         /* caller-allocated fp32 [out_capacity_rows][d_model]: final residual stream of
+                                  the new rows, in prompt order (no final norm)                             */
+  int64_t  out_capacity_rows;  /* fewer than n_new -> PERCACHE_E_CAPACITY                                   */
+  int32_t  out_on_device;      /* 1: out_hidden is device memory                                            */
+  uint8_t* hit_mask;           /* caller-allocated host [n_chunks] or NULL; 1 = served from the store       */
+  int32_t  n_new, n_total;     /* written by the call: new rows and total context tokens of this prompt     */
+} percache_result_t;
+
+/* Reuse-prefill of a batch of independent prompts (paper Section 3.2.2, Appendix B.1).
+ * Hits are decided against the store as it is when the call starts: a chunk hits when its id is stored
+ * with the same length (different length -> PERCACHE_E_LEN_MISMATCH).  On success every missed chunk is
+ * stored (its K/V as computed inside its prompt; if two prompts of the batch miss the same id, the
+ * first prompt's is kept) and query tokens are not.  Too few free pages -> PERCACHE_E_NOSPACE.
+ * Synchronous: returns after the stream has drained. */
+int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
+                     percache_result_t* results /*[n_prompts]*/);
+
+/* *n_tokens = stored length, or PERCACHE_E_NOTFOUND. n_tokens may be NULL. */
+int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n_tokens);
+
+/* Remove a chunk and free its pages (used to restore the cache state between timed runs). */
+int percache_drop_chunk(percache_t* h, uint64_t chunk_id);
+
+/* Read a stored chunk back: k, v host buffers bf16 [n_layers][n_tokens][n_kv_heads][head_dim]. */
+int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* v_host);
+
+/* Fill a new chunk with the synthetic integer pool values of the batched-serving workload:
+ * element e of (chunk, which in {K=0,V=1}, layer) takes the 64-bit counter
+ *   ((((seed << 20) + chunk_id) * 2 + which) * 64 + layer) << 24) + e
+ * through the SplitMix64 output function, and the value (b0 + b1 + b2 + b3 - 126) / 64 with b_i the four
+ * lowest 6-bit fields of the result (exact in bf16).  Same errors as percache_put_chunk_kv. */
+int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tokens, uint64_t seed);
+
+/* Kernel classes for phase timing. */
+enum {
+  PERCACHE_PH_GATHER = 0,   /* gather + re-RoPE of hit tokens, all layers                */
+  PERCACHE_PH_NORM,         /* both RMSNorms                                              */
+  PERCACHE_PH_QKV,          /* QKV projection + RoPE + scatter                           */
+  PERCACHE_PH_ATTN,         /* causal GQA attention of the new rows                      */
+  PERCACHE_PH_OPROJ,        /* output projection + residual                              */
+  PERCACHE_PH_GATEUP,       /* gate/up projection + SwiGLU                               */
+  PERCACHE_PH_DOWN,         /* down projection + residual                                */
+  PERCACHE_PH_IO,           /* input staging and output copies                           */
+  PERCACHE_PH_COUNT
+};
+
+typedef struct {
+  /* last percache_prefill call */
+  int32_t n_prompts, chunks_hit, chunks_missed;
+  int64_t ctx_tokens, hit_tokens, new_rows;
+  int64_t pages_used, pages_free;
+  double  host_plan_us;                        /* lookup + page allocation + index assembly       */
+  double  device_us;                           /* first kernel start to last kernel end (events)  */
+  double  phase_us[PERCACHE_PH_COUNT];         /* filled when PERCACHE_FLAG_PHASE_TIMING is set   */
+  int32_t phase_launches[PERCACHE_PH_COUNT];   /* kernels launched per class (always filled)      */
+  int64_t attn_visible_pairs;                  /* sum over new rows of (position + 1)             */
+} percache_stats_t;
+
+int percache_get_stats(percache_t* h, percache_stats_t* out);
+
+/* Switch PERCACHE_FLAG_PHASE_TIMING / PERCACHE_FLAG_REFERENCE_KERNELS after creation. */
+int percache_set_flags(percache_t* h, uint32_t flags);
+
+/* Integer plan of the last successful percache_prefill (host int32 arrays, caller-allocated).
+ * which: 0 cu_ctx [n_prompts+1]; 1 cu_new [n_prompts+1]; 2 slot_chunk [ctx_tokens] (index into the prompt's
+ * chunk list, n_chunks for query tokens); 3 slot_offset [ctx_tokens]; 4 slot_is_new [ctx_tokens];
+ * 5 row_slot [new_rows] (slot of every new row inside its prompt = its position).
+ * Returns the number of elements written, or a negative code (PERCACHE_E_CAPACITY if capacity is short). */
+int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity);
+
+/* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
+ * [n_total][n_kv_heads][head_dim], copied to host buffers. */
+int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
+
+/* C[M][N] (fp32, host) = A[M][K] * B[N][K]^T with fp16 inputs (host), through the tcgen05 GEMM
+ * (use_reference = 0) or the plain kernel (1).  Test hook for the GEMM core. */
+int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
+                        float* c, int32_t use_reference);
+
+const char* percache_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* PERCACHE_H_ */
