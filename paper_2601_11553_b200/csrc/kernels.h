@@ -1,0 +1,112 @@
+// Internal interface between the host runtime and the CUDA kernels (not part of the C ABI).
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace pc {
+
+constexpr int PAGE_TOKENS = 16;
+constexpr int HEAD_DIM = 128;
+constexpr int ROPE_HALF = HEAD_DIM / 2;
+
+// One unit of gather work: up to 16 consecutive tokens of one stored page go to consecutive
+// context slots of one prompt.  `pos` is the position (slot inside the prompt) of the first token.
+struct GatherItem {
+  int32_t dst_slot;   // global context slot (prompts of a batch are laid out back to back)
+  int32_t src_page;   // page of the store
+  int32_t n_tok;      // 1..16
+  int32_t pos;        // RoPE position of the first token
+};
+
+// Per new row (device arrays of length M).
+struct RowIndex {
+  const int32_t* slot;      // global context slot of the row
+  const int32_t* pos;       // position inside its prompt
+  const int32_t* pool_tok;  // page * 16 + offset where the row's unrotated K/V is kept, or -1
+};
+
+// Attention work tile: up to 128 consecutive new rows of one prompt.
+struct AttnTile {
+  int32_t row0;       // first new row (global row index)
+  int32_t n_rows;     // 1..128
+  int32_t ctx0;       // global context slot of the prompt's slot 0
+  int32_t kv_len;     // context slots the tile can see: (position of its last row) + 1
+  int32_t min_pos;    // position of its first row
+  int32_t pad0, pad1, pad2;
+};
+
+struct ModelDims {
+  int32_t n_layers, d_model, n_q_heads, n_kv_heads, d_ffn;
+  int32_t q_dim, kv_dim, qkv_dim;
+  float rms_eps;
+};
+
+// ---- element-wise and memory-bound kernels (kernels_mem.cu)
+void launch_build_rope_table(float2* table, int max_pos, double theta, cudaStream_t s);
+void launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, int64_t n, cudaStream_t s);
+// dst[(2*b + which) * blk + r][:] = src_which[b * blk + r][:]  (gate/up row interleave in blocks of blk rows)
+void launch_interleave_rows_bf16_to_f16(const __nv_bfloat16* gate, const __nv_bfloat16* up, __half* dst, int rows,
+                                        int cols, int blk, cudaStream_t s);
+void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStream_t s);
+void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s);
+void launch_gather_rerope(const GatherItem* items, int n_items, int n_layers, const __nv_bfloat16* kpool,
+                          const __nv_bfloat16* vpool, int64_t pool_pages, __half* kctx, __half* vctx,
+                          int64_t ctx_cap, int kv_dim, const float2* rope, cudaStream_t s);
+// chunk [L][n][kv_dim] <-> pages (to_pool = 1: chunk -> pool)
+void launch_chunk_pages_copy(__nv_bfloat16* chunk, __nv_bfloat16* pool, const int32_t* pages, int n_tokens,
+                             int n_layers, int64_t pool_pages, int kv_dim, int to_pool, cudaStream_t s);
+void launch_fill_synthetic(__nv_bfloat16* kpool, __nv_bfloat16* vpool, const int32_t* pages, int n_tokens,
+                           int n_layers, int64_t pool_pages, int kv_dim, uint64_t seed, uint64_t chunk_id,
+                           cudaStream_t s);
+
+// ---- epilogue parameter blocks shared by the reference and the tcgen05 GEMMs
+struct QkvEpilogue {
+  RowIndex rows;
+  const float2* rope;
+  __half* q_out;              // [M][q_dim]
+  __nv_bfloat16* kpool;       // layer base: [pool_pages*16][kv_dim]
+  __nv_bfloat16* vpool;
+  __half* kctx;               // layer base: [ctx_cap][kv_dim]
+  __half* vctx;
+  int32_t n_q_heads, n_kv_heads;
+};
+struct ResidualEpilogue { float* resid; int32_t ld; };          // resid[row][col] += acc
+struct SwigluEpilogue { __half* act; int32_t ld; };             // act[row][j] = silu(gate) * up
+
+// ---- plain reference kernels (kernels_ref.cu)
+void launch_ref_gemm(const __half* A, const __half* B, float* C, int M, int N, int K, cudaStream_t s);
+void launch_ref_qkv_epilogue(const float* C, int M, const QkvEpilogue& e, cudaStream_t s);
+void launch_ref_residual_epilogue(const float* C, int M, int N, const ResidualEpilogue& e, cudaStream_t s);
+void launch_ref_swiglu_epilogue(const float* C, int M, int F, int blk, const SwigluEpilogue& e, cudaStream_t s);
+void launch_ref_attention(const __half* q, const __half* kctx, const __half* vctx, __half* out, const int32_t* row_pos,
+                          const int32_t* row_ctx0, int M, int n_q_heads, int n_kv_heads, cudaStream_t s);
+
+// ---- tcgen05 GEMM (gemm_umma.cu).  A [M][K] fp16 row-major, B [N][K] fp16 row-major, D = A * B^T.
+enum GemmEpilogueKind { EPI_STORE_F32 = 0, EPI_QKV = 1, EPI_RESIDUAL = 2, EPI_SWIGLU = 3 };
+struct GemmOperand {           // a tensor map made once for a fixed buffer
+  CUtensorMap map;
+};
+// rows x cols fp16 row-major matrix; box = box_rows x 64 columns, 128-byte swizzle
+int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t cols, int box_rows);
+int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
+                     GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
+                     cudaStream_t s);
+int umma_gemm_block_n(GemmEpilogueKind kind);    // block_n a B operand map must be built for
+
+// rank-N fp16 tensor map with 128-byte swizzle; dims/strides innermost first (strides in bytes, from dim 1)
+int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                   const uint32_t* box);
+
+// ---- tcgen05 attention (attn_umma.cu)
+struct AttnMaps { CUtensorMap q, k, v; };
+int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, const __half* kctx_layer,
+                   const __half* vctx_layer, int64_t ctx_cap, int kv_dim);
+int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
+                          __half* out, int n_q_heads, int n_kv_heads, int* err_word, int n_sms, cudaStream_t s);
+
+int init_driver_api();   // resolves cuTensorMapEncodeTiled once; 0 on success
+
+}  // namespace pc
