@@ -1,0 +1,315 @@
+// Dense GEMM on the 5th-generation tensor cores: D[M][N] = A[M][K] * B[N][K]^T, fp16 operands,
+// fp32 accumulation in TMEM, fused epilogues (QKV + RoPE + scatter, residual add, SwiGLU).
+//
+// One persistent CTA per SM, 192 threads, warp-specialised:
+//   warp 0    TMA producer: one lane streams 128x64 A tiles and BNx64 B tiles (128-byte swizzle) into
+//             a ring of shared-memory stages, signalling `full` mbarriers by transaction bytes;
+//   warp 1    owns the TMEM allocation; one lane issues tcgen05.mma (128 x BN x 16) on each stage and
+//             commits to the stage's `empty` barrier, then to the accumulator's `tmem_full` barrier;
+//   warps 2-5 epilogue: each reads its 32-lane quarter of the accumulator with tcgen05.ld, applies the
+//             epilogue and stores; two accumulator stages let the next tile's MMAs overlap it.
+// Every wait is bounded (ptx.cuh); on a timeout the roles fall through to the common teardown,
+// the producer gives its outstanding copies time to land, TMEM is freed and the host sees the error word.
+#include "epilogue.cuh"
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace pc {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;                       // 64 fp16 = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int GEMM_THREADS = 192;
+constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
+
+template <int BN> struct GemmCfg {
+  static constexpr int B_STAGE_BYTES = BN * BK * 2;
+  static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+  static constexpr int STAGES = (BN >= 256) ? 4 : 6;
+  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+  static constexpr int TMEM_COLS = 2 * BN;                         // two accumulator stages
+};
+
+struct GemmArgs {
+  int32_t M, N, K;
+  float* c;                  // EPI_STORE_F32
+  QkvEpilogue qkv;           // EPI_QKV
+  ResidualEpilogue res;      // EPI_RESIDUAL
+  SwigluEpilogue swi;        // EPI_SWIGLU
+  int* err_word;
+};
+
+__device__ __forceinline__ void u32x8_to_float(const uint32_t* r, float (&f)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[i]);
+}
+
+template <int BN, int KIND>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs args) {
+  using Cfg = GemmCfg<BN>;
+  constexpr int STAGES = Cfg::STAGES;
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t full_bar[STAGES];
+  __shared__ __align__(8) uint64_t empty_bar[STAGES];
+  __shared__ __align__(8) uint64_t tmem_full_bar[2];
+  __shared__ __align__(8) uint64_t tmem_empty_bar[2];
+  __shared__ uint32_t tmem_base_slot;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+
+  const int n_m_tiles = (args.M + BM - 1) / BM;
+  const int n_n_tiles = args.N / BN;
+  const int n_tiles = n_m_tiles * n_n_tiles;
+  const int n_kb = args.K / BK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 4); }
+    fence_mbar_init();
+  }
+  if (warp == 1) {
+    tmem_alloc<Cfg::TMEM_COLS>(&tmem_base_slot);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tmA);
+      prefetch_tmap(&tmB);
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+        const int m_idx = tile / n_n_tiles, n_idx = tile % n_n_tiles;
+        for (int kb = 0; kb < n_kb; ++kb) {
+          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
+          uint8_t* a_dst = ring + stage * Cfg::STAGE_BYTES;
+          uint8_t* b_dst = a_dst + A_STAGE_BYTES;
+          mbar_arrive_expect_tx(&full_bar[stage], Cfg::STAGE_BYTES);
+          tma_load_2d(a_dst, &tmA, &full_bar[stage], kb * BK, m_idx * BM);
+          tma_load_2d(b_dst, &tmB, &full_bar[stage], kb * BK, n_idx * BN);
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        // Error path only: give copies already issued time to land before shared memory is released.
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = make_idesc_f16(BM, BN, /*fp16*/ 0, 0, 0);
+      int stage = 0;
+      uint32_t phase = 0;
+      int it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+        const int acc = it & 1;
+        const uint32_t acc_phase = (it >> 1) & 1u;
+        if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+        for (int kb = 0; kb < n_kb; ++kb) {
+          if (!mbar_wait(&full_bar[stage], phase, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
+          tc_fence_after_sync();
+          const uint32_t a_addr = smem_u32(ring + stage * Cfg::STAGE_BYTES);
+          const uint32_t b_addr = a_addr + A_STAGE_BYTES;
+          const uint64_t a_desc = make_smem_desc_sw128(a_addr, 16, 1024);
+          const uint64_t b_desc = make_smem_desc_sw128(b_addr, 16, 1024);
+#pragma unroll
+          for (int k = 0; k < BK / UMMA_K; ++k) {
+            // 16 elements along K = 32 bytes = 2 units of the descriptor's 16-byte address field
+            umma_ss(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(2 * k), idesc,
+                    (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&empty_bar[stage]);      // stage reusable once these MMAs have read it
+          if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) umma_commit(&tmem_full_bar[acc]);
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter + 32)
+    const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+    int it = 0;
+    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
+      const int m_idx = tile / n_n_tiles, n_idx = tile % n_n_tiles;
+      const int acc = it & 1;
+      const uint32_t acc_phase = (it >> 1) & 1u;
+      bool ok = mbar_wait(&tmem_full_bar[acc], acc_phase, args.err_word, DEV_ERR_GEMM_EPILOGUE);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t t_acc = tmem_base + lane_base + static_cast<uint32_t>(acc * BN);
+      const int row = m_idx * BM + quarter * 32 + lane;
+      const bool row_ok = row < args.M;
+      if constexpr (KIND == EPI_STORE_F32 || KIND == EPI_RESIDUAL) {
+#pragma unroll 1
+        for (int c = 0; c < BN; c += 32) {
+          uint32_t r[32];
+          tmem_ld_32x32(t_acc + c, r);
+          tmem_wait_ld();
+          if (row_ok) {
+            const int col = n_idx * BN + c;
+            if constexpr (KIND == EPI_STORE_F32) {
+              float4* dst = reinterpret_cast<float4*>(args.c + static_cast<size_t>(row) * args.N + col);
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                                     __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            } else {
+#pragma unroll
+              for (int i = 0; i < 8; ++i)
+                residual_add4(args.res, row, col + 4 * i, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
+                              __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+            }
+          }
+        }
+      } else if constexpr (KIND == EPI_QKV) {
+#pragma unroll 1
+        for (int hl = 0; hl < BN / HEAD_DIM; ++hl) {
+          const int hb = n_idx * (BN / HEAD_DIM) + hl;
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            uint32_t rlo[32], rhi[32];
+            tmem_ld_32x32(t_acc + hl * HEAD_DIM + half * 32, rlo);
+            tmem_ld_32x32(t_acc + hl * HEAD_DIM + ROPE_HALF + half * 32, rhi);
+            tmem_wait_ld();
+            if (row_ok) {
+#pragma unroll
+              for (int seg = 0; seg < 4; ++seg) {
+                float lo[8], hi[8];
+                u32x8_to_float(rlo + seg * 8, lo);
+                u32x8_to_float(rhi + seg * 8, hi);
+                qkv_store8(args.qkv, row, hb, half * 32 + seg * 8, lo, hi);
+              }
+            }
+          }
+        }
+      } else {   // EPI_SWIGLU: tile columns [0, BN/2) are gate, [BN/2, BN) the matching up columns
+#pragma unroll 1
+        for (int c = 0; c < BN / 2; c += 32) {
+          uint32_t rg[32], ru[32];
+          tmem_ld_32x32(t_acc + c, rg);
+          tmem_ld_32x32(t_acc + BN / 2 + c, ru);
+          tmem_wait_ld();
+          if (row_ok) {
+#pragma unroll
+            for (int seg = 0; seg < 4; ++seg) {
+              float g[8], u[8];
+              u32x8_to_float(rg + seg * 8, g);
+              u32x8_to_float(ru + seg * 8, u);
+              swiglu_store8(args.swi, row, n_idx * (BN / 2) + c + seg * 8, g, u);
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown (every thread gets here)
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc<Cfg::TMEM_COLS>(tmem_base);
+  }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+
+template <int BN, int KIND>
+int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, int n_sms, cudaStream_t s) {
+  using Cfg = GemmCfg<BN>;
+  if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           Cfg::SMEM_BYTES) != cudaSuccess)
+    return -1;
+  const int n_tiles = ((args.M + BM - 1) / BM) * (args.N / BN);
+  if (n_tiles <= 0) return 0;
+  const int grid = n_tiles < n_sms ? n_tiles : n_sms;
+  umma_gemm_kernel<BN, KIND><<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, s>>>(A.map, B.map, args);
+  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+}
+
+}  // namespace
+
+int init_driver_api() {
+  if (g_encode) return 0;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess) return -1;
+  if (qres != cudaDriverEntryPointSuccess || fn == nullptr) return -1;
+  g_encode = reinterpret_cast<EncodeTiledFn>(fn);
+  return 0;
+}
+
+int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                   const uint32_t* box) {
+  if (init_driver_api() != 0) return -1;
+  cuuint64_t gdim[5];
+  cuuint64_t gstr[4];
+  cuuint32_t bx[5], es[5];
+  for (int i = 0; i < rank; ++i) { gdim[i] = dims[i]; bx[i] = box[i]; es[i] = 1; }
+  for (int i = 0; i + 1 < rank; ++i) gstr[i] = strides_bytes[i];
+  const CUresult r = g_encode(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, static_cast<cuuint32_t>(rank),
+                              const_cast<void*>(base), gdim, gstr, bx, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                              CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? 0 : -1;
+}
+
+int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t cols, int box_rows) {
+  const uint64_t dims[2] = {static_cast<uint64_t>(cols), static_cast<uint64_t>(rows)};
+  const uint64_t strides[1] = {static_cast<uint64_t>(cols) * 2};
+  const uint32_t box[2] = {static_cast<uint32_t>(BK), static_cast<uint32_t>(box_rows)};
+  return encode_f16_map(&out->map, base, 2, dims, strides, box);
+}
+
+int umma_gemm_block_n(GemmEpilogueKind kind) {
+  (void)kind;
+  return 128;
+}
+
+int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
+                     GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
+                     cudaStream_t s) {
+  if (M <= 0) return 0;
+  if (K % BK != 0 || N % block_n != 0 || block_n != 128) return -1;
+  GemmArgs args{};
+  args.M = M; args.N = N; args.K = K; args.c = c_f32; args.err_word = err_word;
+  switch (kind) {
+    case EPI_STORE_F32:
+      return launch_one<128, EPI_STORE_F32>(A, B, args, n_sms, s);
+    case EPI_QKV:
+      args.qkv = *static_cast<const QkvEpilogue*>(epilogue);
+      return launch_one<128, EPI_QKV>(A, B, args, n_sms, s);
+    case EPI_RESIDUAL:
+      args.res = *static_cast<const ResidualEpilogue*>(epilogue);
+      return launch_one<128, EPI_RESIDUAL>(A, B, args, n_sms, s);
+    case EPI_SWIGLU:
+      args.swi = *static_cast<const SwigluEpilogue*>(epilogue);
+      return launch_one<128, EPI_SWIGLU>(A, B, args, n_sms, s);
+  }
+  return -1;
+}
+
+}  // namespace pc
