@@ -1,0 +1,827 @@
+// Host runtime behind the C ABI: paged store (free list + chunk table), per-call integer plan
+// (hit test, page allocation, slot/position/row arrays, gather items, attention tiles), kernel
+// launches on the caller's stream, commit of missed chunks after success.
+#include <algorithm>
+#include <chrono>
+#include <cstring>
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/percache.h"
+#include "kernels.h"
+
+using namespace pc;
+
+namespace {
+
+struct ChunkEntry {
+  int32_t n_tokens;
+  std::vector<int32_t> pages;
+};
+
+struct LayerWeights {
+  __half *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr;
+  float *g_attn = nullptr, *g_ffn = nullptr;
+  GemmOperand m_wqkv, m_wo, m_wgu, m_wd;
+  AttnMaps attn_maps;
+};
+
+struct Plan {   // integer description of the last successful call (host)
+  std::vector<int32_t> cu_ctx, cu_new, slot_chunk, slot_offset, slot_is_new, row_slot;
+};
+
+constexpr int MAX_EVENTS = 1024;
+
+}  // namespace
+
+struct percache {
+  percache_config_t cfg{};
+  ModelDims dims{};
+  cudaStream_t stream = nullptr;
+  int n_sms = 148;
+  uint32_t flags = 0;
+  int gu_blk = 64;                          // gate/up interleave block (half the GEMM's N tile)
+
+  std::vector<void*> dev_allocs;
+  std::vector<LayerWeights> layers;
+  float2* rope = nullptr;
+  __nv_bfloat16 *kpool = nullptr, *vpool = nullptr;    // [L][pool_pages][16][kv_dim]
+  __half *kctx = nullptr, *vctx = nullptr;              // [L][ctx_cap][kv_dim]
+  float* resid = nullptr;                               // [m_cap][d]
+  __nv_bfloat16* xin = nullptr;                         // [m_cap][d]
+  __half *xn = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr;
+  float* cref = nullptr;                                // reference kernels only
+  GemmOperand m_xn, m_attn, m_act;
+  int64_t m_cap = 0, ctx_cap = 0;
+
+  // index block: host (pinned) mirror and device copy
+  int32_t* h_index = nullptr;
+  int32_t* d_index = nullptr;
+  size_t index_ints = 0;
+  int* d_err = nullptr;
+  int* h_err = nullptr;
+
+  std::unordered_map<uint64_t, ChunkEntry> table;
+  std::vector<int32_t> free_pages;
+
+  Plan plan;
+  percache_stats_t stats{};
+  std::vector<cudaEvent_t> events;
+  cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+};
+
+namespace {
+
+template <typename T>
+bool dev_alloc(percache* h, T** out, size_t count) {
+  void* p = nullptr;
+  if (cudaMalloc(&p, std::max<size_t>(count * sizeof(T), 256)) != cudaSuccess) {
+    cudaGetLastError();
+    return false;
+  }
+  h->dev_allocs.push_back(p);
+  *out = static_cast<T*>(p);
+  return true;
+}
+
+void destroy_impl(percache* h) {
+  if (!h) return;
+  cudaSetDevice(h->cfg.device);
+  cudaStreamSynchronize(h->stream);
+  for (void* p : h->dev_allocs) cudaFree(p);
+  if (h->h_index) cudaFreeHost(h->h_index);
+  if (h->h_err) cudaFreeHost(h->h_err);
+  for (cudaEvent_t e : h->events)
+    if (e) cudaEventDestroy(e);
+  if (h->ev_begin) cudaEventDestroy(h->ev_begin);
+  if (h->ev_end) cudaEventDestroy(h->ev_end);
+  cudaGetLastError();
+  delete h;
+}
+
+// a bf16 matrix that may live on the host: copy to `tmp` on the device if so; returns what to read
+const __nv_bfloat16* stage_bf16(const void* src, size_t elems, int on_device, __nv_bfloat16* tmp, cudaStream_t s,
+                                bool* ok) {
+  if (on_device) return static_cast<const __nv_bfloat16*>(src);
+  if (cudaMemcpyAsync(tmp, src, elems * 2, cudaMemcpyHostToDevice, s) != cudaSuccess) *ok = false;
+  return tmp;
+}
+
+struct PhaseTimer {
+  percache* h;
+  bool on;
+  size_t next = 0;
+  std::vector<int> phase_of;
+  explicit PhaseTimer(percache* hh) : h(hh), on((hh->flags & PERCACHE_FLAG_PHASE_TIMING) != 0) {}
+  bool room() const { return on && next + 2 <= h->events.size(); }
+  void begin(int phase) {
+    h->stats.phase_launches[phase]++;
+    if (!room()) return;
+    cudaEventRecord(h->events[next], h->stream);
+    phase_of.push_back(phase);
+  }
+  void end() {
+    if (!room()) return;
+    cudaEventRecord(h->events[next + 1], h->stream);
+    next += 2;
+  }
+  void collect() {
+    for (size_t i = 0; i < next; i += 2) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, h->events[i], h->events[i + 1]) == cudaSuccess)
+        h->stats.phase_us[phase_of[i / 2]] += 1000.0 * ms;
+    }
+  }
+};
+
+int alloc_pages(percache* h, int n, std::vector<int32_t>* out) {
+  if (static_cast<size_t>(n) > h->free_pages.size()) return PERCACHE_E_NOSPACE;
+  for (int i = 0; i < n; ++i) {
+    out->push_back(h->free_pages.back());
+    h->free_pages.pop_back();
+  }
+  return PERCACHE_OK;
+}
+void release_pages(percache* h, const std::vector<int32_t>& pages) {
+  for (auto p = pages.rbegin(); p != pages.rend(); ++p) h->free_pages.push_back(*p);
+}
+void refresh_page_stats(percache* h) {
+  h->stats.pages_free = static_cast<int64_t>(h->free_pages.size());
+  h->stats.pages_used = h->cfg.pool_pages - h->stats.pages_free;
+}
+
+// upload a page list through the pinned index block and run `fn` with the device pointer
+template <typename Fn>
+int with_chunk_pages(percache* h, const std::vector<int32_t>& pages, Fn fn) {
+  if (pages.size() > h->index_ints) return PERCACHE_E_CAPACITY;
+  std::memcpy(h->h_index, pages.data(), pages.size() * sizeof(int32_t));
+  if (cudaMemcpyAsync(h->d_index, h->h_index, pages.size() * sizeof(int32_t), cudaMemcpyHostToDevice, h->stream) !=
+      cudaSuccess)
+    return PERCACHE_E_CUDA;
+  fn(h->d_index);
+  if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) return PERCACHE_E_CUDA;
+  return PERCACHE_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* percache_strerror(int code) {
+  switch (code) {
+    case PERCACHE_OK: return "ok";
+    case PERCACHE_E_INVAL: return "invalid argument";
+    case PERCACHE_E_NOMEM: return "out of memory";
+    case PERCACHE_E_NOSPACE: return "paged store is full";
+    case PERCACHE_E_EXISTS: return "chunk id already stored";
+    case PERCACHE_E_LEN_MISMATCH: return "chunk stored with a different length";
+    case PERCACHE_E_MISS_NO_INPUT: return "chunk not stored and no hidden states given";
+    case PERCACHE_E_CAPACITY: return "capacity fixed at creation exceeded";
+    case PERCACHE_E_DEVICE_TIMEOUT: return "bounded wait inside a kernel ran out";
+    case PERCACHE_E_CUDA: return "CUDA call failed";
+    case PERCACHE_E_NOTFOUND: return "chunk id not stored";
+    default: return "unknown error";
+  }
+}
+
+int percache_create(const percache_config_t* cfg, const percache_layer_weights_t* lw, int32_t weights_on_device,
+                    percache_t** out) {
+  if (!cfg || !lw || !out) return PERCACHE_E_INVAL;
+  *out = nullptr;
+  if (cfg->n_layers <= 0 || cfg->n_layers > 64 || cfg->head_dim != HEAD_DIM || cfg->page_tokens != PAGE_TOKENS ||
+      cfg->d_model <= 0 || cfg->d_model % 128 != 0 || cfg->d_ffn <= 0 || cfg->d_ffn % 64 != 0 ||
+      cfg->n_kv_heads <= 0 || cfg->n_q_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads != 0 ||
+      cfg->pool_pages <= 0 || cfg->max_prompt_tokens <= 0 || cfg->max_batch_prompts <= 0 ||
+      cfg->max_batch_ctx_tokens <= 0 || cfg->max_batch_new_rows <= 0 || cfg->pool_pages > (INT32_MAX / PAGE_TOKENS) ||
+      cfg->max_batch_ctx_tokens > INT32_MAX / 2 || cfg->max_batch_new_rows > INT32_MAX / 2)
+    return PERCACHE_E_INVAL;
+  for (int l = 0; l < cfg->n_layers; ++l) {
+    const percache_layer_weights_t& S = lw[l];
+    if (!S.attn_norm || !S.wq || !S.wk || !S.wv || !S.wo || !S.ffn_norm || !S.w_gate || !S.w_up || !S.w_down)
+      return PERCACHE_E_INVAL;
+  }
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || cfg->device < 0 || cfg->device >= n_dev) {
+    cudaGetLastError();
+    return PERCACHE_E_CUDA;
+  }
+  if (cudaSetDevice(cfg->device) != cudaSuccess) return PERCACHE_E_CUDA;
+  if (init_driver_api() != 0) return PERCACHE_E_CUDA;
+
+  percache* h = new (std::nothrow) percache();
+  if (!h) return PERCACHE_E_NOMEM;
+  h->cfg = *cfg;
+  h->stream = static_cast<cudaStream_t>(cfg->stream);
+  h->flags = cfg->flags;
+  ModelDims& D = h->dims;
+  D.n_layers = cfg->n_layers; D.d_model = cfg->d_model; D.n_q_heads = cfg->n_q_heads; D.n_kv_heads = cfg->n_kv_heads;
+  D.d_ffn = cfg->d_ffn; D.q_dim = cfg->n_q_heads * HEAD_DIM; D.kv_dim = cfg->n_kv_heads * HEAD_DIM;
+  D.qkv_dim = D.q_dim + 2 * D.kv_dim; D.rms_eps = cfg->rms_eps;
+  h->m_cap = cfg->max_batch_new_rows;
+  h->ctx_cap = cfg->max_batch_ctx_tokens;
+  cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device);
+  h->gu_blk = umma_gemm_block_n(EPI_SWIGLU) / 2;
+
+  const int L = D.n_layers, d = D.d_model, F = D.d_ffn;
+  bool ok = true;
+  const size_t pool_elems = static_cast<size_t>(L) * cfg->pool_pages * PAGE_TOKENS * D.kv_dim;
+  const size_t ctx_elems = static_cast<size_t>(L) * h->ctx_cap * D.kv_dim;
+  ok = ok && dev_alloc(h, &h->kpool, pool_elems) && dev_alloc(h, &h->vpool, pool_elems);
+  ok = ok && dev_alloc(h, &h->kctx, ctx_elems) && dev_alloc(h, &h->vctx, ctx_elems);
+  ok = ok && dev_alloc(h, &h->rope, static_cast<size_t>(cfg->max_prompt_tokens) * ROPE_HALF);
+  ok = ok && dev_alloc(h, &h->resid, static_cast<size_t>(h->m_cap) * d);
+  ok = ok && dev_alloc(h, &h->xin, static_cast<size_t>(h->m_cap) * d);
+  ok = ok && dev_alloc(h, &h->xn, static_cast<size_t>(h->m_cap) * d);
+  ok = ok && dev_alloc(h, &h->qbuf, static_cast<size_t>(h->m_cap) * D.q_dim);
+  ok = ok && dev_alloc(h, &h->attn_out, static_cast<size_t>(h->m_cap) * D.q_dim);
+  ok = ok && dev_alloc(h, &h->act, static_cast<size_t>(h->m_cap) * F);
+  ok = ok && dev_alloc(h, &h->d_err, 1);
+  // index block: 4 row arrays + gather items (worst case one per context token) + attention tiles
+  const size_t max_tiles = static_cast<size_t>(h->m_cap / 128 + cfg->max_batch_prompts + 2);
+  h->index_ints = 4 * static_cast<size_t>(h->m_cap) + 4 * static_cast<size_t>(h->ctx_cap) + 8 * max_tiles;
+  ok = ok && dev_alloc(h, &h->d_index, h->index_ints);
+  if (ok && cudaMallocHost(reinterpret_cast<void**>(&h->h_index), h->index_ints * sizeof(int32_t)) != cudaSuccess) ok = false;
+  if (ok && cudaMallocHost(reinterpret_cast<void**>(&h->h_err), sizeof(int)) != cudaSuccess) ok = false;
+  h->layers.resize(L);
+  for (int l = 0; ok && l < L; ++l) {
+    LayerWeights& W = h->layers[l];
+    ok = ok && dev_alloc(h, &W.wqkv, static_cast<size_t>(D.qkv_dim) * d) && dev_alloc(h, &W.wo, static_cast<size_t>(d) * D.q_dim) &&
+         dev_alloc(h, &W.wgu, static_cast<size_t>(2 * F) * d) && dev_alloc(h, &W.wd, static_cast<size_t>(d) * F) &&
+         dev_alloc(h, &W.g_attn, d) && dev_alloc(h, &W.g_ffn, d);
+  }
+  if (!ok) {
+    cudaGetLastError();
+    destroy_impl(h);
+    return PERCACHE_E_NOMEM;
+  }
+  if (cudaEventCreate(&h->ev_begin) != cudaSuccess || cudaEventCreate(&h->ev_end) != cudaSuccess) {
+    destroy_impl(h);
+    return PERCACHE_E_CUDA;
+  }
+  h->events.assign(MAX_EVENTS, nullptr);
+  for (auto& e : h->events)
+    if (cudaEventCreate(&e) != cudaSuccess) { destroy_impl(h); return PERCACHE_E_CUDA; }
+
+  // ---- weights: bf16 -> fp16 copies in the layouts the GEMMs read.  Every bf16 value of magnitude
+  // >= 2^-17 is exactly representable in fp16; smaller ones round with absolute error <= 2^-25.
+  cudaStream_t s = h->stream;
+  __nv_bfloat16 *tmp0 = nullptr, *tmp1 = nullptr;
+  const size_t max_w = std::max<size_t>(static_cast<size_t>(F) * d, static_cast<size_t>(D.q_dim) * d);
+  bool cuda_ok = true;
+  if (!weights_on_device) {
+    if (cudaMalloc(reinterpret_cast<void**>(&tmp0), max_w * 2) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&tmp1), max_w * 2) != cudaSuccess) {
+      cudaGetLastError();
+      if (tmp0) cudaFree(tmp0);
+      destroy_impl(h);
+      return PERCACHE_E_NOMEM;
+    }
+  }
+  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
+  for (int l = 0; l < L && cuda_ok; ++l) {
+    LayerWeights& W = h->layers[l];
+    const percache_layer_weights_t& S = lw[l];
+    const __nv_bfloat16* p;
+    // stream order keeps each conversion ahead of the next copy into the same staging buffer
+    p = stage_bf16(S.wq, static_cast<size_t>(D.q_dim) * d, weights_on_device, tmp0, s, &cuda_ok);
+    launch_bf16_to_f16(p, W.wqkv, static_cast<int64_t>(D.q_dim) * d, s);
+    p = stage_bf16(S.wk, static_cast<size_t>(D.kv_dim) * d, weights_on_device, tmp1, s, &cuda_ok);
+    launch_bf16_to_f16(p, W.wqkv + static_cast<size_t>(D.q_dim) * d, static_cast<int64_t>(D.kv_dim) * d, s);
+    p = stage_bf16(S.wv, static_cast<size_t>(D.kv_dim) * d, weights_on_device, tmp0, s, &cuda_ok);
+    launch_bf16_to_f16(p, W.wqkv + static_cast<size_t>(D.q_dim + D.kv_dim) * d, static_cast<int64_t>(D.kv_dim) * d, s);
+    p = stage_bf16(S.wo, static_cast<size_t>(d) * D.q_dim, weights_on_device, tmp1, s, &cuda_ok);
+    launch_bf16_to_f16(p, W.wo, static_cast<int64_t>(d) * D.q_dim, s);
+    const __nv_bfloat16* pg = stage_bf16(S.w_gate, static_cast<size_t>(F) * d, weights_on_device, tmp0, s, &cuda_ok);
+    const __nv_bfloat16* pu = stage_bf16(S.w_up, static_cast<size_t>(F) * d, weights_on_device, tmp1, s, &cuda_ok);
+    launch_interleave_rows_bf16_to_f16(pg, pu, W.wgu, F, d, h->gu_blk, s);
+    p = stage_bf16(S.w_down, static_cast<size_t>(d) * F, weights_on_device, tmp0, s, &cuda_ok);
+    launch_bf16_to_f16(p, W.wd, static_cast<int64_t>(d) * F, s);
+    p = stage_bf16(S.attn_norm, d, weights_on_device, tmp1, s, &cuda_ok);
+    launch_bf16_to_f32(p, W.g_attn, d, s);
+    p = stage_bf16(S.ffn_norm, d, weights_on_device, tmp0, s, &cuda_ok);
+    launch_bf16_to_f32(p, W.g_ffn, d, s);
+    const int bn = umma_gemm_block_n(EPI_QKV);
+    cuda_ok = cuda_ok && make_operand_map(&W.m_wqkv, W.wqkv, D.qkv_dim, d, bn) == 0 &&
+              make_operand_map(&W.m_wo, W.wo, d, D.q_dim, bn) == 0 &&
+              make_operand_map(&W.m_wgu, W.wgu, 2 * F, d, bn) == 0 && make_operand_map(&W.m_wd, W.wd, d, F, bn) == 0;
+    cuda_ok = cuda_ok && make_attn_maps(&W.attn_maps, h->qbuf, h->m_cap, D.q_dim, h->kctx + l * ctx_layer,
+                                        h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim) == 0;
+  }
+  launch_build_rope_table(h->rope, cfg->max_prompt_tokens, static_cast<double>(cfg->rope_theta), s);
+  cuda_ok = cuda_ok && make_operand_map(&h->m_xn, h->xn, h->m_cap, d, 128) == 0 &&
+            make_operand_map(&h->m_attn, h->attn_out, h->m_cap, D.q_dim, 128) == 0 &&
+            make_operand_map(&h->m_act, h->act, h->m_cap, F, 128) == 0;
+  if (cudaStreamSynchronize(s) != cudaSuccess) cuda_ok = false;
+  if (tmp0) cudaFree(tmp0);
+  if (tmp1) cudaFree(tmp1);
+  if (!cuda_ok || cudaGetLastError() != cudaSuccess) {
+    destroy_impl(h);
+    return PERCACHE_E_CUDA;
+  }
+  h->free_pages.resize(static_cast<size_t>(cfg->pool_pages));
+  for (int64_t i = 0; i < cfg->pool_pages; ++i)
+    h->free_pages[static_cast<size_t>(i)] = static_cast<int32_t>(cfg->pool_pages - 1 - i);   // pops give 0, 1, 2, ...
+  refresh_page_stats(h);
+  *out = h;
+  return PERCACHE_OK;
+}
+
+int percache_destroy(percache_t* h) {
+  destroy_impl(h);
+  return PERCACHE_OK;
+}
+
+int percache_set_flags(percache_t* h, uint32_t flags) {
+  if (!h) return PERCACHE_E_INVAL;
+  h->flags = flags;
+  return PERCACHE_OK;
+}
+
+int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n_tokens) {
+  if (!h) return PERCACHE_E_INVAL;
+  auto it = h->table.find(chunk_id);
+  if (it == h->table.end()) return PERCACHE_E_NOTFOUND;
+  if (n_tokens) *n_tokens = it->second.n_tokens;
+  return PERCACHE_OK;
+}
+
+int percache_drop_chunk(percache_t* h, uint64_t chunk_id) {
+  if (!h) return PERCACHE_E_INVAL;
+  auto it = h->table.find(chunk_id);
+  if (it == h->table.end()) return PERCACHE_E_NOTFOUND;
+  release_pages(h, it->second.pages);
+  h->table.erase(it);
+  refresh_page_stats(h);
+  return PERCACHE_OK;
+}
+
+int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, const void* k, const void* v,
+                          int32_t ptr_is_device) {
+  if (!h || !k || !v || n_tokens <= 0) return PERCACHE_E_INVAL;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
+  const int n_pages = (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
+  ChunkEntry ent;
+  ent.n_tokens = n_tokens;
+  int rc = alloc_pages(h, n_pages, &ent.pages);
+  if (rc != PERCACHE_OK) return rc;
+  const size_t elems = static_cast<size_t>(h->dims.n_layers) * n_tokens * h->dims.kv_dim;
+  __nv_bfloat16 *dk = nullptr, *dv = nullptr;
+  if (!ptr_is_device) {
+    if (cudaMalloc(reinterpret_cast<void**>(&dk), elems * 2) != cudaSuccess ||
+        cudaMalloc(reinterpret_cast<void**>(&dv), elems * 2) != cudaSuccess) {
+      cudaGetLastError();
+      if (dk) cudaFree(dk);
+      release_pages(h, ent.pages);
+      return PERCACHE_E_NOMEM;
+    }
+    if (cudaMemcpyAsync(dk, k, elems * 2, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
+        cudaMemcpyAsync(dv, v, elems * 2, cudaMemcpyHostToDevice, h->stream) != cudaSuccess)
+      rc = PERCACHE_E_CUDA;
+  } else {
+    dk = static_cast<__nv_bfloat16*>(const_cast<void*>(k));
+    dv = static_cast<__nv_bfloat16*>(const_cast<void*>(v));
+  }
+  if (rc == PERCACHE_OK)
+    rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
+      launch_chunk_pages_copy(dk, h->kpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 1,
+                              h->stream);
+      launch_chunk_pages_copy(dv, h->vpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 1,
+                              h->stream);
+    });
+  if (!ptr_is_device) { cudaFree(dk); cudaFree(dv); }
+  if (rc != PERCACHE_OK) { release_pages(h, ent.pages); return rc; }
+  h->table.emplace(chunk_id, std::move(ent));
+  refresh_page_stats(h);
+  return PERCACHE_OK;
+}
+
+int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tokens, uint64_t seed) {
+  if (!h || n_tokens <= 0) return PERCACHE_E_INVAL;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
+  ChunkEntry ent;
+  ent.n_tokens = n_tokens;
+  int rc = alloc_pages(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
+  if (rc != PERCACHE_OK) return rc;
+  rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
+    launch_fill_synthetic(h->kpool, h->vpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim,
+                          seed, chunk_id, h->stream);
+  });
+  if (rc != PERCACHE_OK) { release_pages(h, ent.pages); return rc; }
+  h->table.emplace(chunk_id, std::move(ent));
+  refresh_page_stats(h);
+  return PERCACHE_OK;
+}
+
+int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* v_host) {
+  if (!h || !k_host || !v_host) return PERCACHE_E_INVAL;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  auto it = h->table.find(chunk_id);
+  if (it == h->table.end()) return PERCACHE_E_NOTFOUND;
+  const ChunkEntry& ent = it->second;
+  const size_t elems = static_cast<size_t>(h->dims.n_layers) * ent.n_tokens * h->dims.kv_dim;
+  __nv_bfloat16 *dk = nullptr, *dv = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&dk), elems * 2) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&dv), elems * 2) != cudaSuccess) {
+    cudaGetLastError();
+    if (dk) cudaFree(dk);
+    return PERCACHE_E_NOMEM;
+  }
+  int rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
+    launch_chunk_pages_copy(dk, h->kpool, d_pages, ent.n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 0,
+                            h->stream);
+    launch_chunk_pages_copy(dv, h->vpool, d_pages, ent.n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 0,
+                            h->stream);
+  });
+  if (rc == PERCACHE_OK && (cudaMemcpy(k_host, dk, elems * 2, cudaMemcpyDeviceToHost) != cudaSuccess ||
+                            cudaMemcpy(v_host, dv, elems * 2, cudaMemcpyDeviceToHost) != cudaSuccess))
+    rc = PERCACHE_E_CUDA;
+  cudaFree(dk);
+  cudaFree(dv);
+  return rc;
+}
+
+int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts, percache_result_t* results) {
+  if (!h || !prompts || !results || n_prompts <= 0) return PERCACHE_E_INVAL;
+  if (n_prompts > h->cfg.max_batch_prompts) return PERCACHE_E_CAPACITY;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  const auto t_host0 = std::chrono::steady_clock::now();
+  const ModelDims& D = h->dims;
+  const int d = D.d_model;
+
+  // ---------------------------------------------------------------- lookup, sizes
+  struct Seg { const void* src; int on_device; int row0; int n; };   // input rows to stage
+  std::vector<Seg> segs;
+  std::vector<std::vector<uint8_t>> hit(n_prompts);
+  std::unordered_map<uint64_t, std::pair<int, int>> first_miss;      // id -> (prompt, chunk) that will store it
+  Plan plan;
+  plan.cu_ctx.assign(1, 0);
+  plan.cu_new.assign(1, 0);
+  int64_t ctx_total = 0, new_total = 0, hit_tokens = 0, pages_needed = 0, visible_pairs = 0;
+  int chunks_hit = 0, chunks_missed = 0;
+  for (int b = 0; b < n_prompts; ++b) {
+    const percache_prompt_t& P = prompts[b];
+    if (P.n_chunks < 0 || P.n_query < 0 || (P.n_chunks > 0 && (!P.chunk_ids || !P.chunk_len)) ||
+        (P.n_query > 0 && !P.query_hidden))
+      return PERCACHE_E_INVAL;
+    hit[b].assign(static_cast<size_t>(P.n_chunks), 0);
+    int64_t T = 0, n_new = 0;
+    for (int i = 0; i < P.n_chunks; ++i) {
+      const int len = P.chunk_len[i];
+      if (len <= 0) return PERCACHE_E_INVAL;
+      auto it = h->table.find(P.chunk_ids[i]);
+      if (it != h->table.end()) {
+        if (it->second.n_tokens != len) return PERCACHE_E_LEN_MISMATCH;
+        hit[b][i] = 1;
+        ++chunks_hit;
+        hit_tokens += len;
+      } else {
+        if (!P.chunk_hidden || !P.chunk_hidden[i]) return PERCACHE_E_MISS_NO_INPUT;
+        ++chunks_missed;
+        n_new += len;
+        if (!first_miss.count(P.chunk_ids[i])) {
+          first_miss.emplace(P.chunk_ids[i], std::make_pair(b, i));
+          pages_needed += (len + PAGE_TOKENS - 1) / PAGE_TOKENS;
+        }
+      }
+      T += len;
+    }
+    T += P.n_query;
+    n_new += P.n_query;
+    if (T <= 0) return PERCACHE_E_INVAL;
+    if (T > h->cfg.max_prompt_tokens) return PERCACHE_E_CAPACITY;
+    if (results[b].out_capacity_rows < n_new || (n_new > 0 && !results[b].out_hidden)) return PERCACHE_E_CAPACITY;
+    ctx_total += T;
+    new_total += n_new;
+    if (ctx_total > h->ctx_cap || new_total > h->m_cap) return PERCACHE_E_CAPACITY;
+    plan.cu_ctx.push_back(static_cast<int32_t>(ctx_total));
+    plan.cu_new.push_back(static_cast<int32_t>(new_total));
+  }
+  if (pages_needed > static_cast<int64_t>(h->free_pages.size())) return PERCACHE_E_NOSPACE;
+
+  // ---------------------------------------------------------------- pages for the chunks that will be stored
+  std::vector<std::pair<uint64_t, ChunkEntry>> pending;
+  std::vector<int32_t> all_new_pages;
+  std::unordered_map<uint64_t, size_t> pending_of;
+  for (int b = 0; b < n_prompts; ++b)
+    for (int i = 0; i < prompts[b].n_chunks; ++i) {
+      if (hit[b][i]) continue;
+      const uint64_t id = prompts[b].chunk_ids[i];
+      auto fm = first_miss.find(id);
+      if (fm->second.first != b || fm->second.second != i) continue;
+      ChunkEntry ent;
+      ent.n_tokens = prompts[b].chunk_len[i];
+      alloc_pages(h, (ent.n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
+      all_new_pages.insert(all_new_pages.end(), ent.pages.begin(), ent.pages.end());
+      pending_of.emplace(id, pending.size());
+      pending.emplace_back(id, std::move(ent));
+    }
+  auto fail = [&](int code) {
+    release_pages(h, all_new_pages);
+    return code;
+  };
+
+  // ---------------------------------------------------------------- index assembly
+  const int64_t M = new_total;
+  int32_t* row_slot = h->h_index;
+  int32_t* row_pos = row_slot + h->m_cap;
+  int32_t* row_pool = row_pos + h->m_cap;
+  int32_t* row_ctx0 = row_pool + h->m_cap;
+  GatherItem* items = reinterpret_cast<GatherItem*>(row_ctx0 + h->m_cap);
+  AttnTile* tiles = reinterpret_cast<AttnTile*>(reinterpret_cast<int32_t*>(items) + 4 * h->ctx_cap);
+  int n_items = 0, n_tiles = 0;
+  plan.slot_chunk.resize(static_cast<size_t>(ctx_total));
+  plan.slot_offset.resize(static_cast<size_t>(ctx_total));
+  plan.slot_is_new.resize(static_cast<size_t>(ctx_total));
+  plan.row_slot.resize(static_cast<size_t>(M));
+  int64_t r = 0;
+  for (int b = 0; b < n_prompts; ++b) {
+    const percache_prompt_t& P = prompts[b];
+    const int32_t ctx0 = plan.cu_ctx[b];
+    int32_t t = 0;
+    for (int i = 0; i <= P.n_chunks; ++i) {
+      const bool is_query = (i == P.n_chunks);
+      const int len = is_query ? P.n_query : P.chunk_len[i];
+      if (len == 0) continue;
+      const bool is_hit = !is_query && hit[b][i];
+      for (int o = 0; o < len; ++o) {
+        plan.slot_chunk[ctx0 + t + o] = i;
+        plan.slot_offset[ctx0 + t + o] = o;
+        plan.slot_is_new[ctx0 + t + o] = is_hit ? 0 : 1;
+      }
+      if (is_hit) {
+        const ChunkEntry& ent = h->table.find(P.chunk_ids[i])->second;
+        for (int o = 0; o < len; o += PAGE_TOKENS) {
+          GatherItem& g = items[n_items++];
+          g.dst_slot = ctx0 + t + o;
+          g.src_page = ent.pages[o / PAGE_TOKENS];
+          g.n_tok = std::min(PAGE_TOKENS, len - o);
+          g.pos = t + o;
+        }
+      } else {
+        const ChunkEntry* ent = nullptr;
+        if (!is_query) {
+          auto fm = first_miss.find(P.chunk_ids[i]);
+          if (fm->second.first == b && fm->second.second == i) ent = &pending[pending_of[P.chunk_ids[i]]].second;
+        }
+        segs.push_back(Seg{is_query ? P.query_hidden : P.chunk_hidden[i], P.hidden_on_device, static_cast<int>(r), len});
+        for (int o = 0; o < len; ++o, ++r) {
+          row_slot[r] = ctx0 + t + o;
+          row_pos[r] = t + o;
+          row_pool[r] = ent ? ent->pages[o / PAGE_TOKENS] * PAGE_TOKENS + (o % PAGE_TOKENS) : -1;
+          row_ctx0[r] = ctx0;
+          plan.row_slot[r] = t + o;
+          visible_pairs += t + o + 1;
+        }
+      }
+      t += len;
+    }
+    for (int32_t r0 = plan.cu_new[b]; r0 < plan.cu_new[b + 1]; r0 += 128) {
+      AttnTile& a = tiles[n_tiles++];
+      a.row0 = r0;
+      a.n_rows = std::min(128, plan.cu_new[b + 1] - r0);
+      a.ctx0 = ctx0;
+      a.kv_len = row_pos[r0 + a.n_rows - 1] + 1;
+      a.min_pos = row_pos[r0];
+      a.pad0 = a.pad1 = a.pad2 = 0;
+    }
+  }
+  const double plan_us =
+      std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
+
+  // ---------------------------------------------------------------- device work
+  cudaStream_t s = h->stream;
+  percache_stats_t& st = h->stats;
+  std::memset(st.phase_us, 0, sizeof(st.phase_us));
+  std::memset(st.phase_launches, 0, sizeof(st.phase_launches));
+  PhaseTimer timer(h);
+  bool ok = true;
+  const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(tiles + n_tiles) - h->h_index);
+  ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
+  const int32_t* d_row_slot = h->d_index;
+  const int32_t* d_row_pos = d_row_slot + h->m_cap;
+  const int32_t* d_row_pool = d_row_pos + h->m_cap;
+  const int32_t* d_row_ctx0 = d_row_pool + h->m_cap;
+  const GatherItem* d_items = reinterpret_cast<const GatherItem*>(d_row_ctx0 + h->m_cap);
+  const AttnTile* d_tiles = reinterpret_cast<const AttnTile*>(reinterpret_cast<const int32_t*>(d_items) + 4 * h->ctx_cap);
+
+  const bool use_ref = (h->flags & PERCACHE_FLAG_REFERENCE_KERNELS) != 0;
+  if (use_ref && !h->cref) {
+    const size_t wide = static_cast<size_t>(std::max(std::max(D.qkv_dim, 2 * D.d_ffn), d));
+    if (!dev_alloc(h, &h->cref, static_cast<size_t>(h->m_cap) * wide)) return fail(PERCACHE_E_NOMEM);
+  }
+
+  timer.begin(PERCACHE_PH_IO);
+  for (const Seg& sg : segs)
+    ok = ok && cudaMemcpyAsync(h->xin + static_cast<size_t>(sg.row0) * d, sg.src, static_cast<size_t>(sg.n) * d * 2,
+                               sg.on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s) == cudaSuccess;
+  cudaEventRecord(h->ev_begin, s);
+  launch_bf16_to_f32(h->xin, h->resid, M * d, s);
+  timer.end();
+
+  if (n_items > 0) {
+    timer.begin(PERCACHE_PH_GATHER);
+    launch_gather_rerope(d_items, n_items, D.n_layers, h->kpool, h->vpool, h->cfg.pool_pages, h->kctx, h->vctx,
+                         h->ctx_cap, D.kv_dim, h->rope, s);
+    timer.end();
+  }
+  const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
+  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
+  const int Mi = static_cast<int>(M);
+  for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
+    LayerWeights& W = h->layers[l];
+    timer.begin(PERCACHE_PH_NORM);
+    launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
+    timer.end();
+
+    QkvEpilogue qe;
+    qe.rows = RowIndex{d_row_slot, d_row_pos, d_row_pool};
+    qe.rope = h->rope;
+    qe.q_out = h->qbuf;
+    qe.kpool = h->kpool + l * pool_layer;
+    qe.vpool = h->vpool + l * pool_layer;
+    qe.kctx = h->kctx + l * ctx_layer;
+    qe.vctx = h->vctx + l * ctx_layer;
+    qe.n_q_heads = D.n_q_heads;
+    qe.n_kv_heads = D.n_kv_heads;
+    timer.begin(PERCACHE_PH_QKV);
+    if (use_ref) {
+      launch_ref_gemm(h->xn, W.wqkv, h->cref, Mi, D.qkv_dim, d, s);
+      launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
+    } else {
+      ok = ok && launch_umma_gemm(h->m_xn, W.m_wqkv, Mi, D.qkv_dim, d, 128, EPI_QKV, &qe, nullptr, h->d_err, h->n_sms, s) == 0;
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_ATTN);
+    if (use_ref) {
+      launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
+    } else {
+      ok = ok && launch_umma_attention(W.attn_maps, d_tiles, n_tiles, d_row_pos, h->attn_out, D.n_q_heads, D.n_kv_heads,
+                                       h->d_err, h->n_sms, s) == 0;
+    }
+    timer.end();
+
+    ResidualEpilogue re{h->resid, d};
+    timer.begin(PERCACHE_PH_OPROJ);
+    if (use_ref) {
+      launch_ref_gemm(h->attn_out, W.wo, h->cref, Mi, d, D.q_dim, s);
+      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
+    } else {
+      ok = ok && launch_umma_gemm(h->m_attn, W.m_wo, Mi, d, D.q_dim, 128, EPI_RESIDUAL, &re, nullptr, h->d_err, h->n_sms, s) == 0;
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_NORM);
+    launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
+    timer.end();
+
+    SwigluEpilogue se{h->act, D.d_ffn};
+    timer.begin(PERCACHE_PH_GATEUP);
+    if (use_ref) {
+      launch_ref_gemm(h->xn, W.wgu, h->cref, Mi, 2 * D.d_ffn, d, s);
+      launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
+    } else {
+      ok = ok && launch_umma_gemm(h->m_xn, W.m_wgu, Mi, 2 * D.d_ffn, d, 128, EPI_SWIGLU, &se, nullptr, h->d_err, h->n_sms, s) == 0;
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_DOWN);
+    if (use_ref) {
+      launch_ref_gemm(h->act, W.wd, h->cref, Mi, d, D.d_ffn, s);
+      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
+    } else {
+      ok = ok && launch_umma_gemm(h->m_act, W.m_wd, Mi, d, D.d_ffn, 128, EPI_RESIDUAL, &re, nullptr, h->d_err, h->n_sms, s) == 0;
+    }
+    timer.end();
+  }
+  cudaEventRecord(h->ev_end, s);
+  timer.begin(PERCACHE_PH_IO);
+  for (int b = 0; b < n_prompts && ok; ++b) {
+    const int n_new = plan.cu_new[b + 1] - plan.cu_new[b];
+    if (n_new > 0)
+      ok = ok && cudaMemcpyAsync(results[b].out_hidden, h->resid + static_cast<size_t>(plan.cu_new[b]) * d,
+                                 static_cast<size_t>(n_new) * d * sizeof(float),
+                                 results[b].out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  timer.end();
+  const cudaError_t sync_rc = cudaStreamSynchronize(s);
+  if (!ok || sync_rc != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(PERCACHE_E_CUDA);
+  if (*h->h_err != 0) return fail(PERCACHE_E_DEVICE_TIMEOUT);
+
+  // ---------------------------------------------------------------- commit
+  for (auto& pe : pending) h->table.emplace(pe.first, std::move(pe.second));
+  for (int b = 0; b < n_prompts; ++b) {
+    results[b].n_new = plan.cu_new[b + 1] - plan.cu_new[b];
+    results[b].n_total = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+    if (results[b].hit_mask && prompts[b].n_chunks > 0)
+      std::memcpy(results[b].hit_mask, hit[b].data(), static_cast<size_t>(prompts[b].n_chunks));
+  }
+  h->plan = std::move(plan);
+  st.n_prompts = n_prompts;
+  st.chunks_hit = chunks_hit;
+  st.chunks_missed = chunks_missed;
+  st.ctx_tokens = ctx_total;
+  st.hit_tokens = hit_tokens;
+  st.new_rows = new_total;
+  refresh_page_stats(h);
+  st.host_plan_us = plan_us;
+  st.attn_visible_pairs = visible_pairs;
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
+  st.device_us = 1000.0 * ms;
+  timer.collect();
+  return PERCACHE_OK;
+}
+
+int percache_get_stats(percache_t* h, percache_stats_t* out) {
+  if (!h || !out) return PERCACHE_E_INVAL;
+  *out = h->stats;
+  return PERCACHE_OK;
+}
+
+int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity) {
+  if (!h || !out) return PERCACHE_E_INVAL;
+  const std::vector<int32_t>* v = nullptr;
+  switch (which) {
+    case 0: v = &h->plan.cu_ctx; break;
+    case 1: v = &h->plan.cu_new; break;
+    case 2: v = &h->plan.slot_chunk; break;
+    case 3: v = &h->plan.slot_offset; break;
+    case 4: v = &h->plan.slot_is_new; break;
+    case 5: v = &h->plan.row_slot; break;
+    default: return PERCACHE_E_INVAL;
+  }
+  if (static_cast<int64_t>(v->size()) > capacity) return PERCACHE_E_CAPACITY;
+  if (!v->empty()) std::memcpy(out, v->data(), v->size() * sizeof(int32_t));
+  return static_cast<int64_t>(v->size());
+}
+
+int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host) {
+  if (!h || !k_host || !v_host || layer < 0 || layer >= h->dims.n_layers || prompt < 0 ||
+      prompt + 1 >= static_cast<int32_t>(h->plan.cu_ctx.size()))
+    return PERCACHE_E_INVAL;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * h->dims.kv_dim;
+  const size_t off = layer * ctx_layer + static_cast<size_t>(h->plan.cu_ctx[prompt]) * h->dims.kv_dim;
+  const size_t bytes = static_cast<size_t>(h->plan.cu_ctx[prompt + 1] - h->plan.cu_ctx[prompt]) * h->dims.kv_dim * 2;
+  if (cudaMemcpy(k_host, h->kctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
+      cudaMemcpy(v_host, h->vctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
+    return PERCACHE_E_CUDA;
+  return PERCACHE_OK;
+}
+
+int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
+                        float* c, int32_t use_reference) {
+  if (M <= 0 || N <= 0 || K <= 0 || !a_f16 || !b_f16 || !c) return PERCACHE_E_INVAL;
+  if (!use_reference && (K % 64 != 0 || N % 128 != 0)) return PERCACHE_E_INVAL;
+  int n_dev = 0;
+  if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) { cudaGetLastError(); return PERCACHE_E_CUDA; }
+  if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return PERCACHE_E_CUDA; }
+  if (init_driver_api() != 0) return PERCACHE_E_CUDA;
+  __half *dA = nullptr, *dB = nullptr;
+  float* dC = nullptr;
+  int *dErr = nullptr, hErr = 0;
+  int rc = PERCACHE_OK;
+  const size_t m_pad = static_cast<size_t>((M + 127) / 128) * 128;
+  if (cudaMalloc(reinterpret_cast<void**>(&dA), m_pad * K * 2) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&dB), static_cast<size_t>(N) * K * 2) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&dC), static_cast<size_t>(M) * N * 4) != cudaSuccess ||
+      cudaMalloc(reinterpret_cast<void**>(&dErr), sizeof(int)) != cudaSuccess) {
+    cudaGetLastError();
+    rc = PERCACHE_E_NOMEM;
+  }
+  if (rc == PERCACHE_OK) {
+    cudaMemset(dA, 0, m_pad * K * 2);
+    cudaMemset(dErr, 0, sizeof(int));
+    cudaMemcpy(dA, a_f16, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice);
+    cudaMemcpy(dB, b_f16, static_cast<size_t>(N) * K * 2, cudaMemcpyHostToDevice);
+    if (use_reference) {
+      launch_ref_gemm(dA, dB, dC, M, N, K, nullptr);
+    } else {
+      GemmOperand mA, mB;
+      int n_sms = 148;
+      cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, device);
+      if (make_operand_map(&mA, dA, static_cast<int64_t>(m_pad), K, 128) != 0 || make_operand_map(&mB, dB, N, K, 128) != 0 ||
+          launch_umma_gemm(mA, mB, M, N, K, 128, EPI_STORE_F32, nullptr, dC, dErr, n_sms, nullptr) != 0)
+        rc = PERCACHE_E_CUDA;
+    }
+    if (rc == PERCACHE_OK && (cudaDeviceSynchronize() != cudaSuccess || cudaGetLastError() != cudaSuccess)) rc = PERCACHE_E_CUDA;
+    if (rc == PERCACHE_OK) {
+      cudaMemcpy(&hErr, dErr, sizeof(int), cudaMemcpyDeviceToHost);
+      if (hErr != 0) rc = PERCACHE_E_DEVICE_TIMEOUT;
+      else if (cudaMemcpy(c, dC, static_cast<size_t>(M) * N * 4, cudaMemcpyDeviceToHost) != cudaSuccess) rc = PERCACHE_E_CUDA;
+    }
+  }
+  if (dA) cudaFree(dA);
+  if (dB) cudaFree(dB);
+  if (dC) cudaFree(dC);
+  if (dErr) cudaFree(dErr);
+  return rc;
+}
+
+}  // extern "C"
