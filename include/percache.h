@@ -39,6 +39,12 @@
 extern "C" {
 #endif
 
+#if defined(__GNUC__)
+#define PERCACHE_API __attribute__((visibility("default")))
+#else
+#define PERCACHE_API
+#endif
+
 #define PERCACHE_OK                 0
 #define PERCACHE_E_INVAL           -1   /* bad argument (NULL, negative size, unsupported shape)        */
 #define PERCACHE_E_NOMEM           -2   /* host or device allocation failed                            */
@@ -57,6 +63,7 @@ extern "C" {
 #define PERCACHE_FLAG_REFERENCE_KERNELS  1u  /* debugging aid: run every GEMM and the attention with the plain
                                                 one-thread-per-output CUDA kernels instead of the tcgen05 ones */
 #define PERCACHE_FLAG_PHASE_TIMING       2u  /* record CUDA events around every kernel class (see stats)       */
+#define PERCACHE_FLAG_REFERENCE_ATTENTION 4u /* debugging aid: plain attention kernel, tcgen05 GEMMs            */
 
 typedef struct percache percache_t;   /* opaque */
 
@@ -82,19 +89,19 @@ typedef struct {
 } percache_layer_weights_t;
 
 /* Create a handle: allocates the paged store, work buffers and a private copy of the weights on
- * cfg->device.  Supported shapes: head_dim 128; d_model, d_ffn multiples of 64; n_q_heads a multiple of
- * n_kv_heads.  Device allocation failure -> PERCACHE_E_NOMEM; the handle is not created. */
-int percache_create(const percache_config_t* cfg, const percache_layer_weights_t* layers /*[n_layers]*/,
+ * cfg->device.  Supported shapes: head_dim 128; d_model, d_ffn multiples of 64; n_q_heads an even multiple
+ * of n_kv_heads (the attention kernel pairs the query heads of a KV head).  Device allocation failure -> PERCACHE_E_NOMEM; the handle is not created. */
+PERCACHE_API int percache_create(const percache_config_t* cfg, const percache_layer_weights_t* layers /*[n_layers]*/,
                     int32_t weights_on_device, percache_t** out);
 
 /* Free everything the handle owns.  NULL is accepted. */
-int percache_destroy(percache_t* h);
+PERCACHE_API int percache_destroy(percache_t* h);
 
 /* Insert a chunk's unrotated K and V for all layers (what a prefill of that chunk collected; paper
  * Section 3.2.1).  k, v: bf16 [n_layers][n_tokens][n_kv_heads][head_dim], host or device memory as
  * ptr_is_device says.  Copied into ceil(n_tokens/16) pages before return.  An id that is already stored
  * is not overwritten: PERCACHE_E_EXISTS. */
-int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens,
+PERCACHE_API int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens,
                           const void* k, const void* v, int32_t ptr_is_device);
 
 /* A prompt: ordered chunk list plus query tokens (paper Section 3, system overview). */
@@ -125,24 +132,24 @@ typedef struct {
  * stored (its K/V as computed inside its prompt; if two prompts of the batch miss the same id, the
  * first prompt's is kept) and query tokens are not.  Too few free pages -> PERCACHE_E_NOSPACE.
  * Synchronous: returns after the stream has drained. */
-int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
+PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
 
 /* *n_tokens = stored length, or PERCACHE_E_NOTFOUND. n_tokens may be NULL. */
-int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n_tokens);
+PERCACHE_API int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n_tokens);
 
 /* Remove a chunk and free its pages (used to restore the cache state between timed runs). */
-int percache_drop_chunk(percache_t* h, uint64_t chunk_id);
+PERCACHE_API int percache_drop_chunk(percache_t* h, uint64_t chunk_id);
 
 /* Read a stored chunk back: k, v host buffers bf16 [n_layers][n_tokens][n_kv_heads][head_dim]. */
-int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* v_host);
+PERCACHE_API int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* v_host);
 
 /* Fill a new chunk with the synthetic integer pool values of the batched-serving workload:
  * element e of (chunk, which in {K=0,V=1}, layer) takes the 64-bit counter
  *   ((((seed << 20) + chunk_id) * 2 + which) * 64 + layer) << 24) + e
  * through the SplitMix64 output function, and the value (b0 + b1 + b2 + b3 - 126) / 64 with b_i the four
  * lowest 6-bit fields of the result (exact in bf16).  Same errors as percache_put_chunk_kv. */
-int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tokens, uint64_t seed);
+PERCACHE_API int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tokens, uint64_t seed);
 
 /* Kernel classes for phase timing. */
 enum {
@@ -169,28 +176,28 @@ typedef struct {
   int64_t attn_visible_pairs;                  /* sum over new rows of (position + 1)             */
 } percache_stats_t;
 
-int percache_get_stats(percache_t* h, percache_stats_t* out);
+PERCACHE_API int percache_get_stats(percache_t* h, percache_stats_t* out);
 
 /* Switch PERCACHE_FLAG_PHASE_TIMING / PERCACHE_FLAG_REFERENCE_KERNELS after creation. */
-int percache_set_flags(percache_t* h, uint32_t flags);
+PERCACHE_API int percache_set_flags(percache_t* h, uint32_t flags);
 
 /* Integer plan of the last successful percache_prefill (host int32 arrays, caller-allocated).
  * which: 0 cu_ctx [n_prompts+1]; 1 cu_new [n_prompts+1]; 2 slot_chunk [ctx_tokens] (index into the prompt's
  * chunk list, n_chunks for query tokens); 3 slot_offset [ctx_tokens]; 4 slot_is_new [ctx_tokens];
  * 5 row_slot [new_rows] (slot of every new row inside its prompt = its position).
  * Returns the number of elements written, or a negative code (PERCACHE_E_CAPACITY if capacity is short). */
-int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity);
+PERCACHE_API int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity);
 
 /* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
  * [n_total][n_kv_heads][head_dim], copied to host buffers. */
-int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
+PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
 
 /* C[M][N] (fp32, host) = A[M][K] * B[N][K]^T with fp16 inputs (host), through the tcgen05 GEMM
  * (use_reference = 0) or the plain kernel (1).  Test hook for the GEMM core. */
-int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
+PERCACHE_API int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
                         float* c, int32_t use_reference);
 
-const char* percache_strerror(int code);
+PERCACHE_API const char* percache_strerror(int code);
 
 #ifdef __cplusplus
 }

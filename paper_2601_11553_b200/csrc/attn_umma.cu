@@ -1,0 +1,362 @@
+// Causal grouped-query flash attention of the new rows against the assembled context, on tcgen05.
+//
+// Work unit = (tile of up to 128 consecutive new rows of one prompt, one KV head).  The two query heads
+// that share the KV head are two 128-row M tiles of the unit: they have the same rows, positions and
+// mask and read the same K/V blocks, so every K/V byte fetched into shared memory is used twice.
+//
+// One persistent CTA per SM, 320 threads:
+//   warps 0-3  softmax group of query head 2g      (thread = row; TMEM lanes by warp quarter)
+//   warps 4-7  softmax group of query head 2g + 1
+//   warp 8     TMA producer: Q tiles of both heads, then K and V blocks of 128 context slots into
+//              two-stage rings (each block = two 64-column halves in the 128-byte swizzle)
+//   warp 9     MMA issuer: S_i = Q_i K^T into TMEM, O_i += P_i V with P_i read from TMEM
+// TMEM (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512); P_i (fp16, two per
+// column) overwrites the first 64 columns of S_i.  Per head the chain S -> softmax -> PV -> next S is
+// serial; the two heads alternate so the tensor core works on one while the other is in softmax.
+// The running maximum is only raised when the block maximum exceeds it by more than 8 (in log2
+// units), which keeps P below 2^8 and makes rescaling of O in TMEM rare.
+// A row at position p sees context slots 0..p of its prompt (hit or freshly computed alike).
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace pc {
+
+namespace {
+
+constexpr int ATT_THREADS = 320;
+constexpr int BLK = 128;                       // rows per tile and context slots per block
+constexpr int HALF_TILE_BYTES = BLK * 64 * 2;  // 16 KB: 128 rows x 64 fp16 (one swizzled half)
+constexpr int TILE_BYTES = 2 * HALF_TILE_BYTES;
+constexpr int KV_STAGES = 2;
+constexpr int ATT_SMEM_BYTES = 2 * TILE_BYTES + 2 * KV_STAGES * TILE_BYTES + 1024;
+constexpr uint32_t TMEM_S0 = 0, TMEM_O0 = 256;
+constexpr float RESCALE_THRESHOLD = 8.0f;
+
+struct AttnArgs {
+  const AttnTile* tiles;
+  int32_t n_tiles;
+  const int32_t* row_pos;
+  __half* out;
+  int32_t n_q_heads, n_kv_heads;
+  float scale_log2;      // log2(e) / sqrt(head_dim)
+  int* err_word;
+};
+
+__device__ __forceinline__ float fast_exp2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+__global__ void __launch_bounds__(ATT_THREADS, 1)
+umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+                      const __grid_constant__ CUtensorMap tmV, AttnArgs args) {
+  extern __shared__ uint8_t smem_raw[];
+  __shared__ __align__(8) uint64_t q_full, q_empty;
+  __shared__ __align__(8) uint64_t k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
+  __shared__ __align__(8) uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+  __shared__ uint32_t tmem_base_slot;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* q_smem = base;                                   // [2 heads][2 halves][128][64]
+  uint8_t* k_smem = base + 2 * TILE_BYTES;                  // [stages][2 halves][128][64]
+  uint8_t* v_smem = k_smem + KV_STAGES * TILE_BYTES;
+
+  if (threadIdx.x == 0) {
+    mbar_init(&q_full, 1);
+    mbar_init(&q_empty, 1);
+    for (int s = 0; s < KV_STAGES; ++s) {
+      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4);
+      mbar_init(&o_done[i], 1); mbar_init(&o_free[i], 4);
+    }
+    fence_mbar_init();
+  }
+  if (warp == 9) {
+    tmem_alloc<512>(&tmem_base_slot);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = tmem_base_slot;
+
+  const int n_units = args.n_tiles * args.n_kv_heads;
+  const int group = args.n_q_heads / args.n_kv_heads;      // query heads per KV head (even)
+  // A unit covers query heads (g * group + 2 * pair, +1); units enumerate (tile, g, pair).
+  const int pairs = group / 2;
+  const int n_work = n_units * pairs;
+
+  if (warp == 8) {
+    // ---------------------------------------------------------------- TMA producer
+    if (lane == 0) {
+      prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
+      uint32_t unit_it = 0, kvit = 0;
+      bool ok = true;
+      for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
+        const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
+        const int gp = w % (args.n_kv_heads * pairs);
+        const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
+        const int nb = (t.kv_len + BLK - 1) / BLK;
+        if (!mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+        mbar_arrive_expect_tx(&q_full, 2 * TILE_BYTES);
+        for (int i = 0; i < 2; ++i)
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_2d(q_smem + i * TILE_BYTES + hf * HALF_TILE_BYTES, &tmQ, &q_full, (h0 + i) * HEAD_DIM + hf * 64,
+                        t.row0);
+        for (int j = 0; j < nb; ++j, ++kvit) {
+          const int st = kvit & 1;
+          const uint32_t ph = (kvit >> 1) & 1u;
+          if (!mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+          mbar_arrive_expect_tx(&k_full[st], TILE_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_2d(k_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmK, &k_full[st], g * HEAD_DIM + hf * 64,
+                        t.ctx0 + j * BLK);
+          if (!mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+          mbar_arrive_expect_tx(&v_full[st], TILE_BYTES);
+          for (int hf = 0; hf < 2; ++hf)
+            tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmV, &v_full[st], g * HEAD_DIM + hf * 64,
+                        t.ctx0 + j * BLK);
+        }
+      }
+      if (!ok) {   // error path only: let copies already issued land before shared memory is released
+        const unsigned long long t0 = globaltimer_ns();
+        while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
+      }
+    }
+  } else if (warp == 9) {
+    // ---------------------------------------------------------------- MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, 0, 0, 0);        // A, B K-major
+      constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, 0, 0, 1);   // B (V) MN-major
+      uint32_t unit_it = 0, kvit = 0;
+      bool ok = true;
+      // S_i(kvidx) = Q_i K(kvidx)^T
+      auto issue_s = [&](int i, uint32_t kvidx) {
+        const int st = kvidx & 1;
+        const uint32_t qa = smem_u32(q_smem + i * TILE_BYTES), ka = smem_u32(k_smem + st * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < HEAD_DIM / 16; ++kk) {
+          const uint32_t off = (kk >> 2) * HALF_TILE_BYTES + (kk & 3) * 32;
+          umma_ss(tmem_base + TMEM_S0 + i * BLK, make_smem_desc_sw128(qa + off, 16, 1024),
+                  make_smem_desc_sw128(ka + off, 16, 1024), idesc_qk, kk != 0 ? 1u : 0u);
+        }
+        umma_commit(&s_full[i]);
+      };
+      for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
+        const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
+        const int nb = (t.kv_len + BLK - 1) / BLK;
+        const uint32_t kv0 = kvit;
+        if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+        if (!mbar_wait(&k_full[kv0 & 1], (kv0 >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+        tc_fence_after_sync();
+        issue_s(0, kv0);
+        issue_s(1, kv0);
+        umma_commit(&k_empty[kv0 & 1]);
+        if (nb == 1) umma_commit(&q_empty);
+        for (int j = 0; j < nb && ok; ++j) {
+          const uint32_t kvidx = kv0 + j;
+          const int st = kvidx & 1;
+          for (int i = 0; i < 2; ++i) {
+            if (!mbar_wait(&p_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+            if (j == 0 && !mbar_wait(&o_free[i], (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+            if (i == 0 && !mbar_wait(&v_full[st], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+            tc_fence_after_sync();
+            const uint32_t va = smem_u32(v_smem + st * TILE_BYTES);
+#pragma unroll
+            for (int kk = 0; kk < BLK / 16; ++kk) {
+              // 16 context slots = 16 rows of 128 bytes in each 64-column half; halves are 16 KB apart
+              umma_ts(tmem_base + TMEM_O0 + i * HEAD_DIM, tmem_base + TMEM_S0 + i * BLK + kk * 8,
+                      make_smem_desc_sw128(va + kk * 2048, HALF_TILE_BYTES, 1024), idesc_pv, (j | kk) != 0 ? 1u : 0u);
+            }
+            umma_commit(&o_done[i]);
+            if (i == 1) umma_commit(&v_empty[st]);
+            if (j + 1 < nb) {
+              const uint32_t nxt = kvidx + 1;
+              if (i == 0 && !mbar_wait(&k_full[nxt & 1], (nxt >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+              tc_fence_after_sync();
+              issue_s(i, nxt);
+              if (i == 1) {
+                umma_commit(&k_empty[nxt & 1]);
+                if (j + 2 == nb) umma_commit(&q_empty);
+              }
+            }
+          }
+        }
+        kvit += nb;
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- softmax groups (warps 0..7)
+    const int i = warp >> 2;                      // which query head of the pair
+    const int quarter = warp & 3;
+    const int r_in_tile = quarter * 32 + lane;
+    const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t t_s = tmem_base + lane_base + TMEM_S0 + i * BLK;
+    const uint32_t t_o = tmem_base + lane_base + TMEM_O0 + i * HEAD_DIM;
+    uint32_t unit_it = 0, kvit = 0;
+    bool ok = true;
+    for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
+      const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
+      const int gp = w % (args.n_kv_heads * pairs);
+      const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
+      const int nb = (t.kv_len + BLK - 1) / BLK;
+      const uint32_t kv0 = kvit;
+      const bool valid = r_in_tile < t.n_rows;
+      const int row = t.row0 + (valid ? r_in_tile : t.n_rows - 1);
+      const int pos = args.row_pos[row];
+      float m = -INFINITY, l = 0.f;
+      for (int j = 0; j < nb; ++j) {
+        const uint32_t kvidx = kv0 + j;
+        ok = mbar_wait(&s_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_SOFTMAX);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after_sync();
+        uint32_t s[128];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+        tmem_wait_ld();
+        const int limit = pos - j * BLK;          // columns 0..limit are visible
+        float m_blk = -INFINITY;
+        if (limit >= BLK - 1) {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float x = __uint_as_float(s[c]) * args.scale_log2;
+            s[c] = __float_as_uint(x);
+            m_blk = fmaxf(m_blk, x);
+          }
+        } else {
+#pragma unroll
+          for (int c = 0; c < 128; ++c) {
+            const float x = c <= limit ? __uint_as_float(s[c]) * args.scale_log2 : -INFINITY;
+            s[c] = __float_as_uint(x);
+            m_blk = fmaxf(m_blk, x);
+          }
+        }
+        if (j == 0) {
+          m = m_blk;                               // slot 0 is visible to every row: finite
+        } else {
+          const bool need = m_blk > m + RESCALE_THRESHOLD;
+          if (__any_sync(0xffffffffu, need)) {
+            // O_i must be complete up to the previous block before it is rescaled in place
+            ok = mbar_wait(&o_done[i], (kvidx - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            float alpha = 1.0f;
+            if (need) { alpha = fast_exp2(m - m_blk); m = m_blk; l *= alpha; }
+#pragma unroll 1
+            for (int c = 0; c < 4; ++c) {
+              uint32_t o[32];
+              tmem_ld_32x32(t_o + c * 32, o);
+              tmem_wait_ld();
+#pragma unroll
+              for (int e = 0; e < 32; ++e) o[e] = __float_as_uint(__uint_as_float(o[e]) * alpha);
+              tmem_st_32x32(t_o + c * 32, o);
+            }
+            tmem_wait_st();
+          }
+        }
+        uint32_t p[64];
+        float sum = 0.f;
+#pragma unroll
+        for (int c = 0; c < 64; ++c) {
+          const float p0 = fast_exp2(__uint_as_float(s[2 * c]) - m);
+          const float p1 = fast_exp2(__uint_as_float(s[2 * c + 1]) - m);
+          sum += p0 + p1;
+          __half2 hh = __floats2half2_rn(p0, p1);
+          p[c] = *reinterpret_cast<uint32_t*>(&hh);
+        }
+        l += sum;
+        tmem_st_32x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&p[0]));
+        tmem_st_32x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&p[32]));
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&p_full[i]);
+      }
+      if (!ok) break;
+      // ---- final: O_i / l -> fp16 -> out
+      ok = mbar_wait(&o_done[i], (kv0 + nb - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const float inv_l = 1.0f / l;
+      __half* dst = args.out + (static_cast<size_t>(row) * args.n_q_heads + head) * HEAD_DIM;
+#pragma unroll 1
+      for (int c = 0; c < 4; ++c) {
+        uint32_t o[32];
+        tmem_ld_32x32(t_o + c * 32, o);
+        tmem_wait_ld();
+        if (valid) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            uint32_t pk[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              __half2 hh = __floats2half2_rn(__uint_as_float(o[8 * e + 2 * q]) * inv_l,
+                                             __uint_as_float(o[8 * e + 2 * q + 1]) * inv_l);
+              pk[q] = *reinterpret_cast<uint32_t*>(&hh);
+            }
+            *reinterpret_cast<uint4*>(dst + c * 32 + e * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&o_free[i]);
+      kvit += nb;
+    }
+  }
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 9) {
+    tc_fence_after_sync();
+    tmem_dealloc<512>(tmem_base);
+  }
+}
+
+}  // namespace
+
+int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, const __half* kctx_layer,
+                   const __half* vctx_layer, int64_t ctx_cap, int kv_dim) {
+  const uint32_t box[2] = {64u, static_cast<uint32_t>(BLK)};
+  {
+    const uint64_t dims[2] = {static_cast<uint64_t>(q_dim), static_cast<uint64_t>(m_cap)};
+    const uint64_t str[1] = {static_cast<uint64_t>(q_dim) * 2};
+    if (encode_f16_map(&out->q, q, 2, dims, str, box) != 0) return -1;
+  }
+  const uint64_t dims[2] = {static_cast<uint64_t>(kv_dim), static_cast<uint64_t>(ctx_cap)};
+  const uint64_t str[1] = {static_cast<uint64_t>(kv_dim) * 2};
+  if (encode_f16_map(&out->k, kctx_layer, 2, dims, str, box) != 0) return -1;
+  if (encode_f16_map(&out->v, vctx_layer, 2, dims, str, box) != 0) return -1;
+  return 0;
+}
+
+int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
+                          __half* out, int n_q_heads, int n_kv_heads, int* err_word, int n_sms, cudaStream_t s) {
+  if (n_tiles <= 0) return 0;
+  const int group = n_q_heads / n_kv_heads;
+  if (group < 2 || group % 2 != 0) return -1;
+  if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
+      cudaSuccess)
+    return -1;
+  AttnArgs a{};
+  a.tiles = tiles; a.n_tiles = n_tiles; a.row_pos = row_pos; a.out = out;
+  a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
+  a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
+  a.err_word = err_word;
+  const int n_work = n_tiles * n_kv_heads * (group / 2);
+  const int grid = n_work < n_sms ? n_work : n_sms;
+  umma_attention_kernel<<<grid, ATT_THREADS, ATT_SMEM_BYTES, s>>>(maps.q, maps.k, maps.v, a);
+  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+}
+
+}  // namespace pc

@@ -1,4 +1,5 @@
 // Memory-bound kernels: gather + re-RoPE of cached pages, RMSNorm, format conversions, page copies.
+#include <algorithm>
 #include "kernels.h"
 
 namespace pc {
@@ -31,7 +32,7 @@ __global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half
 }
 void launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, int64_t n, cudaStream_t s) {
   if (n <= 0) return;
-  const int blocks = static_cast<int>(min<int64_t>((n + 255) / 256, 148 * 16));
+  const int blocks = static_cast<int>(std::min<int64_t>((n + 255) / 256, 148 * 16));
   bf16_to_f16_kernel<<<blocks, 256, 0, s>>>(src, dst, n);
 }
 
@@ -59,7 +60,7 @@ __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ src, float*
 }
 void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStream_t s) {
   if (n <= 0) return;
-  const int blocks = static_cast<int>(min<int64_t>((n + 255) / 256, 148 * 16));
+  const int blocks = static_cast<int>(std::min<int64_t>((n + 255) / 256, 148 * 16));
   bf16_to_f32_kernel<<<blocks, 256, 0, s>>>(src, dst, n);
 }
 
@@ -192,7 +193,7 @@ void launch_gather_rerope(const GatherItem* items, int n_items, int n_layers, co
                           int64_t ctx_cap, int kv_dim, const float2* rope, cudaStream_t s) {
   if (n_items <= 0) return;
   const int64_t units = static_cast<int64_t>(n_items) * n_layers;
-  const int blocks = static_cast<int>(min<int64_t>(units, 148 * 8));
+  const int blocks = static_cast<int>(std::min<int64_t>(units, 148 * 8));
   gather_rerope_kernel<<<blocks, GATHER_THREADS, 0, s>>>(items, n_items, n_layers, kpool, vpool, pool_pages, kctx,
                                                          vctx, ctx_cap, kv_dim, rope);
 }
@@ -221,7 +222,7 @@ __global__ void chunk_pages_copy_kernel(__nv_bfloat16* chunk, __nv_bfloat16* poo
 void launch_chunk_pages_copy(__nv_bfloat16* chunk, __nv_bfloat16* pool, const int32_t* pages, int n_tokens,
                              int n_layers, int64_t pool_pages, int kv_dim, int to_pool, cudaStream_t s) {
   const int64_t n = static_cast<int64_t>(n_layers) * n_tokens * (kv_dim / 8);
-  const int blocks = static_cast<int>(min<int64_t>((n + 255) / 256, 148 * 16));
+  const int blocks = static_cast<int>(std::min<int64_t>((n + 255) / 256, 148 * 16));
   chunk_pages_copy_kernel<<<blocks, 256, 0, s>>>(chunk, pool, pages, n_tokens, n_layers, pool_pages, kv_dim, to_pool);
 }
 
@@ -263,7 +264,7 @@ void launch_fill_synthetic(__nv_bfloat16* kpool, __nv_bfloat16* vpool, const int
                            int n_layers, int64_t pool_pages, int kv_dim, uint64_t seed, uint64_t chunk_id,
                            cudaStream_t s) {
   const int64_t n = 2 * static_cast<int64_t>(n_layers) * n_tokens * kv_dim;
-  const int blocks = static_cast<int>(min<int64_t>((n + 255) / 256, 148 * 16));
+  const int blocks = static_cast<int>(std::min<int64_t>((n + 255) / 256, 148 * 16));
   fill_synthetic_kernel<<<blocks, 256, 0, s>>>(kpool, vpool, pages, n_tokens, n_layers, pool_pages, kv_dim, seed,
                                                chunk_id);
 }

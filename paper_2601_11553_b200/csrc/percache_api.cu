@@ -191,7 +191,7 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   *out = nullptr;
   if (cfg->n_layers <= 0 || cfg->n_layers > 64 || cfg->head_dim != HEAD_DIM || cfg->page_tokens != PAGE_TOKENS ||
       cfg->d_model <= 0 || cfg->d_model % 128 != 0 || cfg->d_ffn <= 0 || cfg->d_ffn % 64 != 0 ||
-      cfg->n_kv_heads <= 0 || cfg->n_q_heads <= 0 || cfg->n_q_heads % cfg->n_kv_heads != 0 ||
+      cfg->n_kv_heads <= 0 || cfg->n_q_heads <= 0 || cfg->n_q_heads % (2 * cfg->n_kv_heads) != 0 ||
       cfg->pool_pages <= 0 || cfg->max_prompt_tokens <= 0 || cfg->max_batch_prompts <= 0 ||
       cfg->max_batch_ctx_tokens <= 0 || cfg->max_batch_new_rows <= 0 || cfg->pool_pages > (INT32_MAX / PAGE_TOKENS) ||
       cfg->max_batch_ctx_tokens > INT32_MAX / 2 || cfg->max_batch_new_rows > INT32_MAX / 2)
@@ -262,6 +262,15 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   h->events.assign(MAX_EVENTS, nullptr);
   for (auto& e : h->events)
     if (cudaEventCreate(&e) != cudaSuccess) { destroy_impl(h); return PERCACHE_E_CUDA; }
+
+  // Operand buffers start as zeros: rows and context slots a call does not write are still read by
+  // whole-tile TMA loads (and then masked or never stored), so they must never hold NaN bit patterns.
+  cudaMemsetAsync(h->kctx, 0, ctx_elems * 2, h->stream);
+  cudaMemsetAsync(h->vctx, 0, ctx_elems * 2, h->stream);
+  cudaMemsetAsync(h->qbuf, 0, static_cast<size_t>(h->m_cap) * D.q_dim * 2, h->stream);
+  cudaMemsetAsync(h->attn_out, 0, static_cast<size_t>(h->m_cap) * D.q_dim * 2, h->stream);
+  cudaMemsetAsync(h->xn, 0, static_cast<size_t>(h->m_cap) * d * 2, h->stream);
+  cudaMemsetAsync(h->act, 0, static_cast<size_t>(h->m_cap) * F * 2, h->stream);
 
   // ---- weights: bf16 -> fp16 copies in the layouts the GEMMs read.  Every bf16 value of magnitude
   // >= 2^-17 is exactly representable in fp16; smaller ones round with absolute error <= 2^-25.
@@ -657,7 +666,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     timer.end();
 
     timer.begin(PERCACHE_PH_ATTN);
-    if (use_ref) {
+    if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
       launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
     } else {
       ok = ok && launch_umma_attention(W.attn_maps, d_tiles, n_tiles, d_row_pos, h->attn_out, D.n_q_heads, D.n_kv_heads,
