@@ -1,0 +1,104 @@
+"""Helpers for the GPU parity tests: run one workload through the C ABI and through the oracle."""
+from __future__ import annotations
+
+from typing import Dict, List, Optional, Sequence, Tuple
+
+import numpy as np
+
+from oracle import reuse_prefill as orc
+from paper_2601_11553_b200 import percache as pcb
+from paper_2601_11553_b200 import workloads as wl
+from tests import helpers as H
+
+TOL_MAX_ABS = 3e-2      # final hidden states, stated with the workloads
+TOL_MEAN_ABS = 3e-3
+
+
+def make_handle(shape: wl.ModelShape, weights: List[dict], prompts: Sequence[wl.Prompt], pool_pages: int = 0,
+                flags: int = 0, slack_prompts: int = 0) -> pcb.PerCache:
+    max_t = max(p.n_total for p in prompts)
+    total = sum(p.n_total for p in prompts)
+    if pool_pages <= 0:
+        pool_pages = sum((l + 15) // 16 for p in prompts for l in p.chunk_len) + 64
+    return pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                        n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
+                        pool_pages=pool_pages, max_prompt_tokens=max_t, max_batch_prompts=len(prompts) + slack_prompts,
+                        max_batch_ctx_tokens=total, max_batch_new_rows=total, rope_theta=shape.rope_theta,
+                        rms_eps=shape.rms_eps, flags=flags)
+
+
+def specs_for(prompts: Sequence[wl.Prompt], cached: Sequence[int]) -> List[pcb.PromptSpec]:
+    cached = set(cached)
+    out = []
+    for p in prompts:
+        hid = None
+        if p.chunk_hidden:
+            hid = [None if c in cached else h for c, h in zip(p.chunk_ids, p.chunk_hidden)]
+        out.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, p.query_hidden, p.n_query))
+    return out
+
+
+def oracle_store_alone(model: orc.Model, seed: int, ids_lens: Sequence[Tuple[int, int]]) -> orc.Store:
+    """Cache content made by prefilling every chunk alone (no hits, no query)."""
+    store = orc.Store()
+    for cid, n in ids_lens:
+        H.populate_alone(model, store, seed, cid, n)
+    return store
+
+
+def push_store(handle: pcb.PerCache, store: orc.Store, ids: Sequence[int]) -> None:
+    """Give the library exactly the oracle's cached K/V (bf16 bits)."""
+    for cid in ids:
+        k, v = store.kv[cid]
+        L, n = k.shape[0], k.shape[1]
+        handle.put_chunk_kv(cid, np.ascontiguousarray(orc.f64_to_bf16_bits(k).reshape(L, n, -1)),
+                            np.ascontiguousarray(orc.f64_to_bf16_bits(v).reshape(L, n, -1)))
+
+
+def f16_ulp(x: np.ndarray) -> np.ndarray:
+    """Spacing of fp16 at |x| (normal range), at least the subnormal spacing."""
+    ax = np.maximum(np.abs(x.astype(np.float64)), 2.0 ** -14)
+    return 2.0 ** (np.floor(np.log2(ax)) - 10)
+
+
+def compare_hidden(got: np.ndarray, want: np.ndarray) -> Dict[str, float]:
+    d = np.abs(got.astype(np.float64) - want)
+    return {"max_abs": float(d.max()) if d.size else 0.0, "mean_abs": float(d.mean()) if d.size else 0.0}
+
+
+def check_plan(plan: Dict[str, np.ndarray], layouts: Sequence[orc.Layout]) -> None:
+    """Index assembly must match the oracle's layout bit for bit."""
+    cu_ctx = np.cumsum([0] + [l.n_total for l in layouts]).astype(np.int32)
+    cu_new = np.cumsum([0] + [len(l.new_slots) for l in layouts]).astype(np.int32)
+    assert np.array_equal(plan["cu_ctx"], cu_ctx)
+    assert np.array_equal(plan["cu_new"], cu_new)
+    assert np.array_equal(plan["slot_chunk"], np.concatenate([l.slot_chunk for l in layouts]))
+    assert np.array_equal(plan["slot_offset"], np.concatenate([l.slot_offset for l in layouts]))
+    assert np.array_equal(plan["slot_is_new"], np.concatenate([l.slot_is_new for l in layouts]).astype(np.int32))
+    assert np.array_equal(plan["row_slot"], np.concatenate([l.new_slots for l in layouts]))
+
+
+def check_ctx(handle: pcb.PerCache, results: Sequence[orc.PromptResult], layers: Sequence[int]) -> Dict[str, float]:
+    """Assembled context against the oracle's: hit slots' V bit-exact, rotated K within 1 fp16 ulp of the pair."""
+    worst = 0.0
+    for b, res in enumerate(results):
+        lay = res.layout
+        hit = lay.slot_is_new == 0
+        for l in layers:
+            k, v = handle.read_ctx(b, l, lay.n_total)
+            kv_dim = k.shape[1]
+            want_v = res.v_ctx[l].reshape(lay.n_total, kv_dim)
+            want_k = res.k_ctx[l].reshape(lay.n_total, kv_dim)
+            # gathered V: a pure format conversion of identical stored values -> identical bits
+            assert np.array_equal(v[hit].view(np.uint16), want_v[hit].astype(np.float16).view(np.uint16)), \
+                f"gathered V differs (prompt {b}, layer {l})"
+            if hit[0]:     # position 0: rotation by zero, K is a pure copy as well
+                assert np.array_equal(k[0].view(np.uint16), want_k[0].astype(np.float16).view(np.uint16))
+            # rotated K of hit slots: 1 ulp at the magnitude of the rotated pair
+            kk = k[hit].astype(np.float64).reshape(-1, kv_dim // 128, 2, 64)
+            ww = want_k[hit].reshape(-1, kv_dim // 128, 2, 64)
+            mag = np.maximum(np.abs(ww[:, :, 0]), np.abs(ww[:, :, 1]))[:, :, None, :]
+            err = np.abs(kk - ww) / f16_ulp(np.broadcast_to(mag, ww.shape))
+            worst = max(worst, float(err.max()) if err.size else 0.0)
+            assert err.size == 0 or err.max() <= 1.0 + 1e-6, f"rotated K off by {err.max()} ulp (prompt {b}, layer {l})"
+    return {"k_rot_max_ulp": worst}
