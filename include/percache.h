@@ -197,6 +197,25 @@ PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t 
 PERCACHE_API int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
                         float* c, int32_t use_reference);
 
+/* The same GEMM as percache_debug_gemm(use_reference = 0) for callers that cannot allocate device memory.
+ * The paper has no counterpart; this exists for two kinds of caller: one whose process has already given
+ * all device memory to another allocator (so a raw cudaMalloc would fail), and one inside a serving loop
+ * that must avoid the device-wide synchronisation of cudaMalloc / cudaFree.  The device copies of A, B, C
+ * and the kernel's error word live in a fixed PERCACHE_NOALLOC_SCRATCH_BYTES array inside the library image
+ * (every GPU that loads the library holds that much until the process exits).  The call itself performs no
+ * cudaMalloc, cudaFree or other allocating routine.
+ *  - Sizes: 256 + pad128(M)*K*2 + N*K*2 + M*N*4 bytes (each term rounded up to 256) must fit in the array,
+ *    otherwise PERCACHE_E_CAPACITY and nothing runs.  K % 64 == 0, N % 128 == 0 as for percache_debug_gemm.
+ *  - a_f16, b_f16, c are host buffers owned by the caller; the call returns after the result is in c.
+ *  - The first call on a device looks up the array's device address; make that call before starting any
+ *    stream capture on that device.
+ *  - All calls share the one array and it keeps the previous call's bytes; the call clears what must start
+ *    at zero.  Two calls whose GPU work overlaps (for instance from two host threads using the same device)
+ *    race on it: serialise them. */
+#define PERCACHE_NOALLOC_SCRATCH_BYTES (16u << 20)
+PERCACHE_API int percache_debug_gemm_noalloc(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16,
+                                const void* b_f16, float* c);
+
 PERCACHE_API const char* percache_strerror(int code);
 
 #ifdef __cplusplus

@@ -30,7 +30,7 @@ PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
            "percache_get_stats", "percache_set_flags", "percache_debug_read_plan", "percache_debug_read_ctx",
-           "percache_debug_gemm", "percache_strerror")
+           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_strerror")
 
 
 class PerCacheError(RuntimeError):
@@ -97,6 +97,7 @@ def load_library() -> C.CDLL:
     lib.percache_debug_read_plan.restype = i64
     lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
+    lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
     lib.percache_strerror.argtypes = [C.c_int]
     lib.percache_strerror.restype = C.c_char_p
     for name in EXPORTS:
@@ -314,4 +315,22 @@ def debug_gemm(a_f16: np.ndarray, b_f16: np.ndarray, use_reference: bool = False
     c = np.empty((m, n), dtype=np.float32)
     _check(lib.percache_debug_gemm(device, m, n, k, _ptr(np.ascontiguousarray(a_f16)), _ptr(np.ascontiguousarray(b_f16)),
                                    _ptr(c), 1 if use_reference else 0), "percache_debug_gemm")
+    return c
+
+
+NOALLOC_SCRATCH_BYTES = 16 << 20
+
+
+def debug_gemm_noalloc(a_f16: np.ndarray, b_f16: np.ndarray, device: int = 0) -> np.ndarray:
+    """C = A @ B.T through the tcgen05 GEMM without any device allocation (percache_debug_gemm_noalloc).
+
+    For callers that cannot call cudaMalloc: the device copies live in a fixed 16 MiB array inside the
+    library; larger problems raise PerCacheError(E_CAPACITY).  Calls must not overlap on the GPU.
+    """
+    lib = load_library()
+    m, k = a_f16.shape
+    n = b_f16.shape[0]
+    c = np.empty((m, n), dtype=np.float32)
+    _check(lib.percache_debug_gemm_noalloc(device, m, n, k, _ptr(np.ascontiguousarray(a_f16)),
+                                           _ptr(np.ascontiguousarray(b_f16)), _ptr(c)), "percache_debug_gemm_noalloc")
     return c
