@@ -199,20 +199,23 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             }
           }
         }
-      } else {   // EPI_SWIGLU: tile columns [0, BN/2) are gate, [BN/2, BN) the matching up columns
+      } else {   // EPI_SWIGLU: every 128-column block holds 64 gate columns, then the matching 64 up columns
 #pragma unroll 1
-        for (int c = 0; c < BN / 2; c += 32) {
-          uint32_t rg[32], ru[32];
-          tmem_ld_32x32(t_acc + c, rg);
-          tmem_ld_32x32(t_acc + BN / 2 + c, ru);
-          tmem_wait_ld();
-          if (row_ok) {
+        for (int hl = 0; hl < BN / 128; ++hl) {
+#pragma unroll 1
+          for (int half = 0; half < 2; ++half) {
+            uint32_t rg[32], ru[32];
+            tmem_ld_32x32(t_acc + hl * 128 + half * 32, rg);
+            tmem_ld_32x32(t_acc + hl * 128 + 64 + half * 32, ru);
+            tmem_wait_ld();
+            if (row_ok) {
 #pragma unroll
-            for (int seg = 0; seg < 4; ++seg) {
-              float g[8], u[8];
-              u32x8_to_float(rg + seg * 8, g);
-              u32x8_to_float(ru + seg * 8, u);
-              swiglu_store8(args.swi, row, n_idx * (BN / 2) + c + seg * 8, g, u);
+              for (int seg = 0; seg < 4; ++seg) {
+                float g[8], u[8];
+                u32x8_to_float(rg + seg * 8, g);
+                u32x8_to_float(ru + seg * 8, u);
+                swiglu_store8(args.swi, row, (n_idx * (BN / 128) + hl) * 64 + half * 32 + seg * 8, g, u);
+              }
             }
           }
         }
@@ -289,27 +292,41 @@ int umma_gemm_block_n(GemmEpilogueKind kind) {
   return 128;
 }
 
+// Tile width for a problem: 256 columns once that still gives every SM a tile, else 128.
+int umma_gemm_pick_block_n(int M, int N, int n_sms) {
+  if (N % 256 != 0) return 128;
+  const int m_tiles = (M + BM - 1) / BM;
+  return m_tiles * (N / 256) >= n_sms ? 256 : 128;
+}
+
+template <int BN>
+static int launch_bn(const GemmOperand& A, const GemmOperand& B, GemmArgs& args, GemmEpilogueKind kind,
+                     const void* epilogue, int n_sms, cudaStream_t s) {
+  switch (kind) {
+    case EPI_STORE_F32:
+      return launch_one<BN, EPI_STORE_F32>(A, B, args, n_sms, s);
+    case EPI_QKV:
+      args.qkv = *static_cast<const QkvEpilogue*>(epilogue);
+      return launch_one<BN, EPI_QKV>(A, B, args, n_sms, s);
+    case EPI_RESIDUAL:
+      args.res = *static_cast<const ResidualEpilogue*>(epilogue);
+      return launch_one<BN, EPI_RESIDUAL>(A, B, args, n_sms, s);
+    case EPI_SWIGLU:
+      args.swi = *static_cast<const SwigluEpilogue*>(epilogue);
+      return launch_one<BN, EPI_SWIGLU>(A, B, args, n_sms, s);
+  }
+  return -1;
+}
+
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
                      cudaStream_t s) {
   if (M <= 0) return 0;
-  if (K % BK != 0 || N % block_n != 0 || block_n != 128) return -1;
+  if (K % BK != 0 || N % block_n != 0 || (block_n != 128 && block_n != 256)) return -1;
   GemmArgs args{};
   args.M = M; args.N = N; args.K = K; args.c = c_f32; args.err_word = err_word;
-  switch (kind) {
-    case EPI_STORE_F32:
-      return launch_one<128, EPI_STORE_F32>(A, B, args, n_sms, s);
-    case EPI_QKV:
-      args.qkv = *static_cast<const QkvEpilogue*>(epilogue);
-      return launch_one<128, EPI_QKV>(A, B, args, n_sms, s);
-    case EPI_RESIDUAL:
-      args.res = *static_cast<const ResidualEpilogue*>(epilogue);
-      return launch_one<128, EPI_RESIDUAL>(A, B, args, n_sms, s);
-    case EPI_SWIGLU:
-      args.swi = *static_cast<const SwigluEpilogue*>(epilogue);
-      return launch_one<128, EPI_SWIGLU>(A, B, args, n_sms, s);
-  }
-  return -1;
+  return block_n == 256 ? launch_bn<256>(A, B, args, kind, epilogue, n_sms, s)
+                        : launch_bn<128>(A, B, args, kind, epilogue, n_sms, s);
 }
 
 }  // namespace pc

@@ -94,7 +94,8 @@ int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t c
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
                      cudaStream_t s);
-int umma_gemm_block_n(GemmEpilogueKind kind);    // block_n a B operand map must be built for
+int umma_gemm_block_n(GemmEpilogueKind kind);    // narrowest N tile (a B operand map needs box_rows = the tile used)
+int umma_gemm_pick_block_n(int M, int N, int n_sms);   // 128 or 256 for this problem
 
 // rank-N fp16 tensor map with 128-byte swizzle; dims/strides innermost first (strides in bytes, from dim 1)
 int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,

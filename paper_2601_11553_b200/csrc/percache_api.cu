@@ -23,7 +23,8 @@ struct ChunkEntry {
 struct LayerWeights {
   __half *wqkv = nullptr, *wo = nullptr, *wgu = nullptr, *wd = nullptr;
   float *g_attn = nullptr, *g_ffn = nullptr;
-  GemmOperand m_wqkv, m_wo, m_wgu, m_wd;
+  GemmOperand m_wqkv, m_wo, m_wgu, m_wd;                  // B maps with 128-row boxes
+  GemmOperand m_wqkv256, m_wo256, m_wgu256, m_wd256;      // and with 256-row boxes
   AttnMaps attn_maps;
 };
 
@@ -314,6 +315,9 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
     cuda_ok = cuda_ok && make_operand_map(&W.m_wqkv, W.wqkv, D.qkv_dim, d, bn) == 0 &&
               make_operand_map(&W.m_wo, W.wo, d, D.q_dim, bn) == 0 &&
               make_operand_map(&W.m_wgu, W.wgu, 2 * F, d, bn) == 0 && make_operand_map(&W.m_wd, W.wd, d, F, bn) == 0;
+    cuda_ok = cuda_ok && make_operand_map(&W.m_wqkv256, W.wqkv, D.qkv_dim, d, 256) == 0 &&
+              make_operand_map(&W.m_wo256, W.wo, d, D.q_dim, 256) == 0 &&
+              make_operand_map(&W.m_wgu256, W.wgu, 2 * F, d, 256) == 0 && make_operand_map(&W.m_wd256, W.wd, d, F, 256) == 0;
     cuda_ok = cuda_ok && make_attn_maps(&W.attn_maps, h->qbuf, h->m_cap, D.q_dim, h->kctx + l * ctx_layer,
                                         h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim) == 0;
   }
@@ -661,7 +665,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_gemm(h->xn, W.wqkv, h->cref, Mi, D.qkv_dim, d, s);
       launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
     } else {
-      ok = ok && launch_umma_gemm(h->m_xn, W.m_wqkv, Mi, D.qkv_dim, d, 128, EPI_QKV, &qe, nullptr, h->d_err, h->n_sms, s) == 0;
+      {
+        const int bn = umma_gemm_pick_block_n(Mi, D.qkv_dim, h->n_sms);
+        ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
+                                    h->d_err, h->n_sms, s) == 0;
+      }
     }
     timer.end();
 
@@ -680,7 +688,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_gemm(h->attn_out, W.wo, h->cref, Mi, d, D.q_dim, s);
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
-      ok = ok && launch_umma_gemm(h->m_attn, W.m_wo, Mi, d, D.q_dim, 128, EPI_RESIDUAL, &re, nullptr, h->d_err, h->n_sms, s) == 0;
+      {
+        const int bn = umma_gemm_pick_block_n(Mi, d, h->n_sms);
+        ok = ok && launch_umma_gemm(h->m_attn, bn == 256 ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s) == 0;
+      }
     }
     timer.end();
 
@@ -694,7 +706,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_gemm(h->xn, W.wgu, h->cref, Mi, 2 * D.d_ffn, d, s);
       launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
     } else {
-      ok = ok && launch_umma_gemm(h->m_xn, W.m_wgu, Mi, 2 * D.d_ffn, d, 128, EPI_SWIGLU, &se, nullptr, h->d_err, h->n_sms, s) == 0;
+      {
+        const int bn = umma_gemm_pick_block_n(Mi, 2 * D.d_ffn, h->n_sms);
+        ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
+                                    h->d_err, h->n_sms, s) == 0;
+      }
     }
     timer.end();
 
@@ -703,7 +719,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_gemm(h->act, W.wd, h->cref, Mi, d, D.d_ffn, s);
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
-      ok = ok && launch_umma_gemm(h->m_act, W.m_wd, Mi, d, D.d_ffn, 128, EPI_RESIDUAL, &re, nullptr, h->d_err, h->n_sms, s) == 0;
+      {
+        const int bn = umma_gemm_pick_block_n(Mi, d, h->n_sms);
+        ok = ok && launch_umma_gemm(h->m_act, bn == 256 ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s) == 0;
+      }
     }
     timer.end();
   }
@@ -815,8 +835,9 @@ int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const v
       GemmOperand mA, mB;
       int n_sms = 148;
       cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, device);
-      if (make_operand_map(&mA, dA, static_cast<int64_t>(m_pad), K, 128) != 0 || make_operand_map(&mB, dB, N, K, 128) != 0 ||
-          launch_umma_gemm(mA, mB, M, N, K, 128, EPI_STORE_F32, nullptr, dC, dErr, n_sms, nullptr) != 0)
+      const int bn = (N % 256 == 0 && M >= 512) ? 256 : 128;     // both tile widths get exercised by the tests
+      if (make_operand_map(&mA, dA, static_cast<int64_t>(m_pad), K, 128) != 0 || make_operand_map(&mB, dB, N, K, bn) != 0 ||
+          launch_umma_gemm(mA, mB, M, N, K, bn, EPI_STORE_F32, nullptr, dC, dErr, n_sms, nullptr) != 0)
         rc = PERCACHE_E_CUDA;
     }
     if (rc == PERCACHE_OK && (cudaDeviceSynchronize() != cudaSuccess || cudaGetLastError() != cudaSuccess)) rc = PERCACHE_E_CUDA;
