@@ -37,6 +37,8 @@ struct AttnArgs {
   int32_t n_tiles;
   const int32_t* row_pos;
   __half* out;
+  float* partial_o;
+  float* partial_ml;
   int32_t n_q_heads, n_kv_heads;
   float scale_log2;      // log2(e) / sqrt(head_dim)
   int* err_word;
@@ -81,10 +83,13 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     tmem_alloc<512>(&tmem_base_slot);
     tmem_relinquish();
   }
+  if (warp == 8 && lane == 0) { prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV); }
+  pdl_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
+  pdl_wait();                 // Q and the assembled context come from earlier kernels
 
   const int n_units = args.n_tiles * args.n_kv_heads;
   const int group = args.n_q_heads / args.n_kv_heads;      // query heads per KV head (even)
@@ -95,14 +100,13 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
-      prefetch_tmap(&tmQ); prefetch_tmap(&tmK); prefetch_tmap(&tmV);
       uint32_t unit_it = 0, kvit = 0;
       bool ok = true;
       for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
         const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
         const int gp = w % (args.n_kv_heads * pairs);
         const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
-        const int nb = (t.kv_len + BLK - 1) / BLK;
+        const int nb = t.blk_end - t.blk_begin;
         if (!mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
         mbar_arrive_expect_tx(&q_full, 2 * TILE_BYTES);
         for (int i = 0; i < 2; ++i)
@@ -116,12 +120,12 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           mbar_arrive_expect_tx(&k_full[st], TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
             tma_load_2d(k_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmK, &k_full[st], g * HEAD_DIM + hf * 64,
-                        t.ctx0 + j * BLK);
+                        t.ctx0 + (t.blk_begin + j) * BLK);
           if (!mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
           mbar_arrive_expect_tx(&v_full[st], TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
             tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmV, &v_full[st], g * HEAD_DIM + hf * 64,
-                        t.ctx0 + j * BLK);
+                        t.ctx0 + (t.blk_begin + j) * BLK);
         }
       }
       if (!ok) {   // error path only: let copies already issued land before shared memory is released
@@ -150,7 +154,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       };
       for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
         const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
-        const int nb = (t.kv_len + BLK - 1) / BLK;
+        const int nb = t.blk_end - t.blk_begin;
         const uint32_t kv0 = kvit;
         if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
         if (!mbar_wait(&k_full[kv0 & 1], (kv0 >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
@@ -205,7 +209,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
       const int gp = w % (args.n_kv_heads * pairs);
       const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
-      const int nb = (t.kv_len + BLK - 1) / BLK;
+      const int nb = t.blk_end - t.blk_begin;
       const uint32_t kv0 = kvit;
       const bool valid = r_in_tile < t.n_rows;
       const int row = t.row0 + (valid ? r_in_tile : t.n_rows - 1);
@@ -221,7 +225,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tmem_wait_ld();
-        const int limit = pos - j * BLK;          // columns 0..limit are visible
+        const int limit = pos - (t.blk_begin + j) * BLK;     // columns 0..limit are visible
         float m_blk = -INFINITY;
         if (limit >= BLK - 1) {
 #pragma unroll
@@ -239,7 +243,8 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
         }
         if (j == 0) {
-          m = m_blk;                               // slot 0 is visible to every row: finite
+          // an item that starts past the row's position sees nothing: keep a finite reference
+          m = m_blk == -INFINITY ? 0.f : m_blk;
         } else {
           const bool need = m_blk > m + RESCALE_THRESHOLD;
           if (__any_sync(0xffffffffu, need)) {
@@ -281,31 +286,48 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         if (lane == 0) mbar_arrive(&p_full[i]);
       }
       if (!ok) break;
-      // ---- final: O_i / l -> fp16 -> out
+      // ---- final: O_i / l -> fp16 -> out, or the unnormalised part -> scratch
       ok = mbar_wait(&o_done[i], (kv0 + nb - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      const float inv_l = 1.0f / l;
-      __half* dst = args.out + (static_cast<size_t>(row) * args.n_q_heads + head) * HEAD_DIM;
+      if (t.partial_base < 0) {
+        const float inv_l = 1.0f / l;
+        __half* dst = args.out + (static_cast<size_t>(row) * args.n_q_heads + head) * HEAD_DIM;
 #pragma unroll 1
-      for (int c = 0; c < 4; ++c) {
-        uint32_t o[32];
-        tmem_ld_32x32(t_o + c * 32, o);
-        tmem_wait_ld();
-        if (valid) {
+        for (int c = 0; c < 4; ++c) {
+          uint32_t o[32];
+          tmem_ld_32x32(t_o + c * 32, o);
+          tmem_wait_ld();
+          if (valid) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            uint32_t pk[4];
+            for (int e = 0; e < 4; ++e) {
+              uint32_t pk[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              __half2 hh = __floats2half2_rn(__uint_as_float(o[8 * e + 2 * q]) * inv_l,
-                                             __uint_as_float(o[8 * e + 2 * q + 1]) * inv_l);
-              pk[q] = *reinterpret_cast<uint32_t*>(&hh);
+              for (int q = 0; q < 4; ++q) {
+                __half2 hh = __floats2half2_rn(__uint_as_float(o[8 * e + 2 * q]) * inv_l,
+                                               __uint_as_float(o[8 * e + 2 * q + 1]) * inv_l);
+                pk[q] = *reinterpret_cast<uint32_t*>(&hh);
+              }
+              *reinterpret_cast<uint4*>(dst + c * 32 + e * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
-            *reinterpret_cast<uint4*>(dst + c * 32 + e * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
           }
         }
+      } else {
+        const size_t slot = static_cast<size_t>(t.partial_base + gp) * 2 + i;
+        float* po = args.partial_o + (slot * BLK + r_in_tile) * HEAD_DIM;
+#pragma unroll 1
+        for (int c = 0; c < 4; ++c) {
+          uint32_t o[32];
+          tmem_ld_32x32(t_o + c * 32, o);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 8; ++e)
+            *reinterpret_cast<uint4*>(po + c * 32 + e * 4) = make_uint4(o[4 * e], o[4 * e + 1], o[4 * e + 2], o[4 * e + 3]);
+        }
+        // a row that saw nothing in this part contributes nothing: l = 0 and reference -inf
+        *reinterpret_cast<float2*>(args.partial_ml + (slot * BLK + r_in_tile) * 2) =
+            make_float2(l > 0.f ? m : -INFINITY, l);
       }
       tc_fence_before_sync();
       __syncwarp();
@@ -340,8 +362,61 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
   return 0;
 }
 
+// Merge of split tiles: out[row][head] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with M = max_s m_s.
+// One warp per (row, head): lanes first take one part each for the (reference, sum) pairs, then every lane
+// owns four output columns and walks the parts with independent 16-byte loads.
+namespace {
+constexpr int MERGE_WARPS = 8;
+__global__ void __launch_bounds__(MERGE_WARPS * 32)
+attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
+                       const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads, int n_kv_heads) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const AttnMerge mg = merges[blockIdx.x];
+  const int group = n_q_heads / n_kv_heads, pairs = group / 2;
+  const int units = n_kv_heads * pairs;
+  const int gp = blockIdx.y >> 1, i = blockIdx.y & 1;
+  const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
+  const int lane = threadIdx.x & 31;
+  const int r = blockIdx.z * MERGE_WARPS + (threadIdx.x >> 5);
+  if (r >= mg.n_rows) return;
+  const size_t slot0 = static_cast<size_t>(mg.partial_base + gp) * 2 + i;
+  const size_t slot_stride = static_cast<size_t>(units) * 2;
+  float M = -INFINITY;
+  for (int s = lane; s < mg.n_parts; s += 32)
+    M = fmaxf(M, partial_ml[((slot0 + s * slot_stride) * BLK + r) * 2]);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+  float l = 0.f;
+#pragma unroll 4
+  for (int s = 0; s < mg.n_parts; ++s) {
+    const size_t slot = slot0 + s * slot_stride;
+    const float2 ml = *reinterpret_cast<const float2*>(partial_ml + (slot * BLK + r) * 2);
+    const float w = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;
+    const float4 o = *reinterpret_cast<const float4*>(partial_o + (slot * BLK + r) * HEAD_DIM + lane * 4);
+    acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
+    acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
+    l = fmaf(w, ml.y, l);
+  }
+  const float inv = 1.0f / l;
+  __half2 a = __floats2half2_rn(acc.x * inv, acc.y * inv), b = __floats2half2_rn(acc.z * inv, acc.w * inv);
+  *reinterpret_cast<uint2*>(out + (static_cast<size_t>(mg.row0 + r) * n_q_heads + head) * HEAD_DIM + lane * 4) =
+      make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+}
+}  // namespace
+
+void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
+                            __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s) {
+  if (n_merges <= 0) return;
+  dim3 grid(n_merges, n_q_heads, BLK / MERGE_WARPS);
+  launch_pdl(attention_merge_kernel, grid, dim3(MERGE_WARPS * 32), 0, s, merges, partial_o, partial_ml, out, n_q_heads,
+             n_kv_heads);
+}
+
 int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
-                          __half* out, int n_q_heads, int n_kv_heads, int* err_word, int n_sms, cudaStream_t s) {
+                          __half* out, float* partial_o, float* partial_ml, int n_q_heads, int n_kv_heads,
+                          int* err_word, int n_sms, cudaStream_t s) {
   if (n_tiles <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0) return -1;
@@ -350,13 +425,14 @@ int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_til
     return -1;
   AttnArgs a{};
   a.tiles = tiles; a.n_tiles = n_tiles; a.row_pos = row_pos; a.out = out;
+  a.partial_o = partial_o; a.partial_ml = partial_ml;
   a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
   a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
   a.err_word = err_word;
   const int n_work = n_tiles * n_kv_heads * (group / 2);
   const int grid = n_work < n_sms ? n_work : n_sms;
-  umma_attention_kernel<<<grid, ATT_THREADS, ATT_SMEM_BYTES, s>>>(maps.q, maps.k, maps.v, a);
-  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+  return launch_pdl(umma_attention_kernel, dim3(grid), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v,
+                    a) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace pc

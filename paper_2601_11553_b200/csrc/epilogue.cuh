@@ -26,11 +26,27 @@ __device__ __forceinline__ uint32_t pack_bf162(__nv_bfloat16 a, __nv_bfloat16 b)
 //      value to the row's position (Appendix B.1: position counter offset by the cached length) and
 //      write it to the assembled context as fp16.
 //   V: round to bf16; keep in the page; write to the assembled context.
-__device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, int hb, int c0, const float (&lo)[8],
-                                           const float (&hi)[8]) {
-  const int pos = e.rows.pos[row];
+// The row's position, context slot and page slot are read once per tile by the caller (QkvRow).
+struct QkvRow { int pos, slot, pool_tok; };
+__device__ __forceinline__ QkvRow load_qkv_row(const QkvEpilogue& e, int row) {
+  return QkvRow{__ldg(e.rows.pos + row), __ldg(e.rows.slot + row), __ldg(e.rows.pool_tok + row)};
+}
+// (cos, sin) of eight consecutive frequencies: read-only path, so the loads may be hoisted above stores
+__device__ __forceinline__ void load_cs8(const float2* cs, float2 (&out)[8]) {
+  const float4* p = reinterpret_cast<const float4*>(cs);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float4 t = __ldg(p + i);
+    out[2 * i] = make_float2(t.x, t.y);
+    out[2 * i + 1] = make_float2(t.z, t.w);
+  }
+}
+__device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c0,
+                                           const float (&lo)[8], const float (&hi)[8]) {
+  const int pos = rw.pos;
   if (hb < e.n_q_heads) {
-    const float2* cs = e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0;
+    float2 cs[8];
+    load_cs8(e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0, cs);
     uint32_t olo[4], ohi[4];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
@@ -46,8 +62,8 @@ __device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, int hb
   const bool is_k = hb < e.n_q_heads + e.n_kv_heads;
   const int kvh = is_k ? hb - e.n_q_heads : hb - e.n_q_heads - e.n_kv_heads;
   const int kv_dim = e.n_kv_heads * HEAD_DIM;
-  const int slot = e.rows.slot[row];
-  const int ptok = e.rows.pool_tok[row];
+  const int slot = rw.slot;
+  const int ptok = rw.pool_tok;
   __nv_bfloat16 blo[8], bhi[8];
 #pragma unroll
   for (int i = 0; i < 8; ++i) {
@@ -63,7 +79,8 @@ __device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, int hb
   }
   uint32_t olo[4], ohi[4];
   if (is_k) {
-    const float2* cs = e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0;
+    float2 cs[8];
+    load_cs8(e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0, cs);
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       const float2 a = cs[2 * i], b = cs[2 * i + 1];
@@ -82,6 +99,21 @@ __device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, int hb
   __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(slot) * kv_dim + kvh * HEAD_DIM + c0;
   *reinterpret_cast<uint4*>(dst) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
   *reinterpret_cast<uint4*>(dst + ROPE_HALF) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+}
+
+// resid[row][col..col+31] += acc: all loads first, then all stores, so the eight 16-byte accesses overlap
+__device__ __forceinline__ void residual_add32(const ResidualEpilogue& e, int row, int col, const uint32_t (&r)[32]) {
+  float4* p = reinterpret_cast<float4*>(e.resid + static_cast<size_t>(row) * e.ld + col);
+  float4 v[8];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = p[i];
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    v[i].x += __uint_as_float(r[4 * i]); v[i].y += __uint_as_float(r[4 * i + 1]);
+    v[i].z += __uint_as_float(r[4 * i + 2]); v[i].w += __uint_as_float(r[4 * i + 3]);
+  }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) p[i] = v[i];
 }
 
 // resid[row][col..col+3] += acc

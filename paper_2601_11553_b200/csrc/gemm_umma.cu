@@ -1,13 +1,14 @@
 // Dense GEMM on the 5th-generation tensor cores: D[M][N] = A[M][K] * B[N][K]^T, fp16 operands,
 // fp32 accumulation in TMEM, fused epilogues (QKV + RoPE + scatter, residual add, SwiGLU).
 //
-// One persistent CTA per SM, 192 threads, warp-specialised:
+// One persistent CTA per SM, 320 threads, warp-specialised:
 //   warp 0    TMA producer: one lane streams 128x64 A tiles and BNx64 B tiles (128-byte swizzle) into
 //             a ring of shared-memory stages, signalling `full` mbarriers by transaction bytes;
 //   warp 1    owns the TMEM allocation; one lane issues tcgen05.mma (128 x BN x 16) on each stage and
 //             commits to the stage's `empty` barrier, then to the accumulator's `tmem_full` barrier;
-//   warps 2-5 epilogue: each reads its 32-lane quarter of the accumulator with tcgen05.ld, applies the
-//             epilogue and stores; two accumulator stages let the next tile's MMAs overlap it.
+//   warps 2-9 epilogue: each reads its 32-lane quarter of the accumulator with tcgen05.ld (two warps per
+//             quarter, alternating 32-column chunks), applies the epilogue and stores; two accumulator
+//             stages let the next tile's MMAs overlap it.
 // Every wait is bounded (ptx.cuh); on a timeout the roles fall through to the common teardown,
 // the producer gives its outstanding copies time to land, TMEM is freed and the host sees the error word.
 #include "epilogue.cuh"
@@ -21,7 +22,7 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;                       // 64 fp16 = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
-constexpr int GEMM_THREADS = 192;
+constexpr int GEMM_THREADS = 320;               // TMA warp, MMA warp, 8 epilogue warps
 constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
 
 template <int BN> struct GemmCfg {
@@ -69,23 +70,27 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 4); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 8); }
     fence_mbar_init();
   }
   if (warp == 1) {
     tmem_alloc<Cfg::TMEM_COLS>(&tmem_base_slot);
     tmem_relinquish();
   }
+  if (warp == 0 && lane == 0) {
+    prefetch_tmap(&tmA);
+    prefetch_tmap(&tmB);
+  }
+  pdl_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
+  pdl_wait();                 // operands and the residual stream come from earlier kernels
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      prefetch_tmap(&tmA);
-      prefetch_tmap(&tmB);
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
@@ -141,8 +146,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------------------------ epilogue (warps 2..9)
+    // Two warps share every TMEM lane quarter and split the tile's columns between them.
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter + 32)
+    const int cgroup = (warp - 2) >> 2;           // 0 or 1: which alternate 32-column chunks this warp takes
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
@@ -158,7 +165,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       const bool row_ok = row < args.M;
       if constexpr (KIND == EPI_STORE_F32 || KIND == EPI_RESIDUAL) {
 #pragma unroll 1
-        for (int c = 0; c < BN; c += 32) {
+        for (int c = cgroup * 32; c < BN; c += 64) {
           uint32_t r[32];
           tmem_ld_32x32(t_acc + c, r);
           tmem_wait_ld();
@@ -171,19 +178,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
                                      __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
             } else {
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                residual_add4(args.res, row, col + 4 * i, __uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
-                              __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+              residual_add32(args.res, row, col, r);
             }
           }
         }
       } else if constexpr (KIND == EPI_QKV) {
+        const QkvRow rw = load_qkv_row(args.qkv, row_ok ? row : 0);
 #pragma unroll 1
         for (int hl = 0; hl < BN / HEAD_DIM; ++hl) {
           const int hb = n_idx * (BN / HEAD_DIM) + hl;
-#pragma unroll 1
-          for (int half = 0; half < 2; ++half) {
+          {
+            const int half = cgroup;
             uint32_t rlo[32], rhi[32];
             tmem_ld_32x32(t_acc + hl * HEAD_DIM + half * 32, rlo);
             tmem_ld_32x32(t_acc + hl * HEAD_DIM + ROPE_HALF + half * 32, rhi);
@@ -194,7 +199,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                 float lo[8], hi[8];
                 u32x8_to_float(rlo + seg * 8, lo);
                 u32x8_to_float(rhi + seg * 8, hi);
-                qkv_store8(args.qkv, row, hb, half * 32 + seg * 8, lo, hi);
+                qkv_store8(args.qkv, row, rw, hb, half * 32 + seg * 8, lo, hi);
               }
             }
           }
@@ -202,8 +207,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       } else {   // EPI_SWIGLU: every 128-column block holds 64 gate columns, then the matching 64 up columns
 #pragma unroll 1
         for (int hl = 0; hl < BN / 128; ++hl) {
-#pragma unroll 1
-          for (int half = 0; half < 2; ++half) {
+          {
+            const int half = cgroup;
             uint32_t rg[32], ru[32];
             tmem_ld_32x32(t_acc + hl * 128 + half * 32, rg);
             tmem_ld_32x32(t_acc + hl * 128 + 64 + half * 32, ru);
@@ -249,8 +254,8 @@ int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args,
   const int n_tiles = ((args.M + BM - 1) / BM) * (args.N / BN);
   if (n_tiles <= 0) return 0;
   const int grid = n_tiles < n_sms ? n_tiles : n_sms;
-  umma_gemm_kernel<BN, KIND><<<grid, GEMM_THREADS, Cfg::SMEM_BYTES, s>>>(A.map, B.map, args);
-  return cudaGetLastError() == cudaSuccess ? 0 : -1;
+  return launch_pdl(umma_gemm_kernel<BN, KIND>, dim3(grid), dim3(GEMM_THREADS), Cfg::SMEM_BYTES, s, A.map, B.map,
+                    args) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace

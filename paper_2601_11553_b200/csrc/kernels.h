@@ -28,14 +28,25 @@ struct RowIndex {
   const int32_t* pool_tok;  // page * 16 + offset where the row's unrotated K/V is kept, or -1
 };
 
-// Attention work tile: up to 128 consecutive new rows of one prompt.
+// Attention work item: up to 128 consecutive new rows of one prompt against the context blocks
+// [blk_begin, blk_end) (128 slots each).  A tile whose context is long and whose batch has few tiles is
+// cut into several items along the context; each then writes an unnormalised partial result to slot
+// `partial_base + (kv head, head pair)` and a second kernel merges the parts.
 struct AttnTile {
-  int32_t row0;       // first new row (global row index)
-  int32_t n_rows;     // 1..128
-  int32_t ctx0;       // global context slot of the prompt's slot 0
-  int32_t kv_len;     // context slots the tile can see: (position of its last row) + 1
-  int32_t min_pos;    // position of its first row
-  int32_t pad0, pad1, pad2;
+  int32_t row0;          // first new row (global row index)
+  int32_t n_rows;        // 1..128
+  int32_t ctx0;          // global context slot of the prompt's slot 0
+  int32_t blk_begin;     // first context block of this item
+  int32_t blk_end;       // one past its last block
+  int32_t partial_base;  // -1: the item covers the tile's whole context and writes the final rows
+  int32_t pad0, pad1;
+};
+
+// Merge of the parts of one split tile.
+struct AttnMerge {
+  int32_t row0, n_rows;
+  int32_t partial_base;  // slot of part 0; part s is at partial_base + s * (kv heads * head pairs)
+  int32_t n_parts;
 };
 
 struct ModelDims {
@@ -105,9 +116,29 @@ int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t*
 struct AttnMaps { CUtensorMap q, k, v; };
 int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, const __half* kctx_layer,
                    const __half* vctx_layer, int64_t ctx_cap, int kv_dim);
+// partial_o: fp32 [slots][2 heads][128 rows][128]; partial_ml: fp32 [slots][2][128][2] (reference max, sum)
 int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
-                          __half* out, int n_q_heads, int n_kv_heads, int* err_word, int n_sms, cudaStream_t s);
+                          __half* out, float* partial_o, float* partial_ml, int n_q_heads, int n_kv_heads,
+                          int* err_word, int n_sms, cudaStream_t s);
+void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
+                            __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
 
 int init_driver_api();   // resolves cuTensorMapEncodeTiled once; 0 on success
+
+// Launch with programmatic stream serialisation (see pdl_wait() in ptx.cuh).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 
 }  // namespace pc

@@ -1,6 +1,7 @@
 // Memory-bound kernels: gather + re-RoPE of cached pages, RMSNorm, format conversions, page copies.
 #include <algorithm>
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace pc {
 
@@ -56,12 +57,14 @@ void launch_interleave_rows_bf16_to_f16(const __nv_bfloat16* gate, const __nv_bf
 __global__ void bf16_to_f32_kernel(const __nv_bfloat16* __restrict__ src, float* __restrict__ dst, int64_t n) {
   int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
+  pdl_launch_dependents();
+  pdl_wait();
   for (; i < n; i += stride) dst[i] = __bfloat162float(src[i]);
 }
 void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStream_t s) {
   if (n <= 0) return;
   const int blocks = static_cast<int>(std::min<int64_t>((n + 255) / 256, 148 * 16));
-  bf16_to_f32_kernel<<<blocks, 256, 0, s>>>(src, dst, n);
+  launch_pdl(bf16_to_f32_kernel, dim3(blocks), dim3(256), 0, s, src, dst, n);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -70,6 +73,8 @@ void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStr
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                       __half* __restrict__ out, int M, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  pdl_launch_dependents();
+  pdl_wait();
   if (row >= M) return;
   const int lane = threadIdx.x & 31;
   const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
@@ -94,7 +99,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 }
 void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s) {
   if (M <= 0) return;
-  rmsnorm_kernel<<<(M + 7) / 8, 256, 0, s>>>(x, gain, out, M, d, eps);
+  launch_pdl(rmsnorm_kernel, dim3((M + 7) / 8), dim3(256), 0, s, x, gain, out, M, d, eps);
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -141,6 +146,8 @@ gather_rerope_kernel(const GatherItem* __restrict__ items, int n_items, int n_la
   const int n_heads = kv_dim / HEAD_DIM;
   const int vec_per_row = kv_dim / 8;
   const int64_t n_units = static_cast<int64_t>(n_items) * n_layers;
+  pdl_launch_dependents();
+  pdl_wait();
   for (int64_t unit = blockIdx.x; unit < n_units; unit += gridDim.x) {
     const int layer = static_cast<int>(unit / n_items);
     const GatherItem it = items[unit % n_items];
@@ -194,8 +201,8 @@ void launch_gather_rerope(const GatherItem* items, int n_items, int n_layers, co
   if (n_items <= 0) return;
   const int64_t units = static_cast<int64_t>(n_items) * n_layers;
   const int blocks = static_cast<int>(std::min<int64_t>(units, 148 * 8));
-  gather_rerope_kernel<<<blocks, GATHER_THREADS, 0, s>>>(items, n_items, n_layers, kpool, vpool, pool_pages, kctx,
-                                                         vctx, ctx_cap, kv_dim, rope);
+  launch_pdl(gather_rerope_kernel, dim3(blocks), dim3(GATHER_THREADS), 0, s, items, n_items, n_layers, kpool, vpool,
+             pool_pages, kctx, vctx, ctx_cap, kv_dim, rope);
 }
 
 // ------------------------------------------------------------------------------------------------

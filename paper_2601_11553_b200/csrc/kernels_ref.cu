@@ -63,7 +63,7 @@ __global__ void ref_qkv_epilogue_kernel(const float* __restrict__ C, int M, QkvE
   float lo[8], hi[8];
 #pragma unroll
   for (int k = 0; k < 8; ++k) { lo[k] = src[k]; hi[k] = src[k + ROPE_HALF]; }
-  qkv_store8(e, row, hb, seg * 8, lo, hi);
+  qkv_store8(e, row, load_qkv_row(e, row), hb, seg * 8, lo, hi);
 }
 void launch_ref_qkv_epilogue(const float* C, int M, const QkvEpilogue& e, cudaStream_t s) {
   if (M <= 0) return;

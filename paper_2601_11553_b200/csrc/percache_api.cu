@@ -3,6 +3,7 @@
 // launches on the caller's stream, commit of missed chunks after success.
 #include <algorithm>
 #include <chrono>
+#include <functional>
 #include <cstring>
 #include <new>
 #include <unordered_map>
@@ -53,6 +54,9 @@ struct percache {
   __nv_bfloat16* xin = nullptr;                         // [m_cap][d]
   __half *xn = nullptr, *qbuf = nullptr, *attn_out = nullptr, *act = nullptr;
   float* cref = nullptr;                                // reference kernels only
+  float *partial_o = nullptr, *partial_ml = nullptr;    // attention parts of split tiles
+  int partial_slots = 0;
+  size_t max_attn_items = 0, max_attn_merges = 0;
   GemmOperand m_xn, m_attn, m_act;
   int64_t m_cap = 0, ctx_cap = 0;
 
@@ -240,7 +244,13 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   ok = ok && dev_alloc(h, &h->d_err, 1);
   // index block: 4 row arrays + gather items (worst case one per context token) + attention tiles
   const size_t max_tiles = static_cast<size_t>(h->m_cap / 128 + cfg->max_batch_prompts + 2);
-  h->index_ints = 4 * static_cast<size_t>(h->m_cap) + 4 * static_cast<size_t>(h->ctx_cap) + 8 * max_tiles;
+  h->partial_slots = 4 * h->n_sms + D.n_q_heads;
+  h->max_attn_items = max_tiles + static_cast<size_t>(h->partial_slots);
+  h->max_attn_merges = max_tiles;
+  h->index_ints = 4 * static_cast<size_t>(h->m_cap) + 4 * static_cast<size_t>(h->ctx_cap) + 8 * h->max_attn_items +
+                  4 * h->max_attn_merges;
+  ok = ok && dev_alloc(h, &h->partial_o, static_cast<size_t>(h->partial_slots) * 2 * 128 * HEAD_DIM);
+  ok = ok && dev_alloc(h, &h->partial_ml, static_cast<size_t>(h->partial_slots) * 2 * 128 * 2);
   ok = ok && dev_alloc(h, &h->d_index, h->index_ints);
   if (ok && cudaMallocHost(reinterpret_cast<void**>(&h->h_index), h->index_ints * sizeof(int32_t)) != cudaSuccess) ok = false;
   if (ok && cudaMallocHost(reinterpret_cast<void**>(&h->h_err), sizeof(int)) != cudaSuccess) ok = false;
@@ -544,7 +554,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   int32_t* row_ctx0 = row_pool + h->m_cap;
   GatherItem* items = reinterpret_cast<GatherItem*>(row_ctx0 + h->m_cap);
   AttnTile* tiles = reinterpret_cast<AttnTile*>(reinterpret_cast<int32_t*>(items) + 4 * h->ctx_cap);
-  int n_items = 0, n_tiles = 0;
+  AttnMerge* merges = reinterpret_cast<AttnMerge*>(reinterpret_cast<int32_t*>(tiles) + 8 * h->max_attn_items);
+  std::vector<AttnTile> base_tiles;
+  int n_items = 0, n_tiles = 0, n_merges = 0;
   plan.slot_chunk.resize(static_cast<size_t>(ctx_total));
   plan.slot_offset.resize(static_cast<size_t>(ctx_total));
   plan.slot_is_new.resize(static_cast<size_t>(ctx_total));
@@ -592,14 +604,76 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       t += len;
     }
     for (int32_t r0 = plan.cu_new[b]; r0 < plan.cu_new[b + 1]; r0 += 128) {
-      AttnTile& a = tiles[n_tiles++];
+      AttnTile a{};
       a.row0 = r0;
       a.n_rows = std::min(128, plan.cu_new[b + 1] - r0);
       a.ctx0 = ctx0;
-      a.kv_len = row_pos[r0 + a.n_rows - 1] + 1;
-      a.min_pos = row_pos[r0];
-      a.pad0 = a.pad1 = a.pad2 = 0;
+      a.blk_begin = 0;
+      a.blk_end = (row_pos[r0 + a.n_rows - 1] + 1 + 127) / 128;     // context blocks its last row can see
+      a.partial_base = -1;
+      base_tiles.push_back(a);
     }
+  }
+  // When the tiles of a batch are few or very unequal, most SMs would idle behind the longest one: tiles may
+  // be cut along the context into parts that a second kernel merges.  The choice is made by a small cost
+  // model (in units of one context block of one item): items are dealt longest-first to the persistent
+  // CTAs; a CTA costs its blocks plus a fixed amount per item, and merging costs a fixed amount.
+  {
+    const int G = D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2);
+    constexpr int ITEM_COST = 3, MERGE_COST = 4;
+    int64_t total_blocks = 0;
+    for (const AttnTile& a : base_tiles) total_blocks += a.blk_end;
+    auto plan_cost = [&](int chunk_blocks, int64_t* slots_out) {
+      std::vector<int> lens;
+      int64_t slots = 0;
+      for (const AttnTile& a : base_tiles) {
+        int n_s = (a.blk_end + chunk_blocks - 1) / chunk_blocks;
+        if (n_s <= 1) { lens.push_back(a.blk_end); continue; }
+        const int part = (a.blk_end + n_s - 1) / n_s;
+        n_s = (a.blk_end + part - 1) / part;
+        slots += static_cast<int64_t>(n_s) * G;
+        for (int sp = 0; sp < n_s; ++sp) lens.push_back(std::min(a.blk_end, (sp + 1) * part) - sp * part);
+      }
+      std::sort(lens.begin(), lens.end(), std::greater<int>());
+      std::vector<int64_t> load(static_cast<size_t>(h->n_sms), 0);
+      size_t w = 0;
+      for (int len : lens)
+        for (int g = 0; g < G; ++g, ++w) load[w % load.size()] += len + ITEM_COST;
+      *slots_out = slots;
+      return *std::max_element(load.begin(), load.end()) + (slots > 0 ? MERGE_COST : 0);
+    };
+    int chunk = INT32_MAX;
+    if (!base_tiles.empty()) {
+      int64_t slots = 0;
+      int64_t best = plan_cost(INT32_MAX, &slots);
+      for (int per_sm = 1; per_sm <= 3; ++per_sm) {
+        const int c = static_cast<int>(std::max<int64_t>(4, (total_blocks * G + per_sm * h->n_sms - 1) / (per_sm * h->n_sms)));
+        const int64_t cost = plan_cost(c, &slots);
+        if (slots <= h->partial_slots && cost * 10 < best * 9) { best = cost; chunk = c; }   // needs a 10 % gain
+      }
+    }
+    int next_slot = 0;
+    std::vector<AttnTile> work;
+    for (const AttnTile& a : base_tiles) {
+      int n_s = (a.blk_end + chunk - 1) / chunk;
+      if (n_s <= 1) { work.push_back(a); continue; }
+      const int part = (a.blk_end + n_s - 1) / n_s;
+      n_s = (a.blk_end + part - 1) / part;
+      AttnMerge& mg = merges[n_merges++];
+      mg.row0 = a.row0; mg.n_rows = a.n_rows; mg.partial_base = next_slot; mg.n_parts = n_s;
+      for (int sp = 0; sp < n_s; ++sp) {
+        AttnTile w = a;
+        w.blk_begin = sp * part;
+        w.blk_end = std::min(a.blk_end, (sp + 1) * part);
+        w.partial_base = next_slot + sp * G;
+        work.push_back(w);
+      }
+      next_slot += n_s * G;
+    }
+    std::stable_sort(work.begin(), work.end(), [](const AttnTile& x, const AttnTile& y) {
+      return (x.blk_end - x.blk_begin) > (y.blk_end - y.blk_begin);
+    });
+    for (const AttnTile& w : work) tiles[n_tiles++] = w;
   }
   const double plan_us =
       std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
@@ -611,7 +685,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   std::memset(st.phase_launches, 0, sizeof(st.phase_launches));
   PhaseTimer timer(h);
   bool ok = true;
-  const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(tiles + n_tiles) - h->h_index);
+  const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(merges + n_merges) - h->h_index);
   ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
   const int32_t* d_row_slot = h->d_index;
@@ -620,6 +694,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   const int32_t* d_row_ctx0 = d_row_pool + h->m_cap;
   const GatherItem* d_items = reinterpret_cast<const GatherItem*>(d_row_ctx0 + h->m_cap);
   const AttnTile* d_tiles = reinterpret_cast<const AttnTile*>(reinterpret_cast<const int32_t*>(d_items) + 4 * h->ctx_cap);
+  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(reinterpret_cast<const int32_t*>(d_tiles) + 8 * h->max_attn_items);
 
   const bool use_ref = (h->flags & PERCACHE_FLAG_REFERENCE_KERNELS) != 0;
   if (use_ref && !h->cref) {
@@ -677,8 +752,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
       launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
     } else {
-      ok = ok && launch_umma_attention(W.attn_maps, d_tiles, n_tiles, d_row_pos, h->attn_out, D.n_q_heads, D.n_kv_heads,
-                                       h->d_err, h->n_sms, s) == 0;
+      ok = ok && launch_umma_attention(W.attn_maps, d_tiles, n_tiles, d_row_pos, h->attn_out, h->partial_o, h->partial_ml,
+                                       D.n_q_heads, D.n_kv_heads, h->d_err, h->n_sms, s) == 0;
+      launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
     }
     timer.end();
 

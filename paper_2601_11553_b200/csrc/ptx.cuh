@@ -30,6 +30,15 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   return t;
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of a prefill call is launched with programmatic stream serialisation: the next kernel's
+// CTAs may start (barrier init, TMEM allocation, descriptor prefetch) while this one is still running.
+// pdl_wait() returns once all kernels this one depends on have completed and their writes are visible;
+// nothing that reads or writes shared buffers may come before it.  Without the launch attribute both
+// are no-ops.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ---------------------------------------------------------------- mbarrier
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
