@@ -17,8 +17,18 @@ __device__ __forceinline__ uint32_t pack_bf162(__nv_bfloat16 a, __nv_bfloat16 b)
   return *reinterpret_cast<uint32_t*>(&h);
 }
 
-// Eight columns c0..c0+7 (c0 < 64, multiple of 8) of the low half of one head and the eight columns
-// 64 higher, for one row.  `hb` is the head block inside the fused QKV output:
+// The row's position, context slot and page slot.
+struct QkvRow { int pos, slot, pool_tok; };
+__device__ __forceinline__ QkvRow load_qkv_row(const QkvEpilogue& e, int row) {
+  return QkvRow{__ldg(e.rows.pos + row), __ldg(e.rows.slot + row), __ldg(e.rows.pool_tok + row)};
+}
+
+__device__ __forceinline__ uint2 pack_half4(float a, float b, float c, float d) {
+  return make_uint2(pack_half2(a, b), pack_half2(c, d));
+}
+
+// Four columns c..c+3 (c < 64, multiple of 4) of the low half of one head and the four columns 64
+// higher, for one row.  `hb` is the head block inside the fused QKV output:
 // [0, Hq) query heads, [Hq, Hq+Hkv) key heads, [Hq+Hkv, Hq+2Hkv) value heads.
 //   Q: rotate to the row's position, round to fp16, write to q_out.
 //   K: round to bf16 (the cache format); keep the unrotated value in the row's page if it has one
@@ -26,112 +36,65 @@ __device__ __forceinline__ uint32_t pack_bf162(__nv_bfloat16 a, __nv_bfloat16 b)
 //      value to the row's position (Appendix B.1: position counter offset by the cached length) and
 //      write it to the assembled context as fp16.
 //   V: round to bf16; keep in the page; write to the assembled context.
-// The row's position, context slot and page slot are read once per tile by the caller (QkvRow).
-struct QkvRow { int pos, slot, pool_tok; };
-__device__ __forceinline__ QkvRow load_qkv_row(const QkvEpilogue& e, int row) {
-  return QkvRow{__ldg(e.rows.pos + row), __ldg(e.rows.slot + row), __ldg(e.rows.pool_tok + row)};
-}
-// (cos, sin) of eight consecutive frequencies: read-only path, so the loads may be hoisted above stores
-__device__ __forceinline__ void load_cs8(const float2* cs, float2 (&out)[8]) {
-  const float4* p = reinterpret_cast<const float4*>(cs);
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    const float4 t = __ldg(p + i);
-    out[2 * i] = make_float2(t.x, t.y);
-    out[2 * i + 1] = make_float2(t.z, t.w);
+// Callers give adjacent lanes adjacent column groups of the same row, so table reads and stores of
+// four lanes cover contiguous 32- to 128-byte pieces.
+__device__ __forceinline__ void qkv_store4(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c, float4 lo,
+                                           float4 hi) {
+  const bool is_q = hb < e.n_q_heads;
+  const bool is_k = !is_q && hb < e.n_q_heads + e.n_kv_heads;
+  float4 t0 = make_float4(1.f, 0.f, 1.f, 0.f), t1 = t0;       // (cos, sin) of columns c, c+1 | c+2, c+3
+  if (is_q || is_k) {
+    const float4* t = reinterpret_cast<const float4*>(e.rope + static_cast<size_t>(rw.pos) * ROPE_HALF + c);
+    t0 = __ldg(t);
+    t1 = __ldg(t + 1);
   }
-}
-__device__ __forceinline__ void qkv_store8(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c0,
-                                           const float (&lo)[8], const float (&hi)[8]) {
-  const int pos = rw.pos;
-  if (hb < e.n_q_heads) {
-    float2 cs[8];
-    load_cs8(e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0, cs);
-    uint32_t olo[4], ohi[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 a = cs[2 * i], b = cs[2 * i + 1];
-      olo[i] = pack_half2(lo[2 * i] * a.x - hi[2 * i] * a.y, lo[2 * i + 1] * b.x - hi[2 * i + 1] * b.y);
-      ohi[i] = pack_half2(hi[2 * i] * a.x + lo[2 * i] * a.y, hi[2 * i + 1] * b.x + lo[2 * i + 1] * b.y);
-    }
-    __half* dst = e.q_out + static_cast<size_t>(row) * (e.n_q_heads * HEAD_DIM) + hb * HEAD_DIM + c0;
-    *reinterpret_cast<uint4*>(dst) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
-    *reinterpret_cast<uint4*>(dst + ROPE_HALF) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
+  if (is_q) {
+    __half* dst = e.q_out + static_cast<size_t>(row) * (e.n_q_heads * HEAD_DIM) + hb * HEAD_DIM + c;
+    *reinterpret_cast<uint2*>(dst) = pack_half4(lo.x * t0.x - hi.x * t0.y, lo.y * t0.z - hi.y * t0.w,
+                                                lo.z * t1.x - hi.z * t1.y, lo.w * t1.z - hi.w * t1.w);
+    *reinterpret_cast<uint2*>(dst + ROPE_HALF) = pack_half4(hi.x * t0.x + lo.x * t0.y, hi.y * t0.z + lo.y * t0.w,
+                                                            hi.z * t1.x + lo.z * t1.y, hi.w * t1.z + lo.w * t1.w);
     return;
   }
-  const bool is_k = hb < e.n_q_heads + e.n_kv_heads;
   const int kvh = is_k ? hb - e.n_q_heads : hb - e.n_q_heads - e.n_kv_heads;
   const int kv_dim = e.n_kv_heads * HEAD_DIM;
-  const int slot = rw.slot;
-  const int ptok = rw.pool_tok;
-  __nv_bfloat16 blo[8], bhi[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    blo[i] = __float2bfloat16_rn(lo[i]);
-    bhi[i] = __float2bfloat16_rn(hi[i]);
+  const __nv_bfloat16 bl0 = __float2bfloat16_rn(lo.x), bl1 = __float2bfloat16_rn(lo.y),
+                      bl2 = __float2bfloat16_rn(lo.z), bl3 = __float2bfloat16_rn(lo.w);
+  const __nv_bfloat16 bh0 = __float2bfloat16_rn(hi.x), bh1 = __float2bfloat16_rn(hi.y),
+                      bh2 = __float2bfloat16_rn(hi.z), bh3 = __float2bfloat16_rn(hi.w);
+  if (rw.pool_tok >= 0) {
+    __nv_bfloat16* p = (is_k ? e.kpool : e.vpool) + static_cast<size_t>(rw.pool_tok) * kv_dim + kvh * HEAD_DIM + c;
+    *reinterpret_cast<uint2*>(p) = make_uint2(pack_bf162(bl0, bl1), pack_bf162(bl2, bl3));
+    *reinterpret_cast<uint2*>(p + ROPE_HALF) = make_uint2(pack_bf162(bh0, bh1), pack_bf162(bh2, bh3));
   }
-  if (ptok >= 0) {
-    __nv_bfloat16* p = (is_k ? e.kpool : e.vpool) + static_cast<size_t>(ptok) * kv_dim + kvh * HEAD_DIM + c0;
-    *reinterpret_cast<uint4*>(p) = make_uint4(pack_bf162(blo[0], blo[1]), pack_bf162(blo[2], blo[3]),
-                                              pack_bf162(blo[4], blo[5]), pack_bf162(blo[6], blo[7]));
-    *reinterpret_cast<uint4*>(p + ROPE_HALF) = make_uint4(pack_bf162(bhi[0], bhi[1]), pack_bf162(bhi[2], bhi[3]),
-                                                          pack_bf162(bhi[4], bhi[5]), pack_bf162(bhi[6], bhi[7]));
-  }
-  uint32_t olo[4], ohi[4];
+  const float l0 = __bfloat162float(bl0), l1 = __bfloat162float(bl1), l2 = __bfloat162float(bl2),
+              l3 = __bfloat162float(bl3);
+  const float h0 = __bfloat162float(bh0), h1 = __bfloat162float(bh1), h2 = __bfloat162float(bh2),
+              h3 = __bfloat162float(bh3);
+  __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(rw.slot) * kv_dim + kvh * HEAD_DIM + c;
   if (is_k) {
-    float2 cs[8];
-    load_cs8(e.rope + static_cast<size_t>(pos) * ROPE_HALF + c0, cs);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float2 a = cs[2 * i], b = cs[2 * i + 1];
-      const float l0 = __bfloat162float(blo[2 * i]), l1 = __bfloat162float(blo[2 * i + 1]);
-      const float h0 = __bfloat162float(bhi[2 * i]), h1 = __bfloat162float(bhi[2 * i + 1]);
-      olo[i] = pack_half2(l0 * a.x - h0 * a.y, l1 * b.x - h1 * b.y);
-      ohi[i] = pack_half2(h0 * a.x + l0 * a.y, h1 * b.x + l1 * b.y);
-    }
+    *reinterpret_cast<uint2*>(dst) = pack_half4(l0 * t0.x - h0 * t0.y, l1 * t0.z - h1 * t0.w, l2 * t1.x - h2 * t1.y,
+                                                l3 * t1.z - h3 * t1.w);
+    *reinterpret_cast<uint2*>(dst + ROPE_HALF) = pack_half4(h0 * t0.x + l0 * t0.y, h1 * t0.z + l1 * t0.w,
+                                                            h2 * t1.x + l2 * t1.y, h3 * t1.z + l3 * t1.w);
   } else {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      olo[i] = pack_half2(__bfloat162float(blo[2 * i]), __bfloat162float(blo[2 * i + 1]));
-      ohi[i] = pack_half2(__bfloat162float(bhi[2 * i]), __bfloat162float(bhi[2 * i + 1]));
-    }
+    *reinterpret_cast<uint2*>(dst) = pack_half4(l0, l1, l2, l3);
+    *reinterpret_cast<uint2*>(dst + ROPE_HALF) = pack_half4(h0, h1, h2, h3);
   }
-  __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(slot) * kv_dim + kvh * HEAD_DIM + c0;
-  *reinterpret_cast<uint4*>(dst) = make_uint4(olo[0], olo[1], olo[2], olo[3]);
-  *reinterpret_cast<uint4*>(dst + ROPE_HALF) = make_uint4(ohi[0], ohi[1], ohi[2], ohi[3]);
-}
-
-// resid[row][col..col+31] += acc: all loads first, then all stores, so the eight 16-byte accesses overlap
-__device__ __forceinline__ void residual_add32(const ResidualEpilogue& e, int row, int col, const uint32_t (&r)[32]) {
-  float4* p = reinterpret_cast<float4*>(e.resid + static_cast<size_t>(row) * e.ld + col);
-  float4 v[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = p[i];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    v[i].x += __uint_as_float(r[4 * i]); v[i].y += __uint_as_float(r[4 * i + 1]);
-    v[i].z += __uint_as_float(r[4 * i + 2]); v[i].w += __uint_as_float(r[4 * i + 3]);
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) p[i] = v[i];
 }
 
 // resid[row][col..col+3] += acc
-__device__ __forceinline__ void residual_add4(const ResidualEpilogue& e, int row, int col, float a0, float a1,
-                                              float a2, float a3) {
+__device__ __forceinline__ void residual_add4(const ResidualEpilogue& e, int row, int col, float4 a) {
   float4* p = reinterpret_cast<float4*>(e.resid + static_cast<size_t>(row) * e.ld + col);
   float4 v = *p;
-  v.x += a0; v.y += a1; v.z += a2; v.w += a3;
+  v.x += a.x; v.y += a.y; v.z += a.z; v.w += a.w;
   *p = v;
 }
 
-// act[row][j0..j0+7] = silu(gate) * up, rounded to fp16
-__device__ __forceinline__ void swiglu_store8(const SwigluEpilogue& e, int row, int j0, const float (&g)[8],
-                                              const float (&u)[8]) {
-  uint32_t o[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) o[i] = pack_half2(silu_f(g[2 * i]) * u[2 * i], silu_f(g[2 * i + 1]) * u[2 * i + 1]);
-  *reinterpret_cast<uint4*>(e.act + static_cast<size_t>(row) * e.ld + j0) = make_uint4(o[0], o[1], o[2], o[3]);
+// act[row][j0..j0+3] = silu(gate) * up, rounded to fp16
+__device__ __forceinline__ void swiglu_store4(const SwigluEpilogue& e, int row, int j0, float4 g, float4 u) {
+  *reinterpret_cast<uint2*>(e.act + static_cast<size_t>(row) * e.ld + j0) =
+      pack_half4(silu_f(g.x) * u.x, silu_f(g.y) * u.y, silu_f(g.z) * u.z, silu_f(g.w) * u.w);
 }
 
 }  // namespace pc

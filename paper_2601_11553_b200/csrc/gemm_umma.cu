@@ -24,12 +24,20 @@ constexpr int BK = 64;                       // 64 fp16 = one 128-byte swizzle r
 constexpr int UMMA_K = 16;
 constexpr int GEMM_THREADS = 320;               // TMA warp, MMA warp, 8 epilogue warps
 constexpr int A_STAGE_BYTES = BM * BK * 2;   // 16 KB
+// Epilogue staging: every epilogue warp owns two buffers of 32 rows x 64 bytes (pitch 80 to spread banks).
+// A thread writes its accumulator row; the warp then reads the buffer back with four lanes per row, so that
+// every global access of the epilogue (residual, RoPE table, outputs) has adjacent lanes on adjacent addresses.
+constexpr int EPI_WARPS = 8;
+constexpr int STG_PITCH = 80;
+constexpr int STG_BUF_BYTES = 32 * STG_PITCH;
+constexpr int EPI_STAGING_BYTES = EPI_WARPS * 2 * STG_BUF_BYTES;   // 40 KB
 
 template <int BN> struct GemmCfg {
   static constexpr int B_STAGE_BYTES = BN * BK * 2;
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  static constexpr int STAGES = (BN >= 256) ? 4 : 6;
-  static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024;   // + slack to align the ring to 1024 B
+  static constexpr int STAGES = (BN >= 256) ? 3 : 5;
+  static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
+  static constexpr int SMEM_BYTES = RING_BYTES + EPI_STAGING_BYTES + 1024;   // + slack to align the ring to 1024 B
   static constexpr int TMEM_COLS = 2 * BN;                         // two accumulator stages
 };
 
@@ -41,11 +49,6 @@ struct GemmArgs {
   SwigluEpilogue swi;        // EPI_SWIGLU
   int* err_word;
 };
-
-__device__ __forceinline__ void u32x8_to_float(const uint32_t* r, float (&f)[8]) {
-#pragma unroll
-  for (int i = 0; i < 8; ++i) f[i] = __uint_as_float(r[i]);
-}
 
 template <int BN, int KIND>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
@@ -150,6 +153,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     // Two warps share every TMEM lane quarter and split the tile's columns between them.
     const int quarter = warp & 3;                 // TMEM lanes [32*quarter, 32*quarter + 32)
     const int cgroup = (warp - 2) >> 2;           // 0 or 1: which alternate 32-column chunks this warp takes
+    uint8_t* stg = ring + Cfg::RING_BYTES + (warp - 2) * 2 * STG_BUF_BYTES;
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     int it = 0;
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
@@ -161,67 +165,78 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t t_acc = tmem_base + lane_base + static_cast<uint32_t>(acc * BN);
-      const int row = m_idx * BM + quarter * 32 + lane;
-      const bool row_ok = row < args.M;
+      const int row_base = m_idx * BM + quarter * 32;          // first of this warp's 32 rows
+      // Two 16-column groups per pass: `ca` and `cb` are tile columns; fn(rl, c4, valid, a, b) gets four
+      // columns of each group (c4 = 0, 4, 8, 12) for local row rl, adjacent lanes on adjacent column groups.
+      auto pass = [&](int ca, int cb, auto&& fn) {
+        uint32_t ra[16], rb[16];
+        tmem_ld_32x16(t_acc + ca, ra);
+        tmem_ld_32x16(t_acc + cb, rb);
+        tmem_wait_ld();
+        uint4* wa = reinterpret_cast<uint4*>(stg + lane * STG_PITCH);
+        uint4* wb = reinterpret_cast<uint4*>(stg + STG_BUF_BYTES + lane * STG_PITCH);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          wa[q] = make_uint4(ra[4 * q], ra[4 * q + 1], ra[4 * q + 2], ra[4 * q + 3]);
+          wb[q] = make_uint4(rb[4 * q], rb[4 * q + 1], rb[4 * q + 2], rb[4 * q + 3]);
+        }
+        __syncwarp();
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          const int rl = it * 8 + (lane >> 2);
+          const float4 a = *reinterpret_cast<const float4*>(stg + rl * STG_PITCH + (lane & 3) * 16);
+          const float4 b = *reinterpret_cast<const float4*>(stg + STG_BUF_BYTES + rl * STG_PITCH + (lane & 3) * 16);
+          fn(rl, (lane & 3) * 4, row_base + rl < args.M, a, b);     // every lane calls fn (it may shuffle)
+        }
+        __syncwarp();
+      };
       if constexpr (KIND == EPI_STORE_F32 || KIND == EPI_RESIDUAL) {
 #pragma unroll 1
         for (int c = cgroup * 32; c < BN; c += 64) {
-          uint32_t r[32];
-          tmem_ld_32x32(t_acc + c, r);
-          tmem_wait_ld();
-          if (row_ok) {
-            const int col = n_idx * BN + c;
+          pass(c, c + 16, [&](int rl, int c4, bool valid, float4 a, float4 b) {
+            if (!valid) return;
+            const int row = row_base + rl, col = n_idx * BN + c + c4;
             if constexpr (KIND == EPI_STORE_F32) {
-              float4* dst = reinterpret_cast<float4*>(args.c + static_cast<size_t>(row) * args.N + col);
-#pragma unroll
-              for (int i = 0; i < 8; ++i)
-                dst[i] = make_float4(__uint_as_float(r[4 * i]), __uint_as_float(r[4 * i + 1]),
-                                     __uint_as_float(r[4 * i + 2]), __uint_as_float(r[4 * i + 3]));
+              float* dst = args.c + static_cast<size_t>(row) * args.N + col;
+              *reinterpret_cast<float4*>(dst) = a;
+              *reinterpret_cast<float4*>(dst + 16) = b;
             } else {
-              residual_add32(args.res, row, col, r);
+              float4* p0 = reinterpret_cast<float4*>(args.res.resid + static_cast<size_t>(row) * args.res.ld + col);
+              float4 v0 = p0[0], v1 = p0[4];
+              v0.x += a.x; v0.y += a.y; v0.z += a.z; v0.w += a.w;
+              v1.x += b.x; v1.y += b.y; v1.z += b.z; v1.w += b.w;
+              p0[0] = v0;
+              p0[4] = v1;
             }
-          }
+          });
         }
       } else if constexpr (KIND == EPI_QKV) {
-        const QkvRow rw = load_qkv_row(args.qkv, row_ok ? row : 0);
+        // every lane keeps the index entries of row (row_base + lane); other lanes fetch them by shuffle
+        const QkvRow mine = load_qkv_row(args.qkv, min(row_base + lane, args.M - 1));
 #pragma unroll 1
         for (int hl = 0; hl < BN / HEAD_DIM; ++hl) {
           const int hb = n_idx * (BN / HEAD_DIM) + hl;
-          {
-            const int half = cgroup;
-            uint32_t rlo[32], rhi[32];
-            tmem_ld_32x32(t_acc + hl * HEAD_DIM + half * 32, rlo);
-            tmem_ld_32x32(t_acc + hl * HEAD_DIM + ROPE_HALF + half * 32, rhi);
-            tmem_wait_ld();
-            if (row_ok) {
-#pragma unroll
-              for (int seg = 0; seg < 4; ++seg) {
-                float lo[8], hi[8];
-                u32x8_to_float(rlo + seg * 8, lo);
-                u32x8_to_float(rhi + seg * 8, hi);
-                qkv_store8(args.qkv, row, rw, hb, half * 32 + seg * 8, lo, hi);
-              }
-            }
+#pragma unroll 1
+          for (int p16 = 0; p16 < 2; ++p16) {
+            const int c0 = cgroup * 32 + p16 * 16;                       // low-half column of this pass
+            pass(hl * HEAD_DIM + c0, hl * HEAD_DIM + ROPE_HALF + c0, [&](int rl, int c4, bool valid, float4 lo, float4 hi) {
+              QkvRow rw;
+              rw.pos = __shfl_sync(0xffffffffu, mine.pos, rl);
+              rw.slot = __shfl_sync(0xffffffffu, mine.slot, rl);
+              rw.pool_tok = __shfl_sync(0xffffffffu, mine.pool_tok, rl);
+              if (valid) qkv_store4(args.qkv, row_base + rl, rw, hb, c0 + c4, lo, hi);
+            });
           }
         }
       } else {   // EPI_SWIGLU: every 128-column block holds 64 gate columns, then the matching 64 up columns
 #pragma unroll 1
         for (int hl = 0; hl < BN / 128; ++hl) {
-          {
-            const int half = cgroup;
-            uint32_t rg[32], ru[32];
-            tmem_ld_32x32(t_acc + hl * 128 + half * 32, rg);
-            tmem_ld_32x32(t_acc + hl * 128 + 64 + half * 32, ru);
-            tmem_wait_ld();
-            if (row_ok) {
-#pragma unroll
-              for (int seg = 0; seg < 4; ++seg) {
-                float g[8], u[8];
-                u32x8_to_float(rg + seg * 8, g);
-                u32x8_to_float(ru + seg * 8, u);
-                swiglu_store8(args.swi, row, (n_idx * (BN / 128) + hl) * 64 + half * 32 + seg * 8, g, u);
-              }
-            }
+#pragma unroll 1
+          for (int p16 = 0; p16 < 2; ++p16) {
+            const int c0 = cgroup * 32 + p16 * 16;
+            pass(hl * 128 + c0, hl * 128 + 64 + c0, [&](int rl, int c4, bool valid, float4 g, float4 u) {
+              if (valid) swiglu_store4(args.swi, row_base + rl, (n_idx * (BN / 128) + hl) * 64 + c0 + c4, g, u);
+            });
           }
         }
       }

@@ -53,21 +53,19 @@ void launch_ref_gemm(const __half* A, const __half* B, float* C, int M, int N, i
 
 __global__ void ref_qkv_epilogue_kernel(const float* __restrict__ C, int M, QkvEpilogue e) {
   const int n_hb = e.n_q_heads + 2 * e.n_kv_heads;
-  const int64_t n = static_cast<int64_t>(M) * n_hb * 8;
+  const int64_t n = static_cast<int64_t>(M) * n_hb * 16;
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   if (i >= n) return;
-  const int seg = static_cast<int>(i % 8);
-  const int hb = static_cast<int>((i / 8) % n_hb);
-  const int row = static_cast<int>(i / (8 * n_hb));
-  const float* src = C + static_cast<size_t>(row) * (n_hb * HEAD_DIM) + hb * HEAD_DIM + seg * 8;
-  float lo[8], hi[8];
-#pragma unroll
-  for (int k = 0; k < 8; ++k) { lo[k] = src[k]; hi[k] = src[k + ROPE_HALF]; }
-  qkv_store8(e, row, load_qkv_row(e, row), hb, seg * 8, lo, hi);
+  const int seg = static_cast<int>(i % 16);
+  const int hb = static_cast<int>((i / 16) % n_hb);
+  const int row = static_cast<int>(i / (16 * n_hb));
+  const float* src = C + static_cast<size_t>(row) * (n_hb * HEAD_DIM) + hb * HEAD_DIM + seg * 4;
+  qkv_store4(e, row, load_qkv_row(e, row), hb, seg * 4, make_float4(src[0], src[1], src[2], src[3]),
+             make_float4(src[ROPE_HALF], src[ROPE_HALF + 1], src[ROPE_HALF + 2], src[ROPE_HALF + 3]));
 }
 void launch_ref_qkv_epilogue(const float* C, int M, const QkvEpilogue& e, cudaStream_t s) {
   if (M <= 0) return;
-  const int64_t n = static_cast<int64_t>(M) * (e.n_q_heads + 2 * e.n_kv_heads) * 8;
+  const int64_t n = static_cast<int64_t>(M) * (e.n_q_heads + 2 * e.n_kv_heads) * 16;
   ref_qkv_epilogue_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(C, M, e);
 }
 
@@ -76,7 +74,7 @@ __global__ void ref_residual_epilogue_kernel(const float* __restrict__ C, int M,
   if (i >= static_cast<int64_t>(M) * (N / 4)) return;
   const int row = static_cast<int>(i / (N / 4)), col = static_cast<int>(i % (N / 4)) * 4;
   const float* c = C + static_cast<size_t>(row) * N + col;
-  residual_add4(e, row, col, c[0], c[1], c[2], c[3]);
+  residual_add4(e, row, col, make_float4(c[0], c[1], c[2], c[3]));
 }
 void launch_ref_residual_epilogue(const float* C, int M, int N, const ResidualEpilogue& e, cudaStream_t s) {
   if (M <= 0) return;
@@ -87,18 +85,16 @@ void launch_ref_residual_epilogue(const float* C, int M, int N, const ResidualEp
 // C is [M][2F] with gate/up interleaved in blocks of `blk` columns: [gate blk | up blk | gate blk | ...]
 __global__ void ref_swiglu_epilogue_kernel(const float* __restrict__ C, int M, int F, int blk, SwigluEpilogue e) {
   const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-  if (i >= static_cast<int64_t>(M) * (F / 8)) return;
-  const int row = static_cast<int>(i / (F / 8)), j0 = static_cast<int>(i % (F / 8)) * 8;
+  if (i >= static_cast<int64_t>(M) * (F / 4)) return;
+  const int row = static_cast<int>(i / (F / 4)), j0 = static_cast<int>(i % (F / 4)) * 4;
   const int b = j0 / blk, jj = j0 % blk;
   const float* g = C + static_cast<size_t>(row) * (2 * F) + static_cast<size_t>(2 * b) * blk + jj;
-  float gv[8], uv[8];
-#pragma unroll
-  for (int k = 0; k < 8; ++k) { gv[k] = g[k]; uv[k] = g[k + blk]; }
-  swiglu_store8(e, row, j0, gv, uv);
+  swiglu_store4(e, row, j0, make_float4(g[0], g[1], g[2], g[3]),
+                make_float4(g[blk], g[blk + 1], g[blk + 2], g[blk + 3]));
 }
 void launch_ref_swiglu_epilogue(const float* C, int M, int F, int blk, const SwigluEpilogue& e, cudaStream_t s) {
   if (M <= 0) return;
-  const int64_t n = static_cast<int64_t>(M) * (F / 8);
+  const int64_t n = static_cast<int64_t>(M) * (F / 4);
   ref_swiglu_epilogue_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(C, M, F, blk, e);
 }
 
