@@ -226,22 +226,20 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tmem_wait_ld();
         const int limit = pos - (t.blk_begin + j) * BLK;     // columns 0..limit are visible
-        float m_blk = -INFINITY;
+        // maximum of the raw scores (the scale is positive, so it commutes with the maximum)
+        float m_raw = -INFINITY;
         if (limit >= BLK - 1) {
 #pragma unroll
-          for (int c = 0; c < 128; ++c) {
-            const float x = __uint_as_float(s[c]) * args.scale_log2;
-            s[c] = __float_as_uint(x);
-            m_blk = fmaxf(m_blk, x);
-          }
+          for (int c = 0; c < 128; c += 2)
+            m_raw = fmaxf(m_raw, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
         } else {
 #pragma unroll
           for (int c = 0; c < 128; ++c) {
-            const float x = c <= limit ? __uint_as_float(s[c]) * args.scale_log2 : -INFINITY;
-            s[c] = __float_as_uint(x);
-            m_blk = fmaxf(m_blk, x);
+            if (c > limit) s[c] = 0xff800000u;                // -inf
+            m_raw = fmaxf(m_raw, __uint_as_float(s[c]));
           }
         }
+        const float m_blk = m_raw * args.scale_log2;
         if (j == 0) {
           // an item that starts past the row's position sees nothing: keep a finite reference
           m = m_blk == -INFINITY ? 0.f : m_blk;
@@ -268,15 +266,18 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
         }
         uint32_t p[64];
-        float sum = 0.f;
+        float sum0 = 0.f, sum1 = 0.f;
+        const float neg_m = -m;
 #pragma unroll
         for (int c = 0; c < 64; ++c) {
-          const float p0 = fast_exp2(__uint_as_float(s[2 * c]) - m);
-          const float p1 = fast_exp2(__uint_as_float(s[2 * c + 1]) - m);
-          sum += p0 + p1;
+          const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * c]), args.scale_log2, neg_m));
+          const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), args.scale_log2, neg_m));
+          sum0 += p0;
+          sum1 += p1;
           __half2 hh = __floats2half2_rn(p0, p1);
           p[c] = *reinterpret_cast<uint32_t*>(&hh);
         }
+        const float sum = sum0 + sum1;
         l += sum;
         tmem_st_32x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&p[0]));
         tmem_st_32x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&p[32]));

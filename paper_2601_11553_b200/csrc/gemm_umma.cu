@@ -312,11 +312,15 @@ int umma_gemm_block_n(GemmEpilogueKind kind) {
   return 128;
 }
 
-// Tile width for a problem: 256 columns once that still gives every SM a tile, else 128.
+// Tile width for a problem.  The main loop is fed at roughly 64 bytes per clock per SM, so a 128 x 128 x 64
+// step (32 KB) costs about 512 clocks and a 128 x 256 x 64 step (48 KB) about 768; the narrower tile only wins
+// when it saves a whole round of tiles over the SMs.
 int umma_gemm_pick_block_n(int M, int N, int n_sms) {
   if (N % 256 != 0) return 128;
   const int m_tiles = (M + BM - 1) / BM;
-  return m_tiles * (N / 256) >= n_sms ? 256 : 128;
+  const int64_t rounds128 = (static_cast<int64_t>(m_tiles) * (N / 128) + n_sms - 1) / n_sms;
+  const int64_t rounds256 = (static_cast<int64_t>(m_tiles) * (N / 256) + n_sms - 1) / n_sms;
+  return rounds256 * 768 <= rounds128 * 512 ? 256 : 128;
 }
 
 template <int BN>
