@@ -43,6 +43,24 @@ def load_peaks():
     return {"hbm_gbs": 6650.0, "tflops_burst": 1590.0, "tflops_sustained": 1400.0, "source": "fallback"}
 
 
+# --------------------------------------------------------------------------- DRAM traffic from ncu
+def kernel_traffic(kernel: str, workload: str):
+    """dram__bytes_read.sum + dram__bytes_write.sum per launch, taken once under ncu (profiles/dram_traffic.json).
+
+    An entry is only used while the kernel's source file still has the hash recorded with it."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    if not os.path.exists(path):
+        return None
+    ent = json.load(open(path)).get(workload, {}).get(kernel)
+    if not ent:
+        return None
+    src = os.path.join(ROOT, "paper_2601_11553_b200", "csrc", ent["source"])
+    if not os.path.exists(src) or hashlib.sha256(open(src, "rb").read()).hexdigest() != ent["sha256"]:
+        return None
+    return ent["dram_bytes_per_launch"]
+
+
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
     """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
@@ -310,6 +328,8 @@ def run_gpu(args):
     roof["peak_source"] = f"{peaks['source']} (sustained bf16 figure x 1.0 nominal fp16/bf16 ratio)" \
         if roof["bound"] == "tensor" else peaks["source"]
     roof["share_of_step"] = phases[dom] / max(sum(phases.values()), 1e-9)
+    roof["traffic"] = kernel_traffic(roof["kernel"], w.name)
+    roof["algorithmic_per_launch"] = gather_bytes if dom == "gather" else fl[dom] / shape.n_layers
     kernels_per_step = (sum(launches[k] for k in pcb.PHASES if k != "io") // args.steps) + 1
 
     cpu = None

@@ -156,10 +156,26 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     uint8_t* stg = ring + Cfg::RING_BYTES + (warp - 2) * 2 * STG_BUF_BYTES;
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
     int it = 0;
+    float4 nv0[4], nv1[4];       // EPI_RESIDUAL: residual values loaded ahead of the pass that consumes them
+    // address of the four columns this lane handles in iteration `it4` of the pass starting at tile column c
+    auto res_ptr = [&](int m_idx, int n_idx, int c, int it4) {
+      const int row = min(m_idx * BM + quarter * 32 + it4 * 8 + (lane >> 2), args.M - 1);
+      return reinterpret_cast<float4*>(args.res.resid + static_cast<size_t>(row) * args.res.ld + n_idx * BN + c +
+                                       (lane & 3) * 4);
+    };
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
       const int m_idx = tile / n_n_tiles, n_idx = tile % n_n_tiles;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
+      if constexpr (KIND == EPI_RESIDUAL) {
+        // the residual values of the tile's first pass travel while the main loop is still running
+#pragma unroll
+        for (int it = 0; it < 4; ++it) {
+          float4* p0 = res_ptr(m_idx, n_idx, cgroup * 32, it);
+          nv0[it] = p0[0];
+          nv1[it] = p0[4];
+        }
+      }
       bool ok = mbar_wait(&tmem_full_bar[acc], acc_phase, args.err_word, DEV_ERR_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -190,23 +206,44 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         }
         __syncwarp();
       };
-      if constexpr (KIND == EPI_STORE_F32 || KIND == EPI_RESIDUAL) {
+      if constexpr (KIND == EPI_STORE_F32) {
 #pragma unroll 1
         for (int c = cgroup * 32; c < BN; c += 64) {
           pass(c, c + 16, [&](int rl, int c4, bool valid, float4 a, float4 b) {
             if (!valid) return;
-            const int row = row_base + rl, col = n_idx * BN + c + c4;
-            if constexpr (KIND == EPI_STORE_F32) {
-              float* dst = args.c + static_cast<size_t>(row) * args.N + col;
-              *reinterpret_cast<float4*>(dst) = a;
-              *reinterpret_cast<float4*>(dst + 16) = b;
-            } else {
-              float4* p0 = reinterpret_cast<float4*>(args.res.resid + static_cast<size_t>(row) * args.res.ld + col);
-              float4 v0 = p0[0], v1 = p0[4];
-              v0.x += a.x; v0.y += a.y; v0.z += a.z; v0.w += a.w;
-              v1.x += b.x; v1.y += b.y; v1.z += b.z; v1.w += b.w;
-              p0[0] = v0;
-              p0[4] = v1;
+            float* dst = args.c + static_cast<size_t>(row_base + rl) * args.N + n_idx * BN + c + c4;
+            *reinterpret_cast<float4*>(dst) = a;
+            *reinterpret_cast<float4*>(dst + 16) = b;
+          });
+        }
+      } else if constexpr (KIND == EPI_RESIDUAL) {
+        // read-modify-write of the fp32 residual stream.  The loads of a pass are issued one pass ahead
+        // (those of the first pass before the accumulator is even waited for, see above) and all before the
+        // stores they pair with: the compiler cannot move a load above a store to the same array by itself.
+#pragma unroll 1
+        for (int c = cgroup * 32; c < BN; c += 64) {
+          float4 v0[4], v1[4];
+#pragma unroll
+          for (int it = 0; it < 4; ++it) { v0[it] = nv0[it]; v1[it] = nv1[it]; }
+          float4* ptr[4];
+#pragma unroll
+          for (int it = 0; it < 4; ++it) {
+            ptr[it] = res_ptr(m_idx, n_idx, c, it);
+            if (c + 64 < BN) {                      // next pass of this tile
+              float4* nx = res_ptr(m_idx, n_idx, c + 64, it);
+              nv0[it] = nx[0];
+              nv1[it] = nx[4];
+            }
+          }
+          int it_ctr = 0;
+          pass(c, c + 16, [&](int rl, int c4, bool valid, float4 a, float4 b) {
+            (void)rl; (void)c4;
+            const int it = it_ctr++;
+            if (valid) {
+              v0[it].x += a.x; v0[it].y += a.y; v0[it].z += a.z; v0[it].w += a.w;
+              v1[it].x += b.x; v1[it].y += b.y; v1[it].z += b.z; v1[it].w += b.w;
+              ptr[it][0] = v0[it];
+              ptr[it][4] = v1[it];
             }
           });
         }
