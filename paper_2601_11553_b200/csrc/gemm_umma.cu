@@ -43,6 +43,7 @@ template <int BN> struct GemmCfg {
 
 struct GemmArgs {
   int32_t M, N, K;
+  int32_t k_splits;          // EPI_RESIDUAL only: the K range of a tile is cut into this many work items
   float* c;                  // EPI_STORE_F32
   QkvEpilogue qkv;           // EPI_QKV
   ResidualEpilogue res;      // EPI_RESIDUAL
@@ -68,8 +69,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   const int n_m_tiles = (args.M + BM - 1) / BM;
   const int n_n_tiles = args.N / BN;
-  const int n_tiles = n_m_tiles * n_n_tiles;
-  const int n_kb = args.K / BK;
+  const int k_splits = (KIND == EPI_RESIDUAL) ? args.k_splits : 1;
+  const int n_tiles = n_m_tiles * n_n_tiles * k_splits;      // work items: (tile, K part)
+  const int n_kb_total = args.K / BK;
+  // item -> (m tile, n tile, first and one-past-last 64-wide K block)
+  auto kb_begin = [&](int item) { return ((item % k_splits) * n_kb_total) / k_splits; };
+  auto kb_end = [&](int item) { return ((item % k_splits + 1) * n_kb_total) / k_splits; };
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
@@ -98,8 +103,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       uint32_t phase = 0;
       bool ok = true;
       for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-        const int m_idx = tile / n_n_tiles, n_idx = tile % n_n_tiles;
-        for (int kb = 0; kb < n_kb; ++kb) {
+        const int m_idx = (tile / k_splits) / n_n_tiles, n_idx = (tile / k_splits) % n_n_tiles;
+        for (int kb = kb_begin(tile); kb < kb_end(tile); ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
           uint8_t* a_dst = ring + stage * Cfg::STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_STAGE_BYTES;
@@ -129,7 +134,8 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
         if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
-        for (int kb = 0; kb < n_kb; ++kb) {
+        const int kb0 = kb_begin(tile), kb1 = kb_end(tile);
+        for (int kb = kb0; kb < kb1; ++kb) {
           if (!mbar_wait(&full_bar[stage], phase, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(ring + stage * Cfg::STAGE_BYTES);
@@ -140,7 +146,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // 16 elements along K = 32 bytes = 2 units of the descriptor's 16-byte address field
             umma_ss(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(2 * k), idesc,
-                    (kb | k) != 0 ? 1u : 0u);
+                    (kb > kb0 || k != 0) ? 1u : 0u);
           }
           umma_commit(&empty_bar[stage]);      // stage reusable once these MMAs have read it
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -164,10 +170,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
                                        (lane & 3) * 4);
     };
     for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const int m_idx = tile / n_n_tiles, n_idx = tile % n_n_tiles;
+      const int m_idx = (tile / k_splits) / n_n_tiles, n_idx = (tile / k_splits) % n_n_tiles;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
-      if constexpr (KIND == EPI_RESIDUAL) {
+      if (KIND == EPI_RESIDUAL && k_splits == 1) {
         // the residual values of the tile's first pass travel while the main loop is still running
 #pragma unroll
         for (int it = 0; it < 4; ++it) {
@@ -214,6 +220,19 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             float* dst = args.c + static_cast<size_t>(row_base + rl) * args.N + n_idx * BN + c + c4;
             *reinterpret_cast<float4*>(dst) = a;
             *reinterpret_cast<float4*>(dst + 16) = b;
+          });
+        }
+      } else if (KIND == EPI_RESIDUAL && k_splits > 1) {
+        // K is split over several work items: each adds its partial sums with vector atomics
+        // (the order of the additions, hence the last bits, then depends on scheduling)
+#pragma unroll 1
+        for (int c = cgroup * 32; c < BN; c += 64) {
+          pass(c, c + 16, [&](int rl, int c4, bool valid, float4 a, float4 b) {
+            if (!valid) return;
+            float4* dst = reinterpret_cast<float4*>(args.res.resid + static_cast<size_t>(row_base + rl) * args.res.ld +
+                                                    n_idx * BN + c + c4);
+            atomicAdd(dst, a);
+            atomicAdd(dst + 4, b);
           });
         }
       } else if constexpr (KIND == EPI_RESIDUAL) {
@@ -303,7 +322,7 @@ int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args,
   if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            Cfg::SMEM_BYTES) != cudaSuccess)
     return -1;
-  const int n_tiles = ((args.M + BM - 1) / BM) * (args.N / BN);
+  const int n_tiles = ((args.M + BM - 1) / BM) * (args.N / BN) * (args.k_splits > 0 ? args.k_splits : 1);
   if (n_tiles <= 0) return 0;
   const int grid = n_tiles < n_sms ? n_tiles : n_sms;
   return launch_pdl(umma_gemm_kernel<BN, KIND>, dim3(grid), dim3(GEMM_THREADS), Cfg::SMEM_BYTES, s, A.map, B.map,
@@ -349,15 +368,33 @@ int umma_gemm_block_n(GemmEpilogueKind kind) {
   return 128;
 }
 
-// Tile width for a problem.  The main loop is fed at roughly 64 bytes per clock per SM, so a 128 x 128 x 64
-// step (32 KB) costs about 512 clocks and a 128 x 256 x 64 step (48 KB) about 768; the narrower tile only wins
-// when it saves a whole round of tiles over the SMs.
-int umma_gemm_pick_block_n(int M, int N, int n_sms) {
-  if (N % 256 != 0) return 128;
+// Tile width (and, for the residual GEMMs, the number of K parts) for a problem.  The main loop is fed at
+// roughly 64 bytes per clock per SM, so a 128 x 128 x 64 step (32 KB) costs about 512 clocks and a
+// 128 x 256 x 64 step (48 KB) about 768; a work item also pays about three steps of ramp-up and tail.
+// The cost of a choice is (rounds of items over the SMs) x (steps per item + 3) x (clocks per step).
+void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, int* block_n, int* k_splits) {
   const int m_tiles = (M + BM - 1) / BM;
-  const int64_t rounds128 = (static_cast<int64_t>(m_tiles) * (N / 128) + n_sms - 1) / n_sms;
-  const int64_t rounds256 = (static_cast<int64_t>(m_tiles) * (N / 256) + n_sms - 1) / n_sms;
-  return rounds256 * 768 <= rounds128 * 512 ? 256 : 128;
+  const int n_kb = K / BK;
+  int64_t best = INT64_MAX;
+  *block_n = 128;
+  *k_splits = 1;
+  for (int bn = 128; bn <= 256; bn += 128) {
+    if (N % bn != 0) continue;
+    const int64_t tiles = static_cast<int64_t>(m_tiles) * (N / bn);
+    for (int sp = 1; sp <= (may_split_k ? 8 : 1); ++sp) {
+      if (sp > 1 && n_kb / sp < 4) break;
+      const int64_t rounds = (tiles * sp + n_sms - 1) / n_sms;
+      const int64_t cost = rounds * ((n_kb + sp - 1) / sp + 3) * (bn == 256 ? 768 : 512);
+      // prefer wider tiles and fewer parts on ties; a split must win by 10 %
+      const bool better = sp == 1 ? cost <= best : cost * 10 < best * 9;
+      if (better) { best = cost; *block_n = bn; *k_splits = sp; }
+    }
+  }
+}
+int umma_gemm_pick_block_n(int M, int N, int n_sms) {
+  int bn, sp;
+  umma_gemm_pick_shape(M, N, 64 * 16, n_sms, false, &bn, &sp);
+  return bn;
 }
 
 template <int BN>
@@ -381,11 +418,12 @@ static int launch_bn(const GemmOperand& A, const GemmOperand& B, GemmArgs& args,
 
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
-                     cudaStream_t s) {
+                     cudaStream_t s, int k_splits) {
   if (M <= 0) return 0;
   if (K % BK != 0 || N % block_n != 0 || (block_n != 128 && block_n != 256)) return -1;
+  if (k_splits < 1 || (k_splits > 1 && kind != EPI_RESIDUAL) || k_splits > K / BK) return -1;
   GemmArgs args{};
-  args.M = M; args.N = N; args.K = K; args.c = c_f32; args.err_word = err_word;
+  args.M = M; args.N = N; args.K = K; args.c = c_f32; args.err_word = err_word; args.k_splits = k_splits;
   return block_n == 256 ? launch_bn<256>(A, B, args, kind, epilogue, n_sms, s)
                         : launch_bn<128>(A, B, args, kind, epilogue, n_sms, s);
 }

@@ -104,9 +104,11 @@ struct GemmOperand {           // a tensor map made once for a fixed buffer
 int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t cols, int box_rows);
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
-                     cudaStream_t s);
+                     cudaStream_t s, int k_splits = 1);
 int umma_gemm_block_n(GemmEpilogueKind kind);    // narrowest N tile (a B operand map needs box_rows = the tile used)
 int umma_gemm_pick_block_n(int M, int N, int n_sms);   // 128 or 256 for this problem
+// tile width and number of K parts (parts > 1 only if may_split_k: the residual epilogue then adds atomically)
+void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, int* block_n, int* k_splits);
 
 // rank-N fp16 tensor map with 128-byte swizzle; dims/strides innermost first (strides in bytes, from dim 1)
 int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,

@@ -741,9 +741,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
     } else {
       {
-        const int bn = umma_gemm_pick_block_n(Mi, D.qkv_dim, h->n_sms);
+        int bn, ks;
+        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, &bn, &ks);
         ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
-                                    h->d_err, h->n_sms, s) == 0;
+                                    h->d_err, h->n_sms, s, ks) == 0;
       }
     }
     timer.end();
@@ -765,9 +766,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
       {
-        const int bn = umma_gemm_pick_block_n(Mi, d, h->n_sms);
+        int bn, ks;
+        umma_gemm_pick_shape(Mi, d, D.q_dim, h->n_sms, true, &bn, &ks);
         ok = ok && launch_umma_gemm(h->m_attn, bn == 256 ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s) == 0;
+                                    h->d_err, h->n_sms, s, ks) == 0;
       }
     }
     timer.end();
@@ -783,9 +785,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
     } else {
       {
-        const int bn = umma_gemm_pick_block_n(Mi, 2 * D.d_ffn, h->n_sms);
+        int bn, ks;
+        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, &bn, &ks);
         ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
-                                    h->d_err, h->n_sms, s) == 0;
+                                    h->d_err, h->n_sms, s, ks) == 0;
       }
     }
     timer.end();
@@ -796,9 +799,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
       {
-        const int bn = umma_gemm_pick_block_n(Mi, d, h->n_sms);
+        int bn, ks;
+        umma_gemm_pick_shape(Mi, d, D.d_ffn, h->n_sms, true, &bn, &ks);
         ok = ok && launch_umma_gemm(h->m_act, bn == 256 ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s) == 0;
+                                    h->d_err, h->n_sms, s, ks) == 0;
       }
     }
     timer.end();
