@@ -64,6 +64,8 @@ extern "C" {
                                                 one-thread-per-output CUDA kernels instead of the tcgen05 ones */
 #define PERCACHE_FLAG_PHASE_TIMING       2u  /* record CUDA events around every kernel class (see stats)       */
 #define PERCACHE_FLAG_REFERENCE_ATTENTION 4u /* debugging aid: plain attention kernel, tcgen05 GEMMs            */
+#define PERCACHE_FLAG_EVICT_LFU          8u  /* when the store is full, evict least-frequently-used chunks instead
+                                                of failing with PERCACHE_E_NOSPACE (see percache_set_store_limit)  */
 
 typedef struct percache percache_t;   /* opaque */
 
@@ -141,6 +143,20 @@ PERCACHE_API int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n
 /* Remove a chunk and free its pages (used to restore the cache state between timed runs). */
 PERCACHE_API int percache_drop_chunk(percache_t* h, uint64_t chunk_id);
 
+/* Capacity management (paper Section 3.2.1: a retrieval counter per cached entry, least-frequently-used
+ * eviction under a configurable storage limit).  Every stored chunk counts the prompts that used it: 1 when a
+ * prompt first stores it (or percache_put_chunk_* inserts it), +1 for every later prompt occurrence that hits it.
+ * With PERCACHE_FLAG_EVICT_LFU, a call that needs more pages than the limit leaves free evicts chunks in order
+ * of (count ascending, insertion order ascending), never one the calling batch itself hits, until the new pages
+ * fit; if they cannot fit the call fails with PERCACHE_E_NOSPACE and nothing is evicted.  Eviction is applied
+ * after every host-side check of the call has passed.
+ * percache_set_store_limit: limit in pages, 1..pool_pages (default pool_pages).  Lowering it below the current
+ * use evicts at once (LFU order) when the flag is set, else fails with PERCACHE_E_NOSPACE. */
+PERCACHE_API int percache_set_store_limit(percache_t* h, int64_t pages);
+
+/* *n_tokens = stored length, *retrievals = the chunk's counter; either pointer may be NULL. */
+PERCACHE_API int percache_chunk_info(percache_t* h, uint64_t chunk_id, int32_t* n_tokens, int64_t* retrievals);
+
 /* Read a stored chunk back: k, v host buffers bf16 [n_layers][n_tokens][n_kv_heads][head_dim]. */
 PERCACHE_API int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* v_host);
 
@@ -174,6 +190,7 @@ typedef struct {
   double  phase_us[PERCACHE_PH_COUNT];         /* filled when PERCACHE_FLAG_PHASE_TIMING is set   */
   int32_t phase_launches[PERCACHE_PH_COUNT];   /* kernels launched per class (always filled)      */
   int64_t attn_visible_pairs;                  /* sum over new rows of (position + 1)             */
+  int64_t evictions;                           /* chunks evicted by the last prefill / put call   */
 } percache_stats_t;
 
 PERCACHE_API int percache_get_stats(percache_t* h, percache_stats_t* out);

@@ -19,6 +19,8 @@ namespace {
 struct ChunkEntry {
   int32_t n_tokens;
   std::vector<int32_t> pages;
+  int64_t retrievals = 1;     // prompts that used this chunk (the one that stored it included)
+  uint64_t serial = 0;        // insertion order
 };
 
 struct LayerWeights {
@@ -69,6 +71,8 @@ struct percache {
 
   std::unordered_map<uint64_t, ChunkEntry> table;
   std::vector<int32_t> free_pages;
+  int64_t store_limit = 0;     // pages the store may use (<= pool_pages)
+  uint64_t next_serial = 0;
 
   Plan plan;
   percache_stats_t stats{};
@@ -154,6 +158,32 @@ void release_pages(percache* h, const std::vector<int32_t>& pages) {
 void refresh_page_stats(percache* h) {
   h->stats.pages_free = static_cast<int64_t>(h->free_pages.size());
   h->stats.pages_used = h->cfg.pool_pages - h->stats.pages_free;
+}
+
+// Pages in use by stored chunks.
+int64_t pages_in_use(const percache* h) { return h->cfg.pool_pages - static_cast<int64_t>(h->free_pages.size()); }
+
+// Make `need` more pages fit under the limit.  Without the LFU flag this only checks.  With it, chunks are
+// evicted least-frequently-used first (ties: oldest first), never one whose id is in `keep`.  Nothing is
+// evicted unless the whole request can be met.  Returns the number of chunks evicted, or a negative code.
+int make_room(percache* h, int64_t need, const std::unordered_map<uint64_t, int64_t>& keep) {
+  int64_t over = pages_in_use(h) + need - h->store_limit;
+  if (over <= 0) return 0;
+  if (!(h->flags & PERCACHE_FLAG_EVICT_LFU)) return PERCACHE_E_NOSPACE;
+  std::vector<std::pair<std::pair<int64_t, uint64_t>, uint64_t>> order;     // ((count, serial), id)
+  for (const auto& kv : h->table)
+    if (!keep.count(kv.first)) order.push_back({{kv.second.retrievals, kv.second.serial}, kv.first});
+  std::sort(order.begin(), order.end());
+  size_t n_evict = 0;
+  for (; n_evict < order.size() && over > 0; ++n_evict)
+    over -= static_cast<int64_t>(h->table[order[n_evict].second].pages.size());
+  if (over > 0) return PERCACHE_E_NOSPACE;
+  for (size_t i = 0; i < n_evict; ++i) {
+    auto it = h->table.find(order[i].second);
+    release_pages(h, it->second.pages);
+    h->table.erase(it);
+  }
+  return static_cast<int>(n_evict);
 }
 
 // upload a page list through the pinned index block and run `fn` with the device pointer
@@ -345,8 +375,29 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   h->free_pages.resize(static_cast<size_t>(cfg->pool_pages));
   for (int64_t i = 0; i < cfg->pool_pages; ++i)
     h->free_pages[static_cast<size_t>(i)] = static_cast<int32_t>(cfg->pool_pages - 1 - i);   // pops give 0, 1, 2, ...
+  h->store_limit = cfg->pool_pages;
   refresh_page_stats(h);
   *out = h;
+  return PERCACHE_OK;
+}
+
+int percache_set_store_limit(percache_t* h, int64_t pages) {
+  if (!h || pages < 1 || pages > h->cfg.pool_pages) return PERCACHE_E_INVAL;
+  const int64_t old = h->store_limit;
+  h->store_limit = pages;
+  const int rc = make_room(h, 0, {});
+  if (rc < 0) { h->store_limit = old; return rc; }
+  h->stats.evictions = rc;
+  refresh_page_stats(h);
+  return PERCACHE_OK;
+}
+
+int percache_chunk_info(percache_t* h, uint64_t chunk_id, int32_t* n_tokens, int64_t* retrievals) {
+  if (!h) return PERCACHE_E_INVAL;
+  auto it = h->table.find(chunk_id);
+  if (it == h->table.end()) return PERCACHE_E_NOTFOUND;
+  if (n_tokens) *n_tokens = it->second.n_tokens;
+  if (retrievals) *retrievals = it->second.retrievals;
   return PERCACHE_OK;
 }
 
@@ -387,7 +438,11 @@ int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, co
   const int n_pages = (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
   ChunkEntry ent;
   ent.n_tokens = n_tokens;
-  int rc = alloc_pages(h, n_pages, &ent.pages);
+  ent.serial = h->next_serial++;
+  int rc = make_room(h, n_pages, {});
+  if (rc < 0) return rc;
+  h->stats.evictions = rc;
+  rc = alloc_pages(h, n_pages, &ent.pages);
   if (rc != PERCACHE_OK) return rc;
   const size_t elems = static_cast<size_t>(h->dims.n_layers) * n_tokens * h->dims.kv_dim;
   __nv_bfloat16 *dk = nullptr, *dv = nullptr;
@@ -426,7 +481,11 @@ int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tok
   if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
   ChunkEntry ent;
   ent.n_tokens = n_tokens;
-  int rc = alloc_pages(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
+  ent.serial = h->next_serial++;
+  int rc = make_room(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, {});
+  if (rc < 0) return rc;
+  h->stats.evictions = rc;
+  rc = alloc_pages(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
   if (rc != PERCACHE_OK) return rc;
   rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
     launch_fill_synthetic(h->kpool, h->vpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim,
@@ -479,6 +538,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   std::vector<Seg> segs;
   std::vector<std::vector<uint8_t>> hit(n_prompts);
   std::unordered_map<uint64_t, std::pair<int, int>> first_miss;      // id -> (prompt, chunk) that will store it
+  std::unordered_map<uint64_t, int64_t> hit_uses;                    // id -> prompt occurrences that hit it
   Plan plan;
   plan.cu_ctx.assign(1, 0);
   plan.cu_new.assign(1, 0);
@@ -500,6 +560,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
         hit[b][i] = 1;
         ++chunks_hit;
         hit_tokens += len;
+        ++hit_uses[P.chunk_ids[i]];
       } else {
         if (!P.chunk_hidden || !P.chunk_hidden[i]) return PERCACHE_E_MISS_NO_INPUT;
         ++chunks_missed;
@@ -522,7 +583,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     plan.cu_ctx.push_back(static_cast<int32_t>(ctx_total));
     plan.cu_new.push_back(static_cast<int32_t>(new_total));
   }
-  if (pages_needed > static_cast<int64_t>(h->free_pages.size())) return PERCACHE_E_NOSPACE;
+  // every host-side check has passed: make the new pages fit (may evict, never a chunk this batch hits)
+  const int evicted = make_room(h, pages_needed, hit_uses);
+  if (evicted < 0) return evicted;
 
   // ---------------------------------------------------------------- pages for the chunks that will be stored
   std::vector<std::pair<uint64_t, ChunkEntry>> pending;
@@ -536,6 +599,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       if (fm->second.first != b || fm->second.second != i) continue;
       ChunkEntry ent;
       ent.n_tokens = prompts[b].chunk_len[i];
+      ent.serial = h->next_serial++;
       alloc_pages(h, (ent.n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
       all_new_pages.insert(all_new_pages.end(), ent.pages.begin(), ent.pages.end());
       pending_of.emplace(id, pending.size());
@@ -824,6 +888,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
 
   // ---------------------------------------------------------------- commit
   for (auto& pe : pending) h->table.emplace(pe.first, std::move(pe.second));
+  for (const auto& hu : hit_uses) h->table[hu.first].retrievals += hu.second;
+  st.evictions = evicted;
   for (int b = 0; b < n_prompts; ++b) {
     results[b].n_new = plan.cu_new[b + 1] - plan.cu_new[b];
     results[b].n_total = plan.cu_ctx[b + 1] - plan.cu_ctx[b];

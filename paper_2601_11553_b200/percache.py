@@ -24,12 +24,12 @@ LIB_PATH = os.path.join(_HERE, "libpercache.so")
 OK = 0
 E_INVAL, E_NOMEM, E_NOSPACE, E_EXISTS, E_LEN_MISMATCH = -1, -2, -3, -4, -5
 E_MISS_NO_INPUT, E_CAPACITY, E_DEVICE_TIMEOUT, E_CUDA, E_NOTFOUND = -6, -7, -8, -9, -10
-FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION = 1, 2, 4
+FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION, FLAG_EVICT_LFU = 1, 2, 4, 8
 PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
-           "percache_get_stats", "percache_set_flags", "percache_debug_read_plan", "percache_debug_read_ctx",
+           "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx",
            "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_strerror")
 
 
@@ -68,7 +68,7 @@ class StatsStruct(C.Structure):
                 ("ctx_tokens", C.c_int64), ("hit_tokens", C.c_int64), ("new_rows", C.c_int64),
                 ("pages_used", C.c_int64), ("pages_free", C.c_int64), ("host_plan_us", C.c_double),
                 ("device_us", C.c_double), ("phase_us", C.c_double * len(PHASES)),
-                ("phase_launches", C.c_int32 * len(PHASES)), ("attn_visible_pairs", C.c_int64)]
+                ("phase_launches", C.c_int32 * len(PHASES)), ("attn_visible_pairs", C.c_int64), ("evictions", C.c_int64)]
 
 
 _lib = None
@@ -93,6 +93,8 @@ def load_library() -> C.CDLL:
     lib.percache_put_chunk_synthetic.argtypes = [vp, u64, i32, u64]
     lib.percache_get_stats.argtypes = [vp, C.POINTER(StatsStruct)]
     lib.percache_set_flags.argtypes = [vp, C.c_uint32]
+    lib.percache_set_store_limit.argtypes = [vp, i64]
+    lib.percache_chunk_info.argtypes = [vp, u64, C.POINTER(i32), C.POINTER(i64)]
     lib.percache_debug_read_plan.argtypes = [vp, i32, C.POINTER(i32), i64]
     lib.percache_debug_read_plan.restype = i64
     lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
@@ -221,6 +223,18 @@ class PerCache:
             return None
         _check(rc, "percache_has_chunk")
         return int(n.value)
+
+    def set_store_limit(self, pages: int) -> None:
+        _check(self._lib.percache_set_store_limit(self._h, pages), "percache_set_store_limit")
+
+    def chunk_info(self, chunk_id: int):
+        """(n_tokens, retrieval count) of a stored chunk, or None."""
+        n, r = C.c_int32(-1), C.c_int64(-1)
+        rc = self._lib.percache_chunk_info(self._h, chunk_id, C.byref(n), C.byref(r))
+        if rc == E_NOTFOUND:
+            return None
+        _check(rc, "percache_chunk_info")
+        return int(n.value), int(r.value)
 
     def drop_chunk(self, chunk_id: int) -> None:
         _check(self._lib.percache_drop_chunk(self._h, chunk_id), "percache_drop_chunk")

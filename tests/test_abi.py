@@ -44,7 +44,7 @@ def test_struct_sizes_match_header():
     assert C.sizeof(pcb.LayerWeights) == 72
     assert C.sizeof(pcb.PromptStruct) == 56
     assert C.sizeof(pcb.ResultStruct) == 40
-    assert C.sizeof(pcb.StatsStruct) == 176
+    assert C.sizeof(pcb.StatsStruct) == 184
 
 
 def test_argument_validation_needs_no_gpu(lib):
