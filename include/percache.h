@@ -106,6 +106,22 @@ PERCACHE_API int percache_destroy(percache_t* h);
 PERCACHE_API int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens,
                           const void* k, const void* v, int32_t ptr_is_device);
 
+/* How the chunks of a prompt are matched against the store.
+ *  PERCACHE_MATCH_CHUNK_ID     a chunk hits when its id is stored, at whatever place of the list it appears (the
+ *                              K/V of layers > 0 were then computed in some other context).
+ *  PERCACHE_MATCH_PREFIX_PATH  the paper's rule (Section 3.2.2): entries are nodes of a tree whose paths are chunk
+ *                              lists; the first chunk is looked up, then the second as its child, and so on until
+ *                              the first mismatch; every later chunk is computed.  The store key of a node is
+ *                              percache_path_key() of the ids from the first chunk to that node, and the chunks a
+ *                              call computes are stored under their path keys.  Reuse then equals full prefill.
+ * Path keys and plain chunk ids share the handle's one 64-bit key space (two keys collide with probability 2^-64);
+ * percache_has_chunk / _drop_chunk / _chunk_info / _get_chunk_kv take whichever key an entry was stored under. */
+#define PERCACHE_MATCH_CHUNK_ID    0
+#define PERCACHE_MATCH_PREFIX_PATH 1
+
+/* Key of the tree node reached by the path chunk_ids[0..n-1] (n = 0: the root's seed). */
+PERCACHE_API uint64_t percache_path_key(const uint64_t* chunk_ids, int32_t n);
+
 /* A prompt: ordered chunk list plus query tokens (paper Section 3, system overview). */
 typedef struct {
   int32_t n_chunks;
@@ -117,6 +133,7 @@ typedef struct {
   int32_t n_query;                      /* >= 0                                                             */
   const void* query_hidden;             /* bf16 [n_query][d_model]                                          */
   int32_t hidden_on_device;             /* 1: chunk_hidden[i] and query_hidden point to device memory       */
+  int32_t match_mode;                   /* PERCACHE_MATCH_*                                                 */
 } percache_prompt_t;
 
 typedef struct {

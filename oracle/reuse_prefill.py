@@ -202,24 +202,40 @@ class Store:
         del self.kv[cid]
 
 
-def assemble_layout(store: Store, prompt: Prompt) -> Layout:
+def store_keys(prompt: Prompt, match_prefix: bool) -> List:
+    """Key of every chunk of the prompt in the store.
+
+    By id: the chunk id.  By prefix (paper Section 3.2.1: each node of the cache tree is a chunk and each path
+    a chunk list retrieved by a query): the tuple of ids from the first chunk of the list down to this one.
+    """
+    if not match_prefix:
+        return list(prompt.chunk_ids)
+    return [tuple(prompt.chunk_ids[: i + 1]) for i in range(len(prompt.chunk_ids))]
+
+
+def assemble_layout(store: Store, prompt: Prompt, match_prefix: bool = False) -> Layout:
     """Slots 0..T-1 are the chunks in the given order, then the query; position(t) = t.
 
-    A chunk hits when its id is stored (with the same length); every other chunk,
+    A chunk hits when its key is stored (with the same length); every other chunk,
     and every query token, is a new row (Section 3.2.2: only the part not covered by
-    loaded tensors is retained and computed).
+    loaded tensors is retained and computed).  With match_prefix the walk of Section
+    3.2.2 is taken: first chunk, then the second as its child, ... and it stops at the
+    first mismatch, after which every chunk is new.
     """
     n_chunks = len(prompt.chunk_ids)
     hit = np.zeros(n_chunks, dtype=np.uint8)
     slot_chunk: List[int] = []
     slot_off: List[int] = []
     is_new: List[int] = []
-    for i, (cid, n) in enumerate(zip(prompt.chunk_ids, prompt.chunk_len)):
-        if store.has(cid):
-            if store.kv[cid][0].shape[1] != n:
-                raise LengthMismatch(f"chunk {cid}: stored {store.kv[cid][0].shape[1]} tokens, prompt says {n}")
+    keys = store_keys(prompt, match_prefix)
+    walking = True
+    for i, (cid, n) in enumerate(zip(keys, prompt.chunk_len)):
+        if store.has(cid) and store.kv[cid][0].shape[1] != n:
+            raise LengthMismatch(f"chunk {cid}: stored {store.kv[cid][0].shape[1]} tokens, prompt says {n}")
+        if store.has(cid) and (walking or not match_prefix):
             hit[i] = 1
         else:
+            walking = False
             if prompt.chunk_hidden is None or i >= len(prompt.chunk_hidden) or prompt.chunk_hidden[i] is None:
                 raise MissNoInput(f"chunk {cid} missed and no hidden states were given")
         for o in range(n):
@@ -248,7 +264,7 @@ class PromptResult:
 
 
 def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit: bool = True,
-                  keep_ctx: bool = False, round_kv: bool = True) -> List[PromptResult]:
+                  keep_ctx: bool = False, round_kv: bool = True, match_prefix: bool = False) -> List[PromptResult]:
     """Prefill a batch of prompts, taking the K/V of stored chunks from the store.
 
     Hits are decided against the store as it is when the call starts; the prompts of
@@ -256,7 +272,7 @@ def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit:
     (its K/V as computed inside this prompt, sliced on the sequence axis), query
     tokens are not.  If two prompts miss the same chunk the first one's slices are kept.
     """
-    layouts = [assemble_layout(store, p) for p in prompts]         # raises before anything changes
+    layouts = [assemble_layout(store, p, match_prefix) for p in prompts]     # raises before anything changes
     results: List[PromptResult] = []
     pending: List[Tuple[int, np.ndarray, np.ndarray]] = []
     hkv, hd, hq = model.n_kv_heads, model.head_dim, model.n_q_heads
@@ -288,7 +304,7 @@ def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit:
             k_pre[new] = k
             v_all[new] = v
             start = 0
-            for i, (cid, n) in enumerate(zip(prompt.chunk_ids, prompt.chunk_len)):
+            for i, (cid, n) in enumerate(zip(store_keys(prompt, match_prefix), prompt.chunk_len)):
                 if lay.hit_mask[i]:                                 # load and place in order
                     ck, cv = store.kv[cid]
                     k_pre[start:start + n] = ck[l]
@@ -308,7 +324,7 @@ def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit:
                 vc_keep.append(v_all)
         # slice the collected K/V of missed chunks on the sequence axis, one slice per chunk
         start = 0
-        for i, (cid, n) in enumerate(zip(prompt.chunk_ids, prompt.chunk_len)):
+        for i, (cid, n) in enumerate(zip(store_keys(prompt, match_prefix), prompt.chunk_len)):
             if not lay.hit_mask[i]:
                 ks = np.stack([kl[start:start + n] for kl in k_pre_layers])
                 vs = np.stack([vl[start:start + n] for vl in v_layers])

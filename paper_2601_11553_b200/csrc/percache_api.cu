@@ -37,6 +37,15 @@ struct Plan {   // integer description of the last successful call (host)
 
 constexpr int MAX_EVENTS = 1024;
 
+// Key of a path of chunk ids (prefix mode): fold the ids with a 64-bit mixer (the SplitMix64 output function).
+constexpr uint64_t PATH_KEY_SEED = 0x70657263616368ull;
+inline uint64_t path_key_step(uint64_t path, uint64_t id) {
+  uint64_t z = (path ^ id) + 0x9E3779B97F4A7C15ull + (path << 6) + (path >> 2);
+  z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+  z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+  return z ^ (z >> 31);
+}
+
 }  // namespace
 
 struct percache {
@@ -401,6 +410,12 @@ int percache_chunk_info(percache_t* h, uint64_t chunk_id, int32_t* n_tokens, int
   return PERCACHE_OK;
 }
 
+uint64_t percache_path_key(const uint64_t* chunk_ids, int32_t n) {
+  uint64_t path = PATH_KEY_SEED;
+  for (int32_t i = 0; chunk_ids && i < n; ++i) path = path_key_step(path, chunk_ids[i]);
+  return path;
+}
+
 int percache_destroy(percache_t* h) {
   destroy_impl(h);
   return PERCACHE_OK;
@@ -539,6 +554,20 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   std::vector<std::vector<uint8_t>> hit(n_prompts);
   std::unordered_map<uint64_t, std::pair<int, int>> first_miss;      // id -> (prompt, chunk) that will store it
   std::unordered_map<uint64_t, int64_t> hit_uses;                    // id -> prompt occurrences that hit it
+  // Store key of every chunk: its id, or in prefix mode the key of the path of ids up to and including it.
+  std::vector<std::vector<uint64_t>> keys(n_prompts);
+  for (int b = 0; b < n_prompts; ++b) {
+    const percache_prompt_t& P = prompts[b];
+    if (P.n_chunks < 0 || (P.n_chunks > 0 && !P.chunk_ids) ||
+        (P.match_mode != PERCACHE_MATCH_CHUNK_ID && P.match_mode != PERCACHE_MATCH_PREFIX_PATH))
+      return PERCACHE_E_INVAL;
+    keys[b].resize(static_cast<size_t>(P.n_chunks));
+    uint64_t path = PATH_KEY_SEED;
+    for (int i = 0; i < P.n_chunks; ++i) {
+      path = path_key_step(path, P.chunk_ids[i]);
+      keys[b][i] = P.match_mode == PERCACHE_MATCH_PREFIX_PATH ? path : P.chunk_ids[i];
+    }
+  }
   Plan plan;
   plan.cu_ctx.assign(1, 0);
   plan.cu_new.assign(1, 0);
@@ -546,27 +575,31 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   int chunks_hit = 0, chunks_missed = 0;
   for (int b = 0; b < n_prompts; ++b) {
     const percache_prompt_t& P = prompts[b];
-    if (P.n_chunks < 0 || P.n_query < 0 || (P.n_chunks > 0 && (!P.chunk_ids || !P.chunk_len)) ||
-        (P.n_query > 0 && !P.query_hidden))
+    if (P.n_query < 0 || (P.n_chunks > 0 && !P.chunk_len) || (P.n_query > 0 && !P.query_hidden))
       return PERCACHE_E_INVAL;
     hit[b].assign(static_cast<size_t>(P.n_chunks), 0);
     int64_t T = 0, n_new = 0;
+    bool walking = true;      // prefix mode: the match walk stops at the first chunk that is not stored
     for (int i = 0; i < P.n_chunks; ++i) {
       const int len = P.chunk_len[i];
       if (len <= 0) return PERCACHE_E_INVAL;
-      auto it = h->table.find(P.chunk_ids[i]);
-      if (it != h->table.end()) {
-        if (it->second.n_tokens != len) return PERCACHE_E_LEN_MISMATCH;
+      const uint64_t key = keys[b][i];
+      auto it = h->table.find(key);
+      const bool stored = it != h->table.end();
+      if (stored && it->second.n_tokens != len) return PERCACHE_E_LEN_MISMATCH;
+      if (stored && (walking || P.match_mode == PERCACHE_MATCH_CHUNK_ID)) {
         hit[b][i] = 1;
         ++chunks_hit;
         hit_tokens += len;
-        ++hit_uses[P.chunk_ids[i]];
+        ++hit_uses[key];
       } else {
+        walking = false;
         if (!P.chunk_hidden || !P.chunk_hidden[i]) return PERCACHE_E_MISS_NO_INPUT;
         ++chunks_missed;
         n_new += len;
-        if (!first_miss.count(P.chunk_ids[i])) {
-          first_miss.emplace(P.chunk_ids[i], std::make_pair(b, i));
+        // a node below an evicted ancestor may still be stored: it is recomputed but not stored again
+        if (!stored && !first_miss.count(key)) {
+          first_miss.emplace(key, std::make_pair(b, i));
           pages_needed += (len + PAGE_TOKENS - 1) / PAGE_TOKENS;
         }
       }
@@ -594,9 +627,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   for (int b = 0; b < n_prompts; ++b)
     for (int i = 0; i < prompts[b].n_chunks; ++i) {
       if (hit[b][i]) continue;
-      const uint64_t id = prompts[b].chunk_ids[i];
+      const uint64_t id = keys[b][i];
       auto fm = first_miss.find(id);
-      if (fm->second.first != b || fm->second.second != i) continue;
+      if (fm == first_miss.end() || fm->second.first != b || fm->second.second != i) continue;
       ChunkEntry ent;
       ent.n_tokens = prompts[b].chunk_len[i];
       ent.serial = h->next_serial++;
@@ -641,7 +674,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
         plan.slot_is_new[ctx0 + t + o] = is_hit ? 0 : 1;
       }
       if (is_hit) {
-        const ChunkEntry& ent = h->table.find(P.chunk_ids[i])->second;
+        const ChunkEntry& ent = h->table.find(keys[b][i])->second;
         for (int o = 0; o < len; o += PAGE_TOKENS) {
           GatherItem& g = items[n_items++];
           g.dst_slot = ctx0 + t + o;
@@ -652,8 +685,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       } else {
         const ChunkEntry* ent = nullptr;
         if (!is_query) {
-          auto fm = first_miss.find(P.chunk_ids[i]);
-          if (fm->second.first == b && fm->second.second == i) ent = &pending[pending_of[P.chunk_ids[i]]].second;
+          auto fm = first_miss.find(keys[b][i]);
+          if (fm != first_miss.end() && fm->second.first == b && fm->second.second == i)
+            ent = &pending[pending_of[keys[b][i]]].second;
         }
         segs.push_back(Seg{is_query ? P.query_hidden : P.chunk_hidden[i], P.hidden_on_device, static_cast<int>(r), len});
         for (int o = 0; o < len; ++o, ++r) {

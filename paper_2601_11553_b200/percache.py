@@ -30,7 +30,7 @@ PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
            "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx",
-           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_strerror")
+           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_strerror")
 
 
 class PerCacheError(RuntimeError):
@@ -55,7 +55,7 @@ class LayerWeights(C.Structure):
 class PromptStruct(C.Structure):
     _fields_ = [("n_chunks", C.c_int32), ("chunk_ids", C.POINTER(C.c_uint64)), ("chunk_len", C.POINTER(C.c_int32)),
                 ("chunk_hidden", C.POINTER(C.c_void_p)), ("n_query", C.c_int32), ("query_hidden", C.c_void_p),
-                ("hidden_on_device", C.c_int32)]
+                ("hidden_on_device", C.c_int32), ("match_mode", C.c_int32)]
 
 
 class ResultStruct(C.Structure):
@@ -100,10 +100,12 @@ def load_library() -> C.CDLL:
     lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
     lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+    lib.percache_path_key.argtypes = [C.POINTER(u64), i32]
+    lib.percache_path_key.restype = u64
     lib.percache_strerror.argtypes = [C.c_int]
     lib.percache_strerror.restype = C.c_char_p
     for name in EXPORTS:
-        if name not in ("percache_debug_read_plan", "percache_strerror"):
+        if name not in ("percache_debug_read_plan", "percache_strerror", "percache_path_key"):
             getattr(lib, name).restype = C.c_int
     _lib = lib
     return lib
@@ -147,6 +149,7 @@ class PromptSpec:
     chunk_hidden: Optional[Sequence[Any]]        # each: [len, d] uint16 numpy (bf16 bits) or device bf16 tensor, or None
     query_hidden: Any                            # [n_query, d]
     n_query: Optional[int] = None
+    match_prefix: bool = False                   # True: PERCACHE_MATCH_PREFIX_PATH (the paper's prefix-tree walk)
 
 
 @dataclass
@@ -273,7 +276,8 @@ class PerCache:
                             raise ValueError("hidden states of one prompt must be all host or all device")
                         hid[i] = _ptr(hcur)
             nq = int(p.n_query if p.n_query is not None else (0 if p.query_hidden is None else p.query_hidden.shape[0]))
-            ps[b] = PromptStruct(nc, ids, lens, hid, nq, _ptr(p.query_hidden) if nq > 0 else None, 1 if on_dev else 0)
+            ps[b] = PromptStruct(nc, ids, lens, hid, nq, _ptr(p.query_hidden) if nq > 0 else None, 1 if on_dev else 0,
+                                 1 if p.match_prefix else 0)
             keep += [ids, lens, hid]
             if out is not None and out[b] is not None:
                 ob = out[b]
@@ -319,6 +323,12 @@ class PerCache:
         v = np.empty_like(k)
         _check(self._lib.percache_debug_read_ctx(self._h, prompt, layer, _ptr(k), _ptr(v)), "percache_debug_read_ctx")
         return k, v
+
+
+def path_key(chunk_ids: Sequence[int]) -> int:
+    """Store key of the prefix-tree node reached by the path `chunk_ids` (percache_path_key)."""
+    arr = (C.c_uint64 * max(len(chunk_ids), 1))(*[int(c) for c in chunk_ids])
+    return int(load_library().percache_path_key(arr, len(chunk_ids)))
 
 
 def debug_gemm(a_f16: np.ndarray, b_f16: np.ndarray, use_reference: bool = False, device: int = 0) -> np.ndarray:

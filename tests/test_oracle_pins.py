@@ -403,3 +403,47 @@ def test_position_of_new_rows_is_their_slot_not_their_row_index():
     k = orc.round_to_bf16((xn @ model.w(0, "wk").T).reshape(3, shape.n_kv_heads, shape.head_dim))
     assert np.allclose(with_hit.k_ctx[0][8:], orc.rope(k, np.array([8, 9, 10]), model.rope_theta), atol=1e-12)
     assert not np.allclose(with_hit.k_ctx[0][8:], orc.rope(k, np.array([0, 1, 2]), model.rope_theta), atol=1e-3)
+
+
+# --------------------------------------------------------------------------- #
+# prefix-tree matching (the paper's walk): reuse equals full prefill, call after call
+# --------------------------------------------------------------------------- #
+def test_prefix_tree_walk_hand_cases():
+    store = orc.Store()
+    z = lambda n: np.zeros((1, n, 1, 2))
+    store.put((7,), z(3), z(3))
+    store.put((7, 9), z(2), z(2))
+    store.put((5,), z(2), z(2))
+    store.put((8, 9, 4), z(1), z(1))            # a node whose ancestors are gone
+    d = 4
+    hid = lambda n: np.zeros((n, d))
+    # 7 -> 9 matches two levels, then 5 is not a child of (7, 9): computed, although (5,) exists as a root
+    lay = orc.assemble_layout(store, orc.Prompt([7, 9, 5], [3, 2, 2], [None, None, hid(2)], hid(1)), match_prefix=True)
+    assert lay.hit_mask.tolist() == [1, 1, 0]
+    # 9 is not a root: nothing matches, the walk stops at once
+    lay = orc.assemble_layout(store, orc.Prompt([9, 7], [2, 3], [hid(2), hid(3)], hid(1)), match_prefix=True)
+    assert lay.hit_mask.tolist() == [0, 0]
+    # ancestors missing: the stored descendant is not used
+    lay = orc.assemble_layout(store, orc.Prompt([8, 9, 4], [1, 2, 1], [hid(1), hid(2), hid(1)], hid(1)), match_prefix=True)
+    assert lay.hit_mask.tolist() == [0, 0, 0]
+    # by id, any stored chunk matches anywhere
+    store.put(9, z(2), z(2))
+    lay = orc.assemble_layout(store, orc.Prompt([3, 9], [1, 2], [hid(1), None], hid(1)))
+    assert lay.hit_mask.tolist() == [0, 1]
+
+
+def test_prefix_tree_reuse_equals_full_prefill_over_a_sequence_of_queries():
+    shape, weights, model = tiny_model(seed=38, n_layers=3)
+    lens = {1: 6, 5: 9, 7: 4, 9: 11, 12: 5}
+    hs = {c: orc.bf16_bits_to_f64(wl.chunk_hidden_for(38, c, n, shape.d_model)) for c, n in lens.items()}
+    store = orc.Store()
+    queries = [([1, 5, 7], [0, 0, 0]), ([1, 5, 9], [1, 1, 0]), ([1, 5, 9, 12], [1, 1, 1, 0]), ([5, 1], [0, 0]),
+               ([1, 5, 7], [1, 1, 1]), ([1, 9], [1, 0])]
+    for qi, (ids, want_mask) in enumerate(queries):
+        qh = orc.bf16_bits_to_f64(wl.make_hidden(38, (2, qi), 3, shape.d_model))
+        pr = orc.Prompt(ids, [lens[c] for c in ids], [hs[c] for c in ids], qh)
+        res = orc.reuse_prefill(model, store, [pr], match_prefix=True)[0]
+        assert res.layout.hit_mask.tolist() == want_mask, (qi, res.layout.hit_mask)
+        full, _, _ = orc.dense_prefill(model, np.concatenate([hs[c] for c in ids] + [qh]))
+        assert np.allclose(res.out_hidden, full[res.layout.new_slots], atol=1e-9), qi
+    assert (1, 5, 9, 12) in store.kv and (5, 1) in store.kv and (1,) in store.kv and 1 not in store.kv
