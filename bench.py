@@ -365,6 +365,45 @@ def run_gpu(args):
         dist.destroy_process_group()
 
 
+def run_qa_bank(args):
+    """QA-bank lookup (cosine top-1 over all stored query embeddings): streams the bank once per call."""
+    import torch
+    from paper_2601_11553_b200 import percache as pcb
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    n, dim = 65536, 1024                       # 268 MB of fp32 embeddings: larger than L2
+    g = torch.Generator(device=dev).manual_seed(5)
+    bank = torch.randn((n, dim), generator=g, device=dev, dtype=torch.float32)
+    peaks = load_peaks()
+    out = {}
+    for nq in (1, 8):
+        queries = bank[:nq] * 1.5 + 0.1 * torch.randn((nq, dim), generator=g, device=dev)
+        queries = queries.contiguous()
+        stream = torch.cuda.current_stream(dev)
+        for _ in range(max(args.warmup, 3)):
+            pcb.qa_top1(bank, queries, 0.85, device=dev.index, stream=stream.cuda_stream)
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        kus = []
+        for a, b in ev:
+            a.record(stream)
+            idx, score, hit, us = pcb.qa_top1(bank, queries, 0.85, device=dev.index, stream=stream.cuda_stream, timing=True)
+            b.record(stream)
+            kus.append(us)
+        torch.cuda.synchronize(dev)
+        ms = float(np.median([a.elapsed_time(b) for a, b in ev]))
+        kms = float(np.median(kus)) / 1000.0
+        out[nq] = {"ms_per_call": ms, "kernel_ms": kms, "gbs": n * dim * 4 / kms / 1e6, "top1": idx.tolist()[:2]}
+    print(json.dumps({"metric": "qa_bank_lookup_gbs", "value": out[1]["gbs"], "unit": "GB/s", "n_gpus": 1,
+                      "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": out[1]["ms_per_call"], "kernel_ms": out[1]["kernel_ms"],
+                      "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+                      "config": {"workload": "qa_bank", "entries": n, "dim": dim, "bytes_per_call": n * dim * 4,
+                                 "l2": "bank (268 MB) exceeds L2"},
+                      "roofline": {"bound": "hbm", "achieved": out[1]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                   "frac": out[1]["gbs"] / peaks["hbm_gbs"], "traffic": None, "kernel": "qa_top1_kernel<1>",
+                                   "peak_source": peaks["source"]},
+                      "batch_of_8_queries": out[8]}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -374,7 +413,9 @@ def main():
     ap.add_argument("--impl", default="percache", choices=["percache", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.workload == "qa_bank":
+        run_qa_bank(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_gpu(args)

@@ -250,6 +250,19 @@ PERCACHE_API int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32
 PERCACHE_API int percache_debug_gemm_noalloc(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16,
                                 const void* b_f16, float* c);
 
+/* QA-bank lookup (paper Section 3.4.1 "Similar Query Reuse"): cosine similarity of each query embedding with
+ * every stored query embedding, the most similar entry, and whether its similarity exceeds tau_query (then the
+ * cached answer of that entry can be returned without running the model).
+ * bank: device fp32 [n_entries][dim] (dim a multiple of 4, rows 16-byte aligned); queries: device fp32
+ * [n_queries][dim], n_queries <= 8 (PERCACHE_E_CAPACITY beyond).  Outputs are host arrays [n_queries]:
+ * best_index (lowest index among equal maxima), best_score (cosine, fp32 arithmetic), hit (score > tau_query).
+ * kernel_us: optional (may be NULL); receives the kernel's duration from CUDA events on the stream.
+ * Runs on `stream` (a cudaStream_t or NULL) and returns after it has finished.  One lookup at a time per
+ * device and process (the running maxima live in one device-side array of the library). */
+PERCACHE_API int percache_qa_top1(int32_t device, void* stream, const float* bank, int32_t n_entries, int32_t dim,
+                     const float* queries, int32_t n_queries, float tau_query, int32_t* best_index,
+                     float* best_score, uint8_t* hit, float* kernel_us);
+
 PERCACHE_API const char* percache_strerror(int code);
 
 #ifdef __cplusplus

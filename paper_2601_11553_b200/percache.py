@@ -30,7 +30,7 @@ PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
            "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx",
-           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_strerror")
+           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_qa_top1", "percache_strerror")
 
 
 class PerCacheError(RuntimeError):
@@ -100,6 +100,7 @@ def load_library() -> C.CDLL:
     lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
     lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+    lib.percache_qa_top1.argtypes = [i32, vp, vp, i32, i32, vp, i32, C.c_float, vp, vp, vp, C.POINTER(C.c_float)]
     lib.percache_path_key.argtypes = [C.POINTER(u64), i32]
     lib.percache_path_key.restype = u64
     lib.percache_strerror.argtypes = [C.c_int]
@@ -358,3 +359,18 @@ def debug_gemm_noalloc(a_f16: np.ndarray, b_f16: np.ndarray, device: int = 0) ->
     _check(lib.percache_debug_gemm_noalloc(device, m, n, k, _ptr(np.ascontiguousarray(a_f16)),
                                            _ptr(np.ascontiguousarray(b_f16)), _ptr(c)), "percache_debug_gemm_noalloc")
     return c
+
+
+def qa_top1(bank: Any, queries: Any, tau_query: float, device: int = 0, stream: int = 0, timing: bool = False):
+    """percache_qa_top1: bank [n, dim] and queries [q, dim] are fp32 device tensors; returns (index, score, hit)
+    arrays, plus the kernel time in microseconds when timing is set."""
+    n, dim = int(bank.shape[0]), int(bank.shape[1])
+    nq = int(queries.shape[0])
+    idx = np.empty(nq, dtype=np.int32)
+    score = np.empty(nq, dtype=np.float32)
+    hit = np.empty(nq, dtype=np.uint8)
+    us = C.c_float(0.0)
+    _check(load_library().percache_qa_top1(device, C.c_void_p(stream or None), _ptr(bank), n, dim, _ptr(queries), nq,
+                                           C.c_float(tau_query), _ptr(idx), _ptr(score), _ptr(hit),
+                                           C.byref(us) if timing else None), "percache_qa_top1")
+    return (idx, score, hit, float(us.value)) if timing else (idx, score, hit)
