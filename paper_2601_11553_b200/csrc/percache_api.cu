@@ -36,6 +36,7 @@ struct Plan {   // integer description of the last successful call (host)
 };
 
 constexpr int MAX_EVENTS = 1024;
+constexpr int64_t GATHER_OVERLAP_MIN_BYTES = 512ll << 20;   // below this the per-layer waits cost more than they hide
 
 // Key of a path of chunk ids (prefix mode): fold the ids with a 64-bit mixer (the SplitMix64 output function).
 constexpr uint64_t PATH_KEY_SEED = 0x70657263616368ull;
@@ -87,6 +88,11 @@ struct percache {
   percache_stats_t stats{};
   std::vector<cudaEvent_t> events;
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
+  // gather / compute overlap: the per-layer gathers of a large fetch run on `side`, layer l's
+  // attention waits for ev_gather[l]
+  cudaStream_t side = nullptr;
+  cudaEvent_t ev_fork = nullptr;
+  std::vector<cudaEvent_t> ev_gather;
 };
 
 namespace {
@@ -114,6 +120,13 @@ void destroy_impl(percache* h) {
     if (e) cudaEventDestroy(e);
   if (h->ev_begin) cudaEventDestroy(h->ev_begin);
   if (h->ev_end) cudaEventDestroy(h->ev_end);
+  if (h->side) {
+    cudaStreamSynchronize(h->side);
+    cudaStreamDestroy(h->side);
+  }
+  if (h->ev_fork) cudaEventDestroy(h->ev_fork);
+  for (cudaEvent_t e : h->ev_gather)
+    if (e) cudaEventDestroy(e);
   cudaGetLastError();
   delete h;
 }
@@ -312,6 +325,14 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   h->events.assign(MAX_EVENTS, nullptr);
   for (auto& e : h->events)
     if (cudaEventCreate(&e) != cudaSuccess) { destroy_impl(h); return PERCACHE_E_CUDA; }
+  if (cudaStreamCreateWithFlags(&h->side, cudaStreamNonBlocking) != cudaSuccess ||
+      cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess) {
+    destroy_impl(h);
+    return PERCACHE_E_CUDA;
+  }
+  h->ev_gather.assign(D.n_layers, nullptr);
+  for (auto& e : h->ev_gather)
+    if (cudaEventCreateWithFlags(&e, cudaEventDisableTiming) != cudaSuccess) { destroy_impl(h); return PERCACHE_E_CUDA; }
 
   // Operand buffers start as zeros: rows and context slots a call does not write are still read by
   // whole-tile TMA loads (and then masked or never stored), so they must never hold NaN bit patterns.
@@ -808,15 +829,30 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   launch_bf16_to_f32(h->xin, h->resid, M * d, s);
   timer.end();
 
-  if (n_items > 0) {
+  const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
+  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
+  const int Mi = static_cast<int>(M);
+  // The fetch depends on nothing the layers compute (it reads pages of chunks stored by earlier
+  // calls), so a large one runs beside them: one launch per layer on the side stream, and layer l's
+  // attention waits for fetch l alone.  The HBM-bound copies then fill the time the tensor-bound
+  // GEMMs leave the memory system idle.  A small fetch stays one launch ahead of layer 0 (the waits
+  // would cost more than they hide), and so does a phase-timed call, whose fetch time must be clean.
+  const int64_t gather_bytes = hit_tokens * D.kv_dim * 8 * D.n_layers;   // K and V, bf16 in + fp16 out
+  const bool overlap_gather = n_items > 0 && Mi > 0 && !use_ref && !(h->flags & PERCACHE_FLAG_PHASE_TIMING) &&
+                              gather_bytes >= GATHER_OVERLAP_MIN_BYTES;
+  if (overlap_gather) {
+    ok = ok && cudaEventRecord(h->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(h->side, h->ev_fork, 0) == cudaSuccess;
+    for (int l = 0; l < D.n_layers && ok; ++l) {
+      launch_gather_rerope(d_items, n_items, 1, h->kpool + l * pool_layer, h->vpool + l * pool_layer, h->cfg.pool_pages,
+                           h->kctx + l * ctx_layer, h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim, h->rope, h->side);
+      ok = ok && cudaEventRecord(h->ev_gather[l], h->side) == cudaSuccess;
+    }
+  } else if (n_items > 0) {
     timer.begin(PERCACHE_PH_GATHER);
     launch_gather_rerope(d_items, n_items, D.n_layers, h->kpool, h->vpool, h->cfg.pool_pages, h->kctx, h->vctx,
                          h->ctx_cap, D.kv_dim, h->rope, s);
     timer.end();
   }
-  const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
-  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
-  const int Mi = static_cast<int>(M);
   for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
     LayerWeights& W = h->layers[l];
     timer.begin(PERCACHE_PH_NORM);
@@ -848,6 +884,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     timer.end();
 
     timer.begin(PERCACHE_PH_ATTN);
+    if (overlap_gather) ok = ok && cudaStreamWaitEvent(s, h->ev_gather[l], 0) == cudaSuccess;
     if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
       launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
     } else {
@@ -917,6 +954,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   ok = ok && cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
   timer.end();
   const cudaError_t sync_rc = cudaStreamSynchronize(s);
+  if (overlap_gather && !ok) cudaStreamSynchronize(h->side);   // a failed call may have skipped the per-layer joins
   if (!ok || sync_rc != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(PERCACHE_E_CUDA);
   if (*h->h_err != 0) return fail(PERCACHE_E_DEVICE_TIMEOUT);
 
