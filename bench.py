@@ -271,6 +271,7 @@ def run_gpu(args):
         torch.cuda.synchronize(dev)
 
     # ---- warm-up, then the timed region (device-resident inputs), max over ranks
+    h.set_flags(args.flags)
     timed(specs_dev, out_dev, max(args.warmup, 3))
     sampler = ClockSampler(local)
     barrier()
@@ -280,10 +281,10 @@ def run_gpu(args):
     clocks = sampler.stop()
     total_ms = float(sum(ms))
     # ---- same steps with per-kernel-class events (separate pass: the extra events cost a few percent)
-    h.set_flags(pcb.FLAG_PHASE_TIMING)
+    h.set_flags(args.flags | pcb.FLAG_PHASE_TIMING)
     timed(specs_dev, out_dev, 2)
     ms_ph, phases, launches_ph, _, _ = timed(specs_dev, out_dev, args.steps)
-    h.set_flags(0)
+    h.set_flags(args.flags)
     # ---- end to end through host buffers
     timed(specs_host, out_host, 3)
     barrier()
@@ -412,6 +413,7 @@ def main():
     ap.add_argument("--workload", default="cfg1")
     ap.add_argument("--impl", default="percache", choices=["percache", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="PERCACHE_FLAG_* bits kept set during the timed passes")
     args = ap.parse_args()
     if args.workload == "qa_bank":
         run_qa_bank(args)

@@ -64,6 +64,7 @@ extern "C" {
                                                 one-thread-per-output CUDA kernels instead of the tcgen05 ones */
 #define PERCACHE_FLAG_PHASE_TIMING       2u  /* record CUDA events around every kernel class (see stats)       */
 #define PERCACHE_FLAG_REFERENCE_ATTENTION 4u /* debugging aid: plain attention kernel, tcgen05 GEMMs            */
+#define PERCACHE_FLAG_SINGLE_CTA_GEMM   16u  /* debugging aid: never run a GEMM on CTA pairs (256 x 256 tiles)     */
 #define PERCACHE_FLAG_EVICT_LFU          8u  /* when the store is full, evict least-frequently-used chunks instead
                                                 of failing with PERCACHE_E_NOSPACE (see percache_set_store_limit)  */
 
@@ -222,12 +223,25 @@ PERCACHE_API int percache_set_flags(percache_t* h, uint32_t flags);
  * Returns the number of elements written, or a negative code (PERCACHE_E_CAPACITY if capacity is short). */
 PERCACHE_API int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity);
 
+/* Host-only: the attention kernel's work schedule for tiles of given lengths, without a device (the part of
+ * percache_prefill's index assembly that cuts every tile's units into items and deals them to the persistent
+ * CTAs; the kernel itself is the causal GQA attention of the new rows over the assembled context, paper
+ * Appendix B.1).  n_blocks [n_tiles]: context blocks (128 slots) each tile sees; units_per_tile: KV heads x
+ * query-head pairs; n_ctas: CTAs available (one per SM); max_partial_slots: parts that may write partial results.
+ * items_out: caller-allocated [items_capacity][6] int32 rows (tile, unit, blk_begin, blk_end, partial_slot or -1,
+ * cta), in execution order.  counts_out [4]: items, CTAs used, split units, estimated makespan in quarter blocks.
+ * Returns PERCACHE_OK, PERCACHE_E_INVAL, or PERCACHE_E_CAPACITY when items_capacity is short. */
+PERCACHE_API int percache_debug_attn_plan(const int32_t* n_blocks, int32_t n_tiles, int32_t units_per_tile, int32_t n_ctas,
+                             int32_t max_partial_slots, int32_t* items_out, int64_t items_capacity,
+                             int64_t* counts_out);
+
 /* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
  * [n_total][n_kv_heads][head_dim], copied to host buffers. */
 PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
 
 /* C[M][N] (fp32, host) = A[M][K] * B[N][K]^T with fp16 inputs (host), through the tcgen05 GEMM
- * (use_reference = 0) or the plain kernel (1).  Test hook for the GEMM core. */
+ * (use_reference = 0), the plain kernel (1), or the tcgen05 GEMM on CTA pairs with 256 x 256 tiles (2; needs
+ * N % 256 == 0).  Test hook for the GEMM core. */
 PERCACHE_API int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
                         float* c, int32_t use_reference);
 

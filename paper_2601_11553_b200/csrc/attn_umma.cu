@@ -3,6 +3,8 @@
 // Work unit = (tile of up to 128 consecutive new rows of one prompt, one KV head).  The two query heads
 // that share the KV head are two 128-row M tiles of the unit: they have the same rows, positions and
 // mask and read the same K/V blocks, so every K/V byte fetched into shared memory is used twice.
+// The host cuts the units' context ranges into items and deals them to the CTAs so that every CTA gets
+// the same number of context blocks; CTA c runs items [cta_first[c], cta_first[c + 1]) in order.
 //
 // One persistent CTA per SM, 320 threads:
 //   warps 0-3  softmax group of query head 2g      (thread = row; TMEM lanes by warp quarter)
@@ -33,8 +35,8 @@ constexpr uint32_t TMEM_S0 = 0, TMEM_O0 = 256;
 constexpr float RESCALE_THRESHOLD = 8.0f;
 
 struct AttnArgs {
-  const AttnTile* tiles;
-  int32_t n_tiles;
+  const AttnItem* items;
+  const int32_t* cta_first;
   const int32_t* row_pos;
   __half* out;
   float* partial_o;
@@ -47,6 +49,13 @@ struct AttnArgs {
 __device__ __forceinline__ float fast_exp2(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// max(a, b, c) in one instruction (three-input form of max.f32)
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
   return y;
 }
 
@@ -91,20 +100,19 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   const uint32_t tmem_base = tmem_base_slot;
   pdl_wait();                 // Q and the assembled context come from earlier kernels
 
-  const int n_units = args.n_tiles * args.n_kv_heads;
   const int group = args.n_q_heads / args.n_kv_heads;      // query heads per KV head (even)
-  // A unit covers query heads (g * group + 2 * pair, +1); units enumerate (tile, g, pair).
+  // An item's `unit` = g * pairs + pair covers query heads (g * group + 2 * pair, +1) and KV head g.
   const int pairs = group / 2;
-  const int n_work = n_units * pairs;
+  const int w_begin = args.cta_first[blockIdx.x], w_end = args.cta_first[blockIdx.x + 1];
 
   if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       uint32_t unit_it = 0, kvit = 0;
       bool ok = true;
-      for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
-        const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
-        const int gp = w % (args.n_kv_heads * pairs);
+      for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
+        const AttnItem t = args.items[w];
+        const int gp = t.unit;
         const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
         const int nb = t.blk_end - t.blk_begin;
         if (!mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
@@ -152,8 +160,8 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         umma_commit(&s_full[i]);
       };
-      for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
-        const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
+      for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
+        const AttnItem t = args.items[w];
         const int nb = t.blk_end - t.blk_begin;
         const uint32_t kv0 = kvit;
         if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
@@ -205,9 +213,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     const uint32_t t_o = tmem_base + lane_base + TMEM_O0 + i * HEAD_DIM;
     uint32_t unit_it = 0, kvit = 0;
     bool ok = true;
-    for (int w = blockIdx.x; w < n_work && ok; w += gridDim.x, ++unit_it) {
-      const AttnTile t = args.tiles[w / (args.n_kv_heads * pairs)];
-      const int gp = w % (args.n_kv_heads * pairs);
+    for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
+      const AttnItem t = args.items[w];
+      const int gp = t.unit;
       const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
       const int nb = t.blk_end - t.blk_begin;
       const uint32_t kv0 = kvit;
@@ -227,18 +235,21 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         tmem_wait_ld();
         const int limit = pos - (t.blk_begin + j) * BLK;     // columns 0..limit are visible
         // maximum of the raw scores (the scale is positive, so it commutes with the maximum)
-        float m_raw = -INFINITY;
-        if (limit >= BLK - 1) {
+        // four independent chains: the reduction is bound by instruction latency, not by issue
+        float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+        if (limit < BLK - 1) {
 #pragma unroll
-          for (int c = 0; c < 128; c += 2)
-            m_raw = fmaxf(m_raw, fmaxf(__uint_as_float(s[c]), __uint_as_float(s[c + 1])));
-        } else {
-#pragma unroll
-          for (int c = 0; c < 128; ++c) {
+          for (int c = 0; c < 128; ++c)
             if (c > limit) s[c] = 0xff800000u;                // -inf
-            m_raw = fmaxf(m_raw, __uint_as_float(s[c]));
-          }
         }
+#pragma unroll
+        for (int c = 0; c < 128; c += 8) {
+          mx0 = fmax3(mx0, __uint_as_float(s[c]), __uint_as_float(s[c + 1]));
+          mx1 = fmax3(mx1, __uint_as_float(s[c + 2]), __uint_as_float(s[c + 3]));
+          mx2 = fmax3(mx2, __uint_as_float(s[c + 4]), __uint_as_float(s[c + 5]));
+          mx3 = fmax3(mx3, __uint_as_float(s[c + 6]), __uint_as_float(s[c + 7]));
+        }
+        const float m_raw = fmax3(fmaxf(mx0, mx1), mx2, mx3);
         const float m_blk = m_raw * args.scale_log2;
         if (j == 0) {
           // an item that starts past the row's position sees nothing: keep a finite reference
@@ -292,7 +303,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
       tc_fence_after_sync();
-      if (t.partial_base < 0) {
+      if (t.partial_slot < 0) {
         const float inv_l = 1.0f / l;
         __half* dst = args.out + (static_cast<size_t>(row) * args.n_q_heads + head) * HEAD_DIM;
 #pragma unroll 1
@@ -315,7 +326,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
         }
       } else {
-        const size_t slot = static_cast<size_t>(t.partial_base + gp) * 2 + i;
+        const size_t slot = static_cast<size_t>(t.partial_slot) * 2 + i;
         float* po = args.partial_o + (slot * BLK + r_in_tile) * HEAD_DIM;
 #pragma unroll 1
         for (int c = 0; c < 4; ++c) {
@@ -363,9 +374,9 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
   return 0;
 }
 
-// Merge of split tiles: out[row][head] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with M = max_s m_s.
-// One warp per (row, head): lanes first take one part each for the (reference, sum) pairs, then every lane
-// owns four output columns and walks the parts with independent 16-byte loads.
+// Merge of the parts of a split unit: out[row][head] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with
+// M = max_s m_s.  One warp per (row, head): lanes first take one part each for the (reference, sum) pairs,
+// then every lane owns four output columns and walks the parts with independent 16-byte loads.
 namespace {
 constexpr int MERGE_WARPS = 8;
 __global__ void __launch_bounds__(MERGE_WARPS * 32)
@@ -375,24 +386,22 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __rest
   pdl_wait();
   const AttnMerge mg = merges[blockIdx.x];
   const int group = n_q_heads / n_kv_heads, pairs = group / 2;
-  const int units = n_kv_heads * pairs;
-  const int gp = blockIdx.y >> 1, i = blockIdx.y & 1;
-  const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
+  const int i = blockIdx.y;
+  const int head = (mg.unit / pairs) * group + 2 * (mg.unit % pairs) + i;
   const int lane = threadIdx.x & 31;
   const int r = blockIdx.z * MERGE_WARPS + (threadIdx.x >> 5);
   if (r >= mg.n_rows) return;
-  const size_t slot0 = static_cast<size_t>(mg.partial_base + gp) * 2 + i;
-  const size_t slot_stride = static_cast<size_t>(units) * 2;
+  const size_t slot0 = static_cast<size_t>(mg.partial_slot0) * 2 + i;     // part s is two slots further each
   float M = -INFINITY;
   for (int s = lane; s < mg.n_parts; s += 32)
-    M = fmaxf(M, partial_ml[((slot0 + s * slot_stride) * BLK + r) * 2]);
+    M = fmaxf(M, partial_ml[((slot0 + 2 * s) * BLK + r) * 2]);
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
   float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
   float l = 0.f;
 #pragma unroll 4
   for (int s = 0; s < mg.n_parts; ++s) {
-    const size_t slot = slot0 + s * slot_stride;
+    const size_t slot = slot0 + 2 * s;
     const float2 ml = *reinterpret_cast<const float2*>(partial_ml + (slot * BLK + r) * 2);
     const float w = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;
     const float4 o = *reinterpret_cast<const float4*>(partial_o + (slot * BLK + r) * HEAD_DIM + lane * 4);
@@ -410,29 +419,27 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __rest
 void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
                             __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s) {
   if (n_merges <= 0) return;
-  dim3 grid(n_merges, n_q_heads, BLK / MERGE_WARPS);
+  dim3 grid(n_merges, 2, BLK / MERGE_WARPS);
   launch_pdl(attention_merge_kernel, grid, dim3(MERGE_WARPS * 32), 0, s, merges, partial_o, partial_ml, out, n_q_heads,
              n_kv_heads);
 }
 
-int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
-                          __half* out, float* partial_o, float* partial_ml, int n_q_heads, int n_kv_heads,
-                          int* err_word, int n_sms, cudaStream_t s) {
-  if (n_tiles <= 0) return 0;
+int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
+                          const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
+                          int n_kv_heads, int* err_word, cudaStream_t s) {
+  if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0) return -1;
   if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
       cudaSuccess)
     return -1;
   AttnArgs a{};
-  a.tiles = tiles; a.n_tiles = n_tiles; a.row_pos = row_pos; a.out = out;
+  a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out;
   a.partial_o = partial_o; a.partial_ml = partial_ml;
   a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
   a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
   a.err_word = err_word;
-  const int n_work = n_tiles * n_kv_heads * (group / 2);
-  const int grid = n_work < n_sms ? n_work : n_sms;
-  return launch_pdl(umma_attention_kernel, dim3(grid), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v,
+  return launch_pdl(umma_attention_kernel, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v,
                     a) == cudaSuccess ? 0 : -1;
 }
 

@@ -9,6 +9,12 @@
 //   warps 2-9 epilogue: each reads its 32-lane quarter of the accumulator with tcgen05.ld (two warps per
 //             quarter, alternating 32-column chunks), applies the epilogue and stores; two accumulator
 //             stages let the next tile's MMAs overlap it.
+// Pair mode (PAIR = true): the grid is made of clusters of two CTAs on a 256 x BN tile.  Each CTA loads its own
+// 128 rows of A and only half of the tile's B rows; the rank-0 CTA issues one cta_group::2 UMMA per K step that
+// reads A and B from both shared memories and fills 128 TMEM lanes in each CTA, so the bytes a CTA pulls from
+// L2 per MMA clock fall by a third (BN = 256) and the main loop stops being bound by that feed.  Barriers:
+// `full` lives in rank 0 and counts both CTAs' TMA bytes; `empty` and `tmem_full` exist in both CTAs and are
+// signalled together by a multicast commit; `tmem_empty` lives in rank 0 and collects both CTAs' epilogue warps.
 // Every wait is bounded (ptx.cuh); on a timeout the roles fall through to the common teardown,
 // the producer gives its outstanding copies time to land, TMEM is freed and the host sees the error word.
 #include "epilogue.cuh"
@@ -32,10 +38,11 @@ constexpr int STG_PITCH = 80;
 constexpr int STG_BUF_BYTES = 32 * STG_PITCH;
 constexpr int EPI_STAGING_BYTES = EPI_WARPS * 2 * STG_BUF_BYTES;   // 40 KB
 
-template <int BN> struct GemmCfg {
-  static constexpr int B_STAGE_BYTES = BN * BK * 2;
+template <int BN, bool PAIR> struct GemmCfg {
+  static constexpr int B_ROWS = PAIR ? BN / 2 : BN;                // rows of B this CTA loads per stage
+  static constexpr int B_STAGE_BYTES = B_ROWS * BK * 2;
   static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
-  static constexpr int STAGES = (BN >= 256) ? 3 : 5;
+  static constexpr int STAGES = (B_ROWS >= 256) ? 3 : (B_ROWS >= 128 ? 5 : 6);
   static constexpr int RING_BYTES = STAGES * STAGE_BYTES;
   static constexpr int SMEM_BYTES = RING_BYTES + EPI_STAGING_BYTES + 1024;   // + slack to align the ring to 1024 B
   static constexpr int TMEM_COLS = 2 * BN;                         // two accumulator stages
@@ -51,10 +58,14 @@ struct GemmArgs {
   int* err_word;
 };
 
-template <int BN, int KIND>
+template <int BN, int KIND, bool PAIR>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, GemmArgs args) {
-  using Cfg = GemmCfg<BN>;
+  using Cfg = GemmCfg<BN, PAIR>;
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;            // rows of a work item (both CTAs of a pair)
+  const uint32_t rank = PAIR ? cluster_ctarank() : 0u;  // 0 issues the MMAs
+  const int worker = PAIR ? static_cast<int>(blockIdx.x >> 1) : static_cast<int>(blockIdx.x);
+  const int n_workers = PAIR ? static_cast<int>(gridDim.x >> 1) : static_cast<int>(gridDim.x);
   constexpr int STAGES = Cfg::STAGES;
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t full_bar[STAGES];
@@ -67,7 +78,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   const int lane = threadIdx.x & 31;
   uint8_t* ring = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
 
-  const int n_m_tiles = (args.M + BM - 1) / BM;
+  const int n_m_tiles = (args.M + TILE_M - 1) / TILE_M;
   const int n_n_tiles = args.N / BN;
   const int k_splits = (KIND == EPI_RESIDUAL) ? args.k_splits : 1;
   const int n_tiles = n_m_tiles * n_n_tiles * k_splits;      // work items: (tile, K part)
@@ -78,12 +89,17 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
-    for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], 8); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], PAIR ? 16 : 8); }
     fence_mbar_init();
   }
   if (warp == 1) {
-    tmem_alloc<Cfg::TMEM_COLS>(&tmem_base_slot);
-    tmem_relinquish();
+    if constexpr (PAIR) {
+      tmem_alloc_pair<Cfg::TMEM_COLS>(&tmem_base_slot);
+      tmem_relinquish_pair();
+    } else {
+      tmem_alloc<Cfg::TMEM_COLS>(&tmem_base_slot);
+      tmem_relinquish();
+    }
   }
   if (warp == 0 && lane == 0) {
     prefetch_tmap(&tmA);
@@ -92,6 +108,10 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   pdl_launch_dependents();
   tc_fence_before_sync();
   __syncthreads();
+  if constexpr (PAIR) {       // the other CTA's barriers must exist before anything is signalled there
+    cluster_arrive();
+    cluster_wait();
+  }
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
   pdl_wait();                 // operands and the residual stream come from earlier kernels
@@ -102,15 +122,23 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+      for (int tile = worker; tile < n_tiles && ok; tile += n_workers) {
         const int m_idx = (tile / k_splits) / n_n_tiles, n_idx = (tile / k_splits) % n_n_tiles;
         for (int kb = kb_begin(tile); kb < kb_end(tile); ++kb) {
           if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
           uint8_t* a_dst = ring + stage * Cfg::STAGE_BYTES;
           uint8_t* b_dst = a_dst + A_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[stage], Cfg::STAGE_BYTES);
-          tma_load_2d(a_dst, &tmA, &full_bar[stage], kb * BK, m_idx * BM);
-          tma_load_2d(b_dst, &tmB, &full_bar[stage], kb * BK, n_idx * BN);
+          if constexpr (PAIR) {
+            // rank 0's barrier counts the bytes of both CTAs; each CTA loads its rows of A and its half of B
+            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * Cfg::STAGE_BYTES);
+            const uint32_t bar0 = mapa_shared(smem_u32(&full_bar[stage]), 0);
+            tma_load_2d_pair(a_dst, &tmA, bar0, kb * BK, m_idx * TILE_M + static_cast<int>(rank) * BM);
+            tma_load_2d_pair(b_dst, &tmB, bar0, kb * BK, n_idx * BN + static_cast<int>(rank) * Cfg::B_ROWS);
+          } else {
+            mbar_arrive_expect_tx(&full_bar[stage], Cfg::STAGE_BYTES);
+            tma_load_2d(a_dst, &tmA, &full_bar[stage], kb * BK, m_idx * BM);
+            tma_load_2d(b_dst, &tmB, &full_bar[stage], kb * BK, n_idx * BN);
+          }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
@@ -122,13 +150,13 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = make_idesc_f16(BM, BN, /*fp16*/ 0, 0, 0);
+    if (lane == 0 && rank == 0) {
+      constexpr uint32_t idesc = make_idesc_f16(TILE_M, BN, /*fp16*/ 0, 0, 0);
       int stage = 0;
       uint32_t phase = 0;
       int it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++it) {
+      for (int tile = worker; tile < n_tiles && ok; tile += n_workers, ++it) {
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
         if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
@@ -145,13 +173,20 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
 #pragma unroll
           for (int k = 0; k < BK / UMMA_K; ++k) {
             // 16 elements along K = 32 bytes = 2 units of the descriptor's 16-byte address field
-            umma_ss(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(2 * k), idesc,
-                    (kb > kb0 || k != 0) ? 1u : 0u);
+            if constexpr (PAIR)
+              umma_ss_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(2 * k), idesc,
+                           (kb > kb0 || k != 0) ? 1u : 0u);
+            else
+              umma_ss(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(2 * k), idesc,
+                      (kb > kb0 || k != 0) ? 1u : 0u);
           }
-          umma_commit(&empty_bar[stage]);      // stage reusable once these MMAs have read it
+          // stage reusable (in both CTAs of a pair) once these MMAs have read it
+          if constexpr (PAIR) umma_commit_pair(&empty_bar[stage]); else umma_commit(&empty_bar[stage]);
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
-        if (ok) umma_commit(&tmem_full_bar[acc]);
+        if (ok) {
+          if constexpr (PAIR) umma_commit_pair(&tmem_full_bar[acc]); else umma_commit(&tmem_full_bar[acc]);
+        }
       }
     }
   } else {
@@ -164,13 +199,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
     int it = 0;
     float4 nv0[4], nv1[4];       // EPI_RESIDUAL: residual values loaded ahead of the pass that consumes them
     // address of the four columns this lane handles in iteration `it4` of the pass starting at tile column c
+    const uint32_t tmem_empty_remote = PAIR ? mapa_shared(smem_u32(&tmem_empty_bar[0]), 0) : 0u;
     auto res_ptr = [&](int m_idx, int n_idx, int c, int it4) {
       const int row = min(m_idx * BM + quarter * 32 + it4 * 8 + (lane >> 2), args.M - 1);
       return reinterpret_cast<float4*>(args.res.resid + static_cast<size_t>(row) * args.res.ld + n_idx * BN + c +
                                        (lane & 3) * 4);
     };
-    for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++it) {
-      const int m_idx = (tile / k_splits) / n_n_tiles, n_idx = (tile / k_splits) % n_n_tiles;
+    for (int tile = worker; tile < n_tiles; tile += n_workers, ++it) {
+      // m_idx counts 128-row blocks: this CTA's half of a pair's 256-row tile
+      const int m_idx = ((tile / k_splits) / n_n_tiles) * (TILE_M / BM) + static_cast<int>(rank);
+      const int n_idx = (tile / k_splits) % n_n_tiles;
       const int acc = it & 1;
       const uint32_t acc_phase = (it >> 1) & 1u;
       if (KIND == EPI_RESIDUAL && k_splits == 1) {
@@ -298,16 +336,24 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tmem_empty_bar[acc]);
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_cluster(tmem_empty_remote + static_cast<uint32_t>(acc) * 8u);
+        else mbar_arrive(&tmem_empty_bar[acc]);
+      }
     }
   }
 
   // ------------------------------------------------------------------ teardown (every thread gets here)
   tc_fence_before_sync();
   __syncthreads();
+  if constexpr (PAIR) {       // neither CTA may leave while the other can still read its memory or signal it
+    cluster_arrive();
+    cluster_wait();
+  }
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc<Cfg::TMEM_COLS>(tmem_base);
+    if constexpr (PAIR) tmem_dealloc_pair<Cfg::TMEM_COLS>(tmem_base);
+    else tmem_dealloc<Cfg::TMEM_COLS>(tmem_base);
   }
 }
 
@@ -316,17 +362,47 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 
-template <int BN, int KIND>
+template <int BN, int KIND, bool PAIR>
 int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, int n_sms, cudaStream_t s) {
-  using Cfg = GemmCfg<BN>;
-  if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  using Cfg = GemmCfg<BN, PAIR>;
+  if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                            Cfg::SMEM_BYTES) != cudaSuccess)
     return -1;
-  const int n_tiles = ((args.M + BM - 1) / BM) * (args.N / BN) * (args.k_splits > 0 ? args.k_splits : 1);
+  constexpr int TILE_M = PAIR ? 2 * BM : BM;
+  const int n_tiles = ((args.M + TILE_M - 1) / TILE_M) * (args.N / BN) * (args.k_splits > 0 ? args.k_splits : 1);
   if (n_tiles <= 0) return 0;
-  const int grid = n_tiles < n_sms ? n_tiles : n_sms;
-  return launch_pdl(umma_gemm_kernel<BN, KIND>, dim3(grid), dim3(GEMM_THREADS), Cfg::SMEM_BYTES, s, A.map, B.map,
-                    args) == cudaSuccess ? 0 : -1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(GEMM_THREADS);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int workers = n_sms;
+  if (PAIR) {
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = 2;
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    // SMs pair up inside a GPC only, so fewer than n_sms / 2 clusters may be resident at once; a persistent
+    // grid larger than that would run its last clusters after all the others
+    static int max_clusters = 0;                // per kernel instantiation (one device model per process)
+    if (max_clusters == 0) {
+      cfg.gridDim = dim3((n_sms / 2) * 2);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, umma_gemm_kernel<BN, KIND, PAIR>, &cfg) != cudaSuccess || n <= 0) {
+        cudaGetLastError();
+        return -1;
+      }
+      max_clusters = n;
+    }
+    workers = max_clusters < n_sms / 2 ? max_clusters : n_sms / 2;
+  }
+  cfg.gridDim = dim3((n_tiles < workers ? n_tiles : workers) * (PAIR ? 2 : 1));
+  return cudaLaunchKernelEx(&cfg, umma_gemm_kernel<BN, KIND, PAIR>, A.map, B.map, args) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace
@@ -368,64 +444,77 @@ int umma_gemm_block_n(GemmEpilogueKind kind) {
   return 128;
 }
 
-// Tile width (and, for the residual GEMMs, the number of K parts) for a problem.  The main loop is fed at
-// roughly 64 bytes per clock per SM, so a 128 x 128 x 64 step (32 KB) costs about 512 clocks and a
-// 128 x 256 x 64 step (48 KB) about 768; a work item also pays about three steps of ramp-up and tail.
-// The cost of a choice is (rounds of items over the SMs) x (steps per item + 3) x (clocks per step).
-void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, int* block_n, int* k_splits) {
-  const int m_tiles = (M + BM - 1) / BM;
+// Tile shape (and, for the residual GEMMs, the number of K parts) for a problem.  The main loop of a single
+// CTA is fed at roughly 64 bytes per clock from L2, so a 128 x 128 x 64 step (32 KB) costs about 512 clocks and
+// a 128 x 256 x 64 step (48 KB) about 768; a CTA pair on a 256 x 256 tile loads 32 KB per CTA and step and its
+// step costs about 600 clocks.  A work item also pays about three steps of ramp-up and tail.  The cost of a
+// choice is (rounds of items over the workers) x (steps per item + 3) x (clocks per step).
+// Measured on B200 (M = 33 024, d = 1024): pairs raise the two residual GEMMs from 990 to 1183 TFLOP/s (K = 2048)
+// and from 1059 to 1280 (K = 3072); the QKV and gate/up GEMMs (K = 1024, rotation / SwiGLU epilogues) are
+// bound by their epilogues at 128 x 256 per CTA either way and lose a few percent to the pair's
+// synchronisation, so callers allow pairs for the residual epilogue only.
+void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
+                          int* k_splits, int* pair) {
   const int n_kb = K / BK;
   int64_t best = INT64_MAX;
   *block_n = 128;
   *k_splits = 1;
-  for (int bn = 128; bn <= 256; bn += 128) {
-    if (N % bn != 0) continue;
-    const int64_t tiles = static_cast<int64_t>(m_tiles) * (N / bn);
+  *pair = 0;
+  for (int shape = 0; shape < 3; ++shape) {           // 128 x 128, 128 x 256, pair 256 x 256
+    const int bn = shape == 0 ? 128 : 256;
+    const bool pr = shape == 2;
+    if (N % bn != 0 || (pr && (!may_pair || n_sms < 2))) continue;
+    const int tile_m = pr ? 2 * BM : BM;
+    const int workers = pr ? n_sms / 2 : n_sms;
+    const int64_t clocks = shape == 0 ? 512 : (shape == 1 ? 768 : 600);
+    const int64_t tiles = static_cast<int64_t>((M + tile_m - 1) / tile_m) * (N / bn);
     for (int sp = 1; sp <= (may_split_k ? 8 : 1); ++sp) {
       if (sp > 1 && n_kb / sp < 4) break;
-      const int64_t rounds = (tiles * sp + n_sms - 1) / n_sms;
-      const int64_t cost = rounds * ((n_kb + sp - 1) / sp + 3) * (bn == 256 ? 768 : 512);
-      // prefer wider tiles and fewer parts on ties; a split must win by 10 %
+      const int64_t rounds = (tiles * sp + workers - 1) / workers;
+      const int64_t cost = rounds * ((n_kb + sp - 1) / sp + 3) * clocks;
+      // prefer later shapes and fewer parts on ties; a split must win by 10 %
       const bool better = sp == 1 ? cost <= best : cost * 10 < best * 9;
-      if (better) { best = cost; *block_n = bn; *k_splits = sp; }
+      if (better) { best = cost; *block_n = bn; *k_splits = sp; *pair = pr ? 1 : 0; }
     }
   }
 }
 int umma_gemm_pick_block_n(int M, int N, int n_sms) {
-  int bn, sp;
-  umma_gemm_pick_shape(M, N, 64 * 16, n_sms, false, &bn, &sp);
+  int bn, sp, pr;
+  umma_gemm_pick_shape(M, N, 64 * 16, n_sms, false, false, &bn, &sp, &pr);
   return bn;
 }
 
-template <int BN>
+template <int BN, bool PAIR>
 static int launch_bn(const GemmOperand& A, const GemmOperand& B, GemmArgs& args, GemmEpilogueKind kind,
                      const void* epilogue, int n_sms, cudaStream_t s) {
   switch (kind) {
     case EPI_STORE_F32:
-      return launch_one<BN, EPI_STORE_F32>(A, B, args, n_sms, s);
+      return launch_one<BN, EPI_STORE_F32, PAIR>(A, B, args, n_sms, s);
     case EPI_QKV:
       args.qkv = *static_cast<const QkvEpilogue*>(epilogue);
-      return launch_one<BN, EPI_QKV>(A, B, args, n_sms, s);
+      return launch_one<BN, EPI_QKV, PAIR>(A, B, args, n_sms, s);
     case EPI_RESIDUAL:
       args.res = *static_cast<const ResidualEpilogue*>(epilogue);
-      return launch_one<BN, EPI_RESIDUAL>(A, B, args, n_sms, s);
+      return launch_one<BN, EPI_RESIDUAL, PAIR>(A, B, args, n_sms, s);
     case EPI_SWIGLU:
       args.swi = *static_cast<const SwigluEpilogue*>(epilogue);
-      return launch_one<BN, EPI_SWIGLU>(A, B, args, n_sms, s);
+      return launch_one<BN, EPI_SWIGLU, PAIR>(A, B, args, n_sms, s);
   }
   return -1;
 }
 
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
-                     cudaStream_t s, int k_splits) {
+                     cudaStream_t s, int k_splits, int pair) {
   if (M <= 0) return 0;
   if (K % BK != 0 || N % block_n != 0 || (block_n != 128 && block_n != 256)) return -1;
   if (k_splits < 1 || (k_splits > 1 && kind != EPI_RESIDUAL) || k_splits > K / BK) return -1;
+  if (pair && (block_n != 256 || n_sms < 2)) return -1;
   GemmArgs args{};
   args.M = M; args.N = N; args.K = K; args.c = c_f32; args.err_word = err_word; args.k_splits = k_splits;
-  return block_n == 256 ? launch_bn<256>(A, B, args, kind, epilogue, n_sms, s)
-                        : launch_bn<128>(A, B, args, kind, epilogue, n_sms, s);
+  if (pair) return launch_bn<256, true>(A, B, args, kind, epilogue, n_sms, s);
+  return block_n == 256 ? launch_bn<256, false>(A, B, args, kind, epilogue, n_sms, s)
+                        : launch_bn<128, false>(A, B, args, kind, epilogue, n_sms, s);
 }
 
 }  // namespace pc

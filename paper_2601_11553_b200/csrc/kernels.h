@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <vector>
+
 namespace pc {
 
 constexpr int PAGE_TOKENS = 16;
@@ -28,26 +30,36 @@ struct RowIndex {
   const int32_t* pool_tok;  // page * 16 + offset where the row's unrotated K/V is kept, or -1
 };
 
-// Attention work item: up to 128 consecutive new rows of one prompt against the context blocks
-// [blk_begin, blk_end) (128 slots each).  A tile whose context is long and whose batch has few tiles is
-// cut into several items along the context; each then writes an unnormalised partial result to slot
-// `partial_base + (kv head, head pair)` and a second kernel merges the parts.
-struct AttnTile {
+// Attention work item: up to 128 consecutive new rows of one prompt (a tile), one unit (KV head g and
+// pair of its query heads: unit = g * pairs + pair), against the context blocks [blk_begin, blk_end)
+// (128 slots each).  The host deals items to the persistent CTAs so that each gets the same number of
+// blocks; a unit whose blocks end up in several items is "split": each part writes an unnormalised
+// partial result to its own slot and a second kernel merges the parts.
+struct AttnItem {
   int32_t row0;          // first new row (global row index)
   int32_t n_rows;        // 1..128
   int32_t ctx0;          // global context slot of the prompt's slot 0
   int32_t blk_begin;     // first context block of this item
   int32_t blk_end;       // one past its last block
-  int32_t partial_base;  // -1: the item covers the tile's whole context and writes the final rows
-  int32_t pad0, pad1;
+  int32_t partial_slot;  // -1: the item covers the unit's whole context and writes the final rows
+  int32_t unit;
+  int32_t pad0;
 };
 
-// Merge of the parts of one split tile.
+// Merge of the parts of one split unit: part s is in slot partial_slot0 + s.
 struct AttnMerge {
   int32_t row0, n_rows;
-  int32_t partial_base;  // slot of part 0; part s is at partial_base + s * (kv heads * head pairs)
-  int32_t n_parts;
+  int32_t partial_slot0, n_parts;
+  int32_t unit;
+  int32_t pad0, pad1, pad2;
 };
+
+// A tile before scheduling: its rows and the number of 128-slot context blocks its last row can see.
+struct AttnBaseTile { int32_t row0, n_rows, ctx0, n_blocks; };
+// Deals (tile, unit, block range) items to at most n_sms CTAs (attn_plan.cu).  cta_first gets one entry per
+// CTA used plus one; returns the plan's estimated makespan in quarter blocks.
+int64_t plan_attention(const std::vector<AttnBaseTile>& tiles, int units_per_tile, int n_sms, int max_partial_slots,
+                       std::vector<AttnItem>* items, std::vector<int32_t>* cta_first, std::vector<AttnMerge>* merges);
 
 struct ModelDims {
   int32_t n_layers, d_model, n_q_heads, n_kv_heads, d_ffn;
@@ -102,13 +114,16 @@ struct GemmOperand {           // a tensor map made once for a fixed buffer
 };
 // rows x cols fp16 row-major matrix; box = box_rows x 64 columns, 128-byte swizzle
 int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t cols, int box_rows);
+// pair = 1 (block_n 256 only): clusters of two CTAs on 256 x 256 tiles; B's map then has box_rows = 128.
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
-                     cudaStream_t s, int k_splits = 1);
+                     cudaStream_t s, int k_splits = 1, int pair = 0);
 int umma_gemm_block_n(GemmEpilogueKind kind);    // narrowest N tile (a B operand map needs box_rows = the tile used)
 int umma_gemm_pick_block_n(int M, int N, int n_sms);   // 128 or 256 for this problem
-// tile width and number of K parts (parts > 1 only if may_split_k: the residual epilogue then adds atomically)
-void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, int* block_n, int* k_splits);
+// tile width, number of K parts (parts > 1 only if may_split_k: the residual epilogue then adds atomically) and
+// whether CTA pairs are used (only if may_pair)
+void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
+                          int* k_splits, int* pair);
 
 // rank-N fp16 tensor map with 128-byte swizzle; dims/strides innermost first (strides in bytes, from dim 1)
 int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
@@ -118,10 +133,11 @@ int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t*
 struct AttnMaps { CUtensorMap q, k, v; };
 int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, const __half* kctx_layer,
                    const __half* vctx_layer, int64_t ctx_cap, int kv_dim);
-// partial_o: fp32 [slots][2 heads][128 rows][128]; partial_ml: fp32 [slots][2][128][2] (reference max, sum)
-int launch_umma_attention(const AttnMaps& maps, const AttnTile* tiles, int n_tiles, const int32_t* row_pos,
-                          __half* out, float* partial_o, float* partial_ml, int n_q_heads, int n_kv_heads,
-                          int* err_word, int n_sms, cudaStream_t s);
+// partial_o: fp32 [slots][2 heads][128 rows][128]; partial_ml: fp32 [slots][2][128][2] (reference max, sum).
+// CTA c (of n_ctas) runs items [cta_first[c], cta_first[c + 1]).
+int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
+                          const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
+                          int n_kv_heads, int* err_word, cudaStream_t s);
 void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
                             __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
 

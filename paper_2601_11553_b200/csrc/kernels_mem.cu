@@ -70,8 +70,46 @@ void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStr
 // ------------------------------------------------------------------------------------------------
 // RMSNorm: out[r][:] = fp16( x[r][:] * rsqrt(mean(x[r]^2) + eps) * gain[:] ), one warp per row.
 // ------------------------------------------------------------------------------------------------
+// The row stays in registers between the two passes (VPL float4 per lane, d <= 128 * VPL); all loads of a row
+// are issued before the first is used.
+template <int VPL>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                       __half* __restrict__ out, int M, int d, float eps) {
+  const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  pdl_launch_dependents();
+  pdl_wait();
+  if (row >= M) return;
+  const int lane = threadIdx.x & 31;
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+  const int nv = d >> 2;
+  float4 v[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int i = lane + 32 * k;
+    v[k] = i < nv ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  float ss = 0.f;
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
+  const float inv = rsqrtf(ss / static_cast<float>(d) + eps);
+  const float4* g4 = reinterpret_cast<const float4*>(gain);
+  uint2* o2 = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int i = lane + 32 * k;
+    if (i < nv) {
+      const float4 g = __ldg(g4 + i);
+      __half2 a = __floats2half2_rn(v[k].x * inv * g.x, v[k].y * inv * g.y);
+      __half2 b = __floats2half2_rn(v[k].z * inv * g.z, v[k].w * inv * g.w);
+      o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+    }
+  }
+}
+// Rows of any length: two passes over global memory.
+__global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+                                                           __half* __restrict__ out, int M, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   pdl_launch_dependents();
   pdl_wait();
@@ -99,7 +137,10 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 }
 void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s) {
   if (M <= 0) return;
-  launch_pdl(rmsnorm_kernel, dim3((M + 7) / 8), dim3(256), 0, s, x, gain, out, M, d, eps);
+  const dim3 grid((M + 7) / 8), block(256);
+  if (d <= 1024) launch_pdl(rmsnorm_kernel<8>, grid, block, 0, s, x, gain, out, M, d, eps);
+  else if (d <= 2048) launch_pdl(rmsnorm_kernel<16>, grid, block, 0, s, x, gain, out, M, d, eps);
+  else launch_pdl(rmsnorm_long_kernel, grid, block, 0, s, x, gain, out, M, d, eps);
 }
 
 // ------------------------------------------------------------------------------------------------

@@ -295,12 +295,14 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   ok = ok && dev_alloc(h, &h->act, static_cast<size_t>(h->m_cap) * F);
   ok = ok && dev_alloc(h, &h->d_err, 1);
   // index block: 4 row arrays + gather items (worst case one per context token) + attention tiles
+  // (an attention item per unit of every tile, plus the parts the scheduler cuts: at most two per CTA)
   const size_t max_tiles = static_cast<size_t>(h->m_cap / 128 + cfg->max_batch_prompts + 2);
-  h->partial_slots = 4 * h->n_sms + D.n_q_heads;
-  h->max_attn_items = max_tiles + static_cast<size_t>(h->partial_slots);
-  h->max_attn_merges = max_tiles;
+  const size_t units_per_tile = static_cast<size_t>(D.n_kv_heads) * (D.n_q_heads / D.n_kv_heads / 2);
+  h->partial_slots = 2 * h->n_sms + 2;
+  h->max_attn_items = max_tiles * units_per_tile + 2 * static_cast<size_t>(h->n_sms);
+  h->max_attn_merges = static_cast<size_t>(h->n_sms) + 1;
   h->index_ints = 4 * static_cast<size_t>(h->m_cap) + 4 * static_cast<size_t>(h->ctx_cap) + 8 * h->max_attn_items +
-                  4 * h->max_attn_merges;
+                  static_cast<size_t>(h->n_sms) + 1 + 8 * h->max_attn_merges;
   ok = ok && dev_alloc(h, &h->partial_o, static_cast<size_t>(h->partial_slots) * 2 * 128 * HEAD_DIM);
   ok = ok && dev_alloc(h, &h->partial_ml, static_cast<size_t>(h->partial_slots) * 2 * 128 * 2);
   ok = ok && dev_alloc(h, &h->d_index, h->index_ints);
@@ -671,10 +673,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   int32_t* row_pool = row_pos + h->m_cap;
   int32_t* row_ctx0 = row_pool + h->m_cap;
   GatherItem* items = reinterpret_cast<GatherItem*>(row_ctx0 + h->m_cap);
-  AttnTile* tiles = reinterpret_cast<AttnTile*>(reinterpret_cast<int32_t*>(items) + 4 * h->ctx_cap);
-  AttnMerge* merges = reinterpret_cast<AttnMerge*>(reinterpret_cast<int32_t*>(tiles) + 8 * h->max_attn_items);
-  std::vector<AttnTile> base_tiles;
-  int n_items = 0, n_tiles = 0, n_merges = 0;
+  AttnItem* attn_items = reinterpret_cast<AttnItem*>(reinterpret_cast<int32_t*>(items) + 4 * h->ctx_cap);
+  int32_t* cta_first = reinterpret_cast<int32_t*>(attn_items) + 8 * h->max_attn_items;
+  AttnMerge* merges = reinterpret_cast<AttnMerge*>(cta_first + h->n_sms + 1);
+  std::vector<AttnBaseTile> base_tiles;
+  int n_items = 0, n_attn_ctas = 0, n_merges = 0;
   plan.slot_chunk.resize(static_cast<size_t>(ctx_total));
   plan.slot_offset.resize(static_cast<size_t>(ctx_total));
   plan.slot_is_new.resize(static_cast<size_t>(ctx_total));
@@ -723,81 +726,42 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       t += len;
     }
     for (int32_t r0 = plan.cu_new[b]; r0 < plan.cu_new[b + 1]; r0 += 128) {
-      AttnTile a{};
+      AttnBaseTile a{};
       a.row0 = r0;
       a.n_rows = std::min(128, plan.cu_new[b + 1] - r0);
       a.ctx0 = ctx0;
-      a.blk_begin = 0;
-      a.blk_end = (row_pos[r0 + a.n_rows - 1] + 1 + 127) / 128;     // context blocks its last row can see
-      a.partial_base = -1;
+      a.n_blocks = (row_pos[r0 + a.n_rows - 1] + 1 + 127) / 128;     // context blocks its last row can see
       base_tiles.push_back(a);
     }
   }
-  // When the tiles of a batch are few or very unequal, most SMs would idle behind the longest one: tiles may
-  // be cut along the context into parts that a second kernel merges.  The choice is made by a small cost
-  // model (in units of one context block of one item): items are dealt longest-first to the persistent
-  // CTAs; a CTA costs its blocks plus a fixed amount per item, and merging costs a fixed amount.
   {
-    const int G = D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2);
-    constexpr int ITEM_COST = 3, MERGE_COST = 4;
-    int64_t total_blocks = 0;
-    for (const AttnTile& a : base_tiles) total_blocks += a.blk_end;
-    auto plan_cost = [&](int chunk_blocks, int64_t* slots_out) {
-      std::vector<int> lens;
-      int64_t slots = 0;
-      for (const AttnTile& a : base_tiles) {
-        int n_s = (a.blk_end + chunk_blocks - 1) / chunk_blocks;
-        if (n_s <= 1) { lens.push_back(a.blk_end); continue; }
-        const int part = (a.blk_end + n_s - 1) / n_s;
-        n_s = (a.blk_end + part - 1) / part;
-        slots += static_cast<int64_t>(n_s) * G;
-        for (int sp = 0; sp < n_s; ++sp) lens.push_back(std::min(a.blk_end, (sp + 1) * part) - sp * part);
-      }
-      std::sort(lens.begin(), lens.end(), std::greater<int>());
-      std::vector<int64_t> load(static_cast<size_t>(h->n_sms), 0);
-      size_t w = 0;
-      for (int len : lens)
-        for (int g = 0; g < G; ++g, ++w) load[w % load.size()] += len + ITEM_COST;
-      *slots_out = slots;
-      return *std::max_element(load.begin(), load.end()) + (slots > 0 ? MERGE_COST : 0);
-    };
-    int chunk = INT32_MAX;
-    if (!base_tiles.empty()) {
-      int64_t slots = 0;
-      int64_t best = plan_cost(INT32_MAX, &slots);
-      for (int per_sm = 1; per_sm <= 3; ++per_sm) {
-        const int c = static_cast<int>(std::max<int64_t>(4, (total_blocks * G + per_sm * h->n_sms - 1) / (per_sm * h->n_sms)));
-        const int64_t cost = plan_cost(c, &slots);
-        if (slots <= h->partial_slots && cost * 10 < best * 9) { best = cost; chunk = c; }   // needs a 10 % gain
-      }
-    }
-    int next_slot = 0;
-    std::vector<AttnTile> work;
-    for (const AttnTile& a : base_tiles) {
-      int n_s = (a.blk_end + chunk - 1) / chunk;
-      if (n_s <= 1) { work.push_back(a); continue; }
-      const int part = (a.blk_end + n_s - 1) / n_s;
-      n_s = (a.blk_end + part - 1) / part;
-      AttnMerge& mg = merges[n_merges++];
-      mg.row0 = a.row0; mg.n_rows = a.n_rows; mg.partial_base = next_slot; mg.n_parts = n_s;
-      for (int sp = 0; sp < n_s; ++sp) {
-        AttnTile w = a;
-        w.blk_begin = sp * part;
-        w.blk_end = std::min(a.blk_end, (sp + 1) * part);
-        w.partial_base = next_slot + sp * G;
-        work.push_back(w);
-      }
-      next_slot += n_s * G;
-    }
-    std::stable_sort(work.begin(), work.end(), [](const AttnTile& x, const AttnTile& y) {
-      return (x.blk_end - x.blk_begin) > (y.blk_end - y.blk_begin);
-    });
-    for (const AttnTile& w : work) tiles[n_tiles++] = w;
+    std::vector<AttnItem> v_items;
+    std::vector<int32_t> v_first;
+    std::vector<AttnMerge> v_merges;
+    plan_attention(base_tiles, D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2), h->n_sms, h->partial_slots, &v_items,
+                   &v_first, &v_merges);
+    if (v_items.size() > h->max_attn_items || v_merges.size() > h->max_attn_merges ||
+        v_first.size() > static_cast<size_t>(h->n_sms) + 1)
+      return fail(PERCACHE_E_CAPACITY);
+    std::copy(v_items.begin(), v_items.end(), attn_items);
+    std::fill(cta_first, cta_first + h->n_sms + 1, static_cast<int32_t>(v_items.size()));
+    std::copy(v_first.begin(), v_first.end(), cta_first);
+    std::copy(v_merges.begin(), v_merges.end(), merges);
+    n_attn_ctas = static_cast<int>(v_first.size()) - 1;
+    n_merges = static_cast<int>(v_merges.size());
   }
   const double plan_us =
       std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
 
   // ---------------------------------------------------------------- device work
+  // The fetch depends on nothing the layers compute (it reads pages of chunks stored by earlier
+  // calls), so a large one runs beside them: one launch per layer on the side stream, and layer l's
+  // attention waits for fetch l alone.  A small fetch stays one launch ahead of layer 0 (the waits
+  // would cost more than they hide), and so does a phase-timed call, whose fetch time must be clean.
+  const bool use_ref = (h->flags & PERCACHE_FLAG_REFERENCE_KERNELS) != 0;
+  const int64_t gather_bytes = hit_tokens * D.kv_dim * 8 * D.n_layers;   // K and V, bf16 in + fp16 out
+  const bool overlap_gather = n_items > 0 && M > 0 && !use_ref && !(h->flags & PERCACHE_FLAG_PHASE_TIMING) &&
+                              gather_bytes >= GATHER_OVERLAP_MIN_BYTES;
   cudaStream_t s = h->stream;
   percache_stats_t& st = h->stats;
   std::memset(st.phase_us, 0, sizeof(st.phase_us));
@@ -812,10 +776,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   const int32_t* d_row_pool = d_row_pos + h->m_cap;
   const int32_t* d_row_ctx0 = d_row_pool + h->m_cap;
   const GatherItem* d_items = reinterpret_cast<const GatherItem*>(d_row_ctx0 + h->m_cap);
-  const AttnTile* d_tiles = reinterpret_cast<const AttnTile*>(reinterpret_cast<const int32_t*>(d_items) + 4 * h->ctx_cap);
-  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(reinterpret_cast<const int32_t*>(d_tiles) + 8 * h->max_attn_items);
+  const AttnItem* d_attn_items = reinterpret_cast<const AttnItem*>(reinterpret_cast<const int32_t*>(d_items) + 4 * h->ctx_cap);
+  const int32_t* d_cta_first = reinterpret_cast<const int32_t*>(d_attn_items) + 8 * h->max_attn_items;
+  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(d_cta_first + h->n_sms + 1);
 
-  const bool use_ref = (h->flags & PERCACHE_FLAG_REFERENCE_KERNELS) != 0;
   if (use_ref && !h->cref) {
     const size_t wide = static_cast<size_t>(std::max(std::max(D.qkv_dim, 2 * D.d_ffn), d));
     if (!dev_alloc(h, &h->cref, static_cast<size_t>(h->m_cap) * wide)) return fail(PERCACHE_E_NOMEM);
@@ -832,14 +796,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
   const int Mi = static_cast<int>(M);
-  // The fetch depends on nothing the layers compute (it reads pages of chunks stored by earlier
-  // calls), so a large one runs beside them: one launch per layer on the side stream, and layer l's
-  // attention waits for fetch l alone.  The HBM-bound copies then fill the time the tensor-bound
-  // GEMMs leave the memory system idle.  A small fetch stays one launch ahead of layer 0 (the waits
-  // would cost more than they hide), and so does a phase-timed call, whose fetch time must be clean.
-  const int64_t gather_bytes = hit_tokens * D.kv_dim * 8 * D.n_layers;   // K and V, bf16 in + fp16 out
-  const bool overlap_gather = n_items > 0 && Mi > 0 && !use_ref && !(h->flags & PERCACHE_FLAG_PHASE_TIMING) &&
-                              gather_bytes >= GATHER_OVERLAP_MIN_BYTES;
+  // CTA pairs pay off where the main loop is the bound: the two residual GEMMs (see umma_gemm_pick_shape)
+  const bool may_pair = !(h->flags & PERCACHE_FLAG_SINGLE_CTA_GEMM);
   if (overlap_gather) {
     ok = ok && cudaEventRecord(h->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(h->side, h->ev_fork, 0) == cudaSuccess;
     for (int l = 0; l < D.n_layers && ok; ++l) {
@@ -875,10 +833,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
     } else {
       {
-        int bn, ks;
-        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, &bn, &ks);
-        ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
-                                    h->d_err, h->n_sms, s, ks) == 0;
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, false, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
       }
     }
     timer.end();
@@ -888,8 +846,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
       launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
     } else {
-      ok = ok && launch_umma_attention(W.attn_maps, d_tiles, n_tiles, d_row_pos, h->attn_out, h->partial_o, h->partial_ml,
-                                       D.n_q_heads, D.n_kv_heads, h->d_err, h->n_sms, s) == 0;
+      ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
+                                       h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s) == 0;
       launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
     }
     timer.end();
@@ -901,10 +859,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
       {
-        int bn, ks;
-        umma_gemm_pick_shape(Mi, d, D.q_dim, h->n_sms, true, &bn, &ks);
-        ok = ok && launch_umma_gemm(h->m_attn, bn == 256 ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s, ks) == 0;
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, d, D.q_dim, h->n_sms, true, may_pair, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_attn, (bn == 256 && !pr) ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
       }
     }
     timer.end();
@@ -920,10 +878,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
     } else {
       {
-        int bn, ks;
-        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, &bn, &ks);
-        ok = ok && launch_umma_gemm(h->m_xn, bn == 256 ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
-                                    h->d_err, h->n_sms, s, ks) == 0;
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, false, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
       }
     }
     timer.end();
@@ -934,10 +892,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
       {
-        int bn, ks;
-        umma_gemm_pick_shape(Mi, d, D.d_ffn, h->n_sms, true, &bn, &ks);
-        ok = ok && launch_umma_gemm(h->m_act, bn == 256 ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s, ks) == 0;
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, d, D.d_ffn, h->n_sms, true, may_pair, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_act, (bn == 256 && !pr) ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
       }
     }
     timer.end();
@@ -991,6 +949,36 @@ int percache_get_stats(percache_t* h, percache_stats_t* out) {
   return PERCACHE_OK;
 }
 
+int percache_debug_attn_plan(const int32_t* n_blocks, int32_t n_tiles, int32_t units_per_tile, int32_t n_ctas,
+                             int32_t max_partial_slots, int32_t* items_out, int64_t items_capacity,
+                             int64_t* counts_out) {
+  if (n_tiles < 0 || units_per_tile <= 0 || n_ctas <= 0 || max_partial_slots < 0 || !counts_out ||
+      (n_tiles > 0 && !n_blocks))
+    return PERCACHE_E_INVAL;
+  std::vector<AttnBaseTile> tiles(static_cast<size_t>(n_tiles));
+  for (int i = 0; i < n_tiles; ++i) {
+    if (n_blocks[i] <= 0) return PERCACHE_E_INVAL;
+    tiles[static_cast<size_t>(i)] = AttnBaseTile{i * 128, 128, 0, n_blocks[i]};   // row0 identifies the tile
+  }
+  std::vector<AttnItem> items;
+  std::vector<int32_t> first;
+  std::vector<AttnMerge> merges;
+  const int64_t makespan = plan_attention(tiles, units_per_tile, n_ctas, max_partial_slots, &items, &first, &merges);
+  counts_out[0] = static_cast<int64_t>(items.size());
+  counts_out[1] = static_cast<int64_t>(first.size()) - 1;
+  counts_out[2] = static_cast<int64_t>(merges.size());
+  counts_out[3] = makespan;
+  if (static_cast<int64_t>(items.size()) > items_capacity || (!items.empty() && !items_out)) return PERCACHE_E_CAPACITY;
+  size_t cta = 0;
+  for (size_t i = 0; i < items.size(); ++i) {
+    while (cta + 1 < first.size() && static_cast<int32_t>(i) >= first[cta + 1]) ++cta;
+    int32_t* o = items_out + 6 * i;
+    o[0] = items[i].row0 / 128; o[1] = items[i].unit; o[2] = items[i].blk_begin; o[3] = items[i].blk_end;
+    o[4] = items[i].partial_slot; o[5] = static_cast<int32_t>(cta);
+  }
+  return PERCACHE_OK;
+}
+
 int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int64_t capacity) {
   if (!h || !out) return PERCACHE_E_INVAL;
   const std::vector<int32_t>* v = nullptr;
@@ -1025,7 +1013,9 @@ int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* 
 int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const void* a_f16, const void* b_f16,
                         float* c, int32_t use_reference) {
   if (M <= 0 || N <= 0 || K <= 0 || !a_f16 || !b_f16 || !c) return PERCACHE_E_INVAL;
-  if (!use_reference && (K % 64 != 0 || N % 128 != 0)) return PERCACHE_E_INVAL;
+  if (use_reference < 0 || use_reference > 2) return PERCACHE_E_INVAL;
+  if (use_reference != 1 && (K % 64 != 0 || N % 128 != 0)) return PERCACHE_E_INVAL;
+  if (use_reference == 2 && N % 256 != 0) return PERCACHE_E_INVAL;
   int n_dev = 0;
   if (cudaGetDeviceCount(&n_dev) != cudaSuccess || device < 0 || device >= n_dev) { cudaGetLastError(); return PERCACHE_E_CUDA; }
   if (cudaSetDevice(device) != cudaSuccess) { cudaGetLastError(); return PERCACHE_E_CUDA; }
@@ -1034,7 +1024,7 @@ int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const v
   float* dC = nullptr;
   int *dErr = nullptr, hErr = 0;
   int rc = PERCACHE_OK;
-  const size_t m_pad = static_cast<size_t>((M + 127) / 128) * 128;
+  const size_t m_pad = static_cast<size_t>((M + 255) / 256) * 256;
   if (cudaMalloc(reinterpret_cast<void**>(&dA), m_pad * K * 2) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&dB), static_cast<size_t>(N) * K * 2) != cudaSuccess ||
       cudaMalloc(reinterpret_cast<void**>(&dC), static_cast<size_t>(M) * N * 4) != cudaSuccess ||
@@ -1047,15 +1037,17 @@ int percache_debug_gemm(int32_t device, int32_t M, int32_t N, int32_t K, const v
     cudaMemset(dErr, 0, sizeof(int));
     cudaMemcpy(dA, a_f16, static_cast<size_t>(M) * K * 2, cudaMemcpyHostToDevice);
     cudaMemcpy(dB, b_f16, static_cast<size_t>(N) * K * 2, cudaMemcpyHostToDevice);
-    if (use_reference) {
+    if (use_reference == 1) {
       launch_ref_gemm(dA, dB, dC, M, N, K, nullptr);
     } else {
       GemmOperand mA, mB;
       int n_sms = 148;
       cudaDeviceGetAttribute(&n_sms, cudaDevAttrMultiProcessorCount, device);
-      const int bn = (N % 256 == 0 && M >= 512) ? 256 : 128;     // both tile widths get exercised by the tests
-      if (make_operand_map(&mA, dA, static_cast<int64_t>(m_pad), K, 128) != 0 || make_operand_map(&mB, dB, N, K, bn) != 0 ||
-          launch_umma_gemm(mA, mB, M, N, K, bn, EPI_STORE_F32, nullptr, dC, dErr, n_sms, nullptr) != 0)
+      const int pair = use_reference == 2 ? 1 : 0;
+      const int bn = pair || (N % 256 == 0 && M >= 512) ? 256 : 128;     // both tile widths get exercised by the tests
+      if (make_operand_map(&mA, dA, static_cast<int64_t>(m_pad), K, 128) != 0 ||
+          make_operand_map(&mB, dB, N, K, pair ? 128 : bn) != 0 ||
+          launch_umma_gemm(mA, mB, M, N, K, bn, EPI_STORE_F32, nullptr, dC, dErr, n_sms, nullptr, 1, pair) != 0)
         rc = PERCACHE_E_CUDA;
     }
     if (rc == PERCACHE_OK && (cudaDeviceSynchronize() != cudaSuccess || cudaGetLastError() != cudaSuccess)) rc = PERCACHE_E_CUDA;

@@ -25,11 +25,12 @@ OK = 0
 E_INVAL, E_NOMEM, E_NOSPACE, E_EXISTS, E_LEN_MISMATCH = -1, -2, -3, -4, -5
 E_MISS_NO_INPUT, E_CAPACITY, E_DEVICE_TIMEOUT, E_CUDA, E_NOTFOUND = -6, -7, -8, -9, -10
 FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION, FLAG_EVICT_LFU = 1, 2, 4, 8
+FLAG_SINGLE_CTA_GEMM = 16
 PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
-           "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx",
+           "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx", "percache_debug_attn_plan",
            "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_qa_top1", "percache_strerror")
 
 
@@ -98,6 +99,7 @@ def load_library() -> C.CDLL:
     lib.percache_debug_read_plan.argtypes = [vp, i32, C.POINTER(i32), i64]
     lib.percache_debug_read_plan.restype = i64
     lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
+    lib.percache_debug_attn_plan.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
     lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
     lib.percache_qa_top1.argtypes = [i32, vp, vp, i32, i32, vp, i32, C.c_float, vp, vp, vp, C.POINTER(C.c_float)]
@@ -326,20 +328,35 @@ class PerCache:
         return k, v
 
 
+def debug_attn_plan(n_blocks: Sequence[int], units_per_tile: int, n_ctas: int = 148, max_partial_slots: int = 298):
+    """percache_debug_attn_plan (host only): returns (items [n][6] = tile, unit, blk_begin, blk_end, partial_slot,
+    cta; CTAs used; split units; estimated makespan in quarter blocks)."""
+    nb = np.ascontiguousarray(np.asarray(n_blocks, dtype=np.int32))
+    cap = int(len(nb)) * units_per_tile + 2 * n_ctas + 8
+    items = np.zeros((cap, 6), dtype=np.int32)
+    counts = np.zeros(4, dtype=np.int64)
+    _check(load_library().percache_debug_attn_plan(_ptr(nb) if len(nb) else None, len(nb), units_per_tile, n_ctas,
+                                                   max_partial_slots, _ptr(items), cap, _ptr(counts)),
+           "percache_debug_attn_plan")
+    return items[:int(counts[0])].copy(), int(counts[1]), int(counts[2]), int(counts[3])
+
+
 def path_key(chunk_ids: Sequence[int]) -> int:
     """Store key of the prefix-tree node reached by the path `chunk_ids` (percache_path_key)."""
     arr = (C.c_uint64 * max(len(chunk_ids), 1))(*[int(c) for c in chunk_ids])
     return int(load_library().percache_path_key(arr, len(chunk_ids)))
 
 
-def debug_gemm(a_f16: np.ndarray, b_f16: np.ndarray, use_reference: bool = False, device: int = 0) -> np.ndarray:
-    """C = A @ B.T through the tcgen05 GEMM core (or the plain kernel): fp16 in, fp32 out, host arrays."""
+def debug_gemm(a_f16: np.ndarray, b_f16: np.ndarray, use_reference: bool = False, device: int = 0,
+               pair: bool = False) -> np.ndarray:
+    """C = A @ B.T through the tcgen05 GEMM core (or the plain kernel, or the CTA-pair variant of the tcgen05
+    GEMM): fp16 in, fp32 out, host arrays."""
     lib = load_library()
     m, k = a_f16.shape
     n = b_f16.shape[0]
     c = np.empty((m, n), dtype=np.float32)
     _check(lib.percache_debug_gemm(device, m, n, k, _ptr(np.ascontiguousarray(a_f16)), _ptr(np.ascontiguousarray(b_f16)),
-                                   _ptr(c), 1 if use_reference else 0), "percache_debug_gemm")
+                                   _ptr(c), 2 if pair else (1 if use_reference else 0)), "percache_debug_gemm")
     return c
 
 
