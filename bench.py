@@ -405,6 +405,91 @@ def run_qa_bank(args):
                       "batch_of_8_queries": out[8]}))
 
 
+def run_decode(args):
+    """Decode steps after a reuse-prefill of the named workload: one token per prompt and step.
+
+    HBM-bound: every step streams all weights once and every prompt's assembled K/V once."""
+    import torch
+    from paper_2601_11553_b200 import percache as pcb
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dev = torch.device("cuda", local)
+    torch.cuda.set_device(dev)
+    w = wl.by_name(args.workload[len("decode_"):])
+    shape = w.shape
+    weights_np = wl.make_weights(shape, w.seed)
+    weights = [{k: torch.from_numpy(v.view(np.int16)).to(dev).view(torch.bfloat16) for k, v in lw.items()}
+               for lw in weights_np]
+    ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
+    steps, warm = args.steps, max(args.warmup, 3)
+    reserve = warm + 2 * steps + 4
+    B = len(w.prompts)
+    stream = torch.cuda.current_stream(dev)
+    h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                     n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
+                     pool_pages=sum((l + 15) // 16 for l in ids_lens.values()) + 64,
+                     max_prompt_tokens=max(p.n_total for p in w.prompts) + reserve, max_batch_prompts=B,
+                     max_batch_ctx_tokens=w.total_tokens + B * reserve, max_batch_new_rows=w.total_tokens, device=local,
+                     stream=stream.cuda_stream)
+    del weights
+    h.set_decode_reserve(reserve)
+    cached = set(w.cached_ids)
+    for c in w.cached_ids:
+        if w.cache_source == "integer_pool":
+            h.put_chunk_synthetic(c, ids_lens[c], w.seed)
+        else:
+            h.prefill([pcb.PromptSpec([c], [ids_lens[c]], [wl.chunk_hidden_for(w.seed, c, ids_lens[c], shape.d_model)], None, 0)])
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+    specs = []
+    for p in w.prompts:
+        hid = [None if c in cached else to_dev(hh) for c, hh in zip(p.chunk_ids, p.chunk_hidden)] if p.chunk_hidden else None
+        specs.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, to_dev(p.query_hidden), p.n_query))
+    h.prefill(specs)
+    tok_dev = to_dev(wl.make_hidden(w.seed, (9, 0), B, shape.d_model))
+    tok_host = torch.from_numpy(wl.make_hidden(w.seed, (9, 0), B, shape.d_model).view(np.int16)).pin_memory().view(torch.bfloat16)
+    out_dev = torch.empty((B, shape.d_model), dtype=torch.float32, device=dev)
+    out_host = torch.empty((B, shape.d_model), dtype=torch.float32).pin_memory()
+
+    def timed(tok, out, n):
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+        ctx = 0
+        for a, b in ev:
+            a.record(stream)
+            h.decode(tok, out=out)
+            b.record(stream)
+            ctx += h.stats()["ctx_tokens"]
+        torch.cuda.synchronize(dev)
+        return [a.elapsed_time(b) for a, b in ev], ctx
+    timed(tok_dev, out_dev, warm)
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms, ctx_tokens = timed(tok_dev, out_dev, steps)
+    clocks = sampler.stop()
+    ms_e2e, _ = timed(tok_host, out_host, steps)
+    launches = sum(h.stats()["phase_launches"].values())
+    total_ms, e2e_ms = float(sum(ms)), float(sum(ms_e2e))
+    peaks = load_peaks()
+    weight_bytes = shape.params_per_layer * shape.n_layers * 2
+    kv_bytes = ctx_tokens / steps * shape.kv_dim * 2 * 2 * shape.n_layers          # fp16 K and V of every slot, every layer
+    gbs = (weight_bytes + kv_bytes) / (total_ms / steps) / 1e6
+    print(json.dumps({
+        "metric": "decode_tokens_per_s", "value": B * steps / (total_ms / 1000.0), "unit": "tokens/s", "n_gpus": 1,
+        "steps": steps, "warmup": warm, "ms_per_step": total_ms / steps, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+        "config": {"workload": args.workload, "description": "one decoded token per prompt and step after the prefill of "
+                   + w.description, "prompts": B, "ctx_tokens": ctx_tokens / steps,
+                   "l2": f"weights ({weight_bytes / 1e6:.0f} MB) exceed L2"},
+        "clocks": clocks,
+        "e2e": {"value": B * steps / (e2e_ms / 1000.0), "unit": "tokens/s", "h2d_bytes_per_step": B * shape.d_model * 2,
+                "d2h_bytes_per_step": B * shape.d_model * 4, "ms_per_step": e2e_ms / steps},
+        "gpu_launches": launches * steps,
+        "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
+                     "traffic": None, "kernel": "whole decode step (weights + assembled K/V streamed once)",
+                     "peak_source": peaks["source"], "algorithmic_per_launch": weight_bytes + kv_bytes}}))
+    h.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -417,6 +502,8 @@ def main():
     args = ap.parse_args()
     if args.workload == "qa_bank":
         run_qa_bank(args)
+    elif args.workload.startswith("decode_"):
+        run_decode(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

@@ -155,6 +155,24 @@ typedef struct {
 PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
 
+/* Decode step after a prefill (paper Section 2.1: inference is a prefill over the prompt followed by a decode
+ * stage that produces one token at a time, attending to the keys and values of everything before it).
+ * One token per prompt of the LAST percache_prefill call: hidden is bf16 [n_prompts][d_model] (row b continues
+ * prompt b; host or device memory per hidden_on_device), n_prompts must equal that call's.  Row b is at position
+ * n_total_b + (tokens decoded so far); it runs through every block like a new row of the prefill and attends to
+ * the prompt's assembled context plus itself; its rotated K and its V are appended to that context (they are
+ * not chunk content: nothing is stored).  out_hidden: caller-allocated fp32 [n_prompts][d_model], final residual
+ * stream (no final norm).  The context keeps percache_set_decode_reserve() free slots behind every prompt; a
+ * prompt that has used them all, or would pass max_prompt_tokens, -> PERCACHE_E_CAPACITY and nothing changes.
+ * Any later percache_prefill starts a new batch and discards the decoded tokens.  Synchronous. */
+PERCACHE_API int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_t hidden_on_device,
+                    float* out_hidden, int32_t out_on_device);
+
+/* Context slots kept free behind every prompt of later percache_prefill calls, so that percache_decode can
+ * append tokens (default 0: no decode).  A batch needs sum(n_total) + n_prompts * tokens_per_prompt <=
+ * max_batch_ctx_tokens, else percache_prefill returns PERCACHE_E_CAPACITY. */
+PERCACHE_API int percache_set_decode_reserve(percache_t* h, int32_t tokens_per_prompt);
+
 /* *n_tokens = stored length, or PERCACHE_E_NOTFOUND. n_tokens may be NULL. */
 PERCACHE_API int percache_has_chunk(percache_t* h, uint64_t chunk_id, int32_t* n_tokens);
 
@@ -236,7 +254,7 @@ PERCACHE_API int percache_debug_attn_plan(const int32_t* n_blocks, int32_t n_til
                              int64_t* counts_out);
 
 /* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
- * [n_total][n_kv_heads][head_dim], copied to host buffers. */
+ * [n_total + tokens decoded since][n_kv_heads][head_dim], copied to host buffers. */
 PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
 
 /* C[M][N] (fp32, host) = A[M][K] * B[N][K]^T with fp16 inputs (host), through the tcgen05 GEMM

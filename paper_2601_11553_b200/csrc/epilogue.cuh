@@ -38,16 +38,24 @@ __device__ __forceinline__ uint2 pack_half4(float a, float b, float c, float d) 
 //   V: round to bf16; keep in the page; write to the assembled context.
 // Callers give adjacent lanes adjacent column groups of the same row, so table reads and stores of
 // four lanes cover contiguous 32- to 128-byte pieces.
-__device__ __forceinline__ void qkv_store4(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c, float4 lo,
-                                           float4 hi) {
+// (cos, sin) of columns c, c+1 | c+2, c+3 at position pos; the identity for value heads.
+struct RopeCs { float4 t0, t1; };
+__device__ __forceinline__ RopeCs qkv_load_cs(const QkvEpilogue& e, int pos, int hb, int c) {
+  RopeCs r;
+  r.t0 = make_float4(1.f, 0.f, 1.f, 0.f);
+  r.t1 = r.t0;
+  if (hb < e.n_q_heads + e.n_kv_heads) {
+    const float4* t = reinterpret_cast<const float4*>(e.rope + static_cast<size_t>(pos) * ROPE_HALF + c);
+    r.t0 = __ldg(t);
+    r.t1 = __ldg(t + 1);
+  }
+  return r;
+}
+__device__ __forceinline__ void qkv_store4_cs(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c, float4 lo,
+                                              float4 hi, const RopeCs& cs) {
   const bool is_q = hb < e.n_q_heads;
   const bool is_k = !is_q && hb < e.n_q_heads + e.n_kv_heads;
-  float4 t0 = make_float4(1.f, 0.f, 1.f, 0.f), t1 = t0;       // (cos, sin) of columns c, c+1 | c+2, c+3
-  if (is_q || is_k) {
-    const float4* t = reinterpret_cast<const float4*>(e.rope + static_cast<size_t>(rw.pos) * ROPE_HALF + c);
-    t0 = __ldg(t);
-    t1 = __ldg(t + 1);
-  }
+  const float4 t0 = cs.t0, t1 = cs.t1;
   if (is_q) {
     __half* dst = e.q_out + static_cast<size_t>(row) * (e.n_q_heads * HEAD_DIM) + hb * HEAD_DIM + c;
     *reinterpret_cast<uint2*>(dst) = pack_half4(lo.x * t0.x - hi.x * t0.y, lo.y * t0.z - hi.y * t0.w,
@@ -81,6 +89,11 @@ __device__ __forceinline__ void qkv_store4(const QkvEpilogue& e, int row, const 
     *reinterpret_cast<uint2*>(dst) = pack_half4(l0, l1, l2, l3);
     *reinterpret_cast<uint2*>(dst + ROPE_HALF) = pack_half4(h0, h1, h2, h3);
   }
+}
+
+__device__ __forceinline__ void qkv_store4(const QkvEpilogue& e, int row, const QkvRow& rw, int hb, int c, float4 lo,
+                                           float4 hi) {
+  qkv_store4_cs(e, row, rw, hb, c, lo, hi, qkv_load_cs(e, rw.pos, hb, c));
 }
 
 // resid[row][col..col+3] += acc

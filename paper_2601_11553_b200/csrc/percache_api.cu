@@ -33,6 +33,8 @@ struct LayerWeights {
 
 struct Plan {   // integer description of the last successful call (host)
   std::vector<int32_t> cu_ctx, cu_new, slot_chunk, slot_offset, slot_is_new, row_slot;
+  std::vector<int32_t> ctx0;      // device context slot of every prompt's slot 0 (prompts are decode_reserve apart)
+  std::vector<int32_t> dec_len;   // tokens appended to every prompt by percache_decode since the prefill
 };
 
 constexpr int MAX_EVENTS = 1024;
@@ -85,6 +87,7 @@ struct percache {
   uint64_t next_serial = 0;
 
   Plan plan;
+  int32_t decode_reserve = 0;     // context slots kept free behind every prompt for percache_decode
   percache_stats_t stats{};
   std::vector<cudaEvent_t> events;
   cudaEvent_t ev_begin = nullptr, ev_end = nullptr;
@@ -219,6 +222,135 @@ int with_chunk_pages(percache* h, const std::vector<int32_t>& pages, Fn fn) {
   fn(h->d_index);
   if (cudaStreamSynchronize(h->stream) != cudaSuccess || cudaGetLastError() != cudaSuccess) return PERCACHE_E_CUDA;
   return PERCACHE_OK;
+}
+
+// Device-side index arrays of a call (inside h->d_index, same layout as the host block).
+struct DevIndex {
+  const int32_t *row_slot, *row_pos, *row_pool, *row_ctx0;
+  const GatherItem* items;
+  const AttnItem* attn_items;
+  const int32_t* cta_first;
+  const AttnMerge* merges;
+};
+DevIndex dev_index(const percache* h) {
+  DevIndex ix;
+  ix.row_slot = h->d_index;
+  ix.row_pos = ix.row_slot + h->m_cap;
+  ix.row_pool = ix.row_pos + h->m_cap;
+  ix.row_ctx0 = ix.row_pool + h->m_cap;
+  ix.items = reinterpret_cast<const GatherItem*>(ix.row_ctx0 + h->m_cap);
+  ix.attn_items = reinterpret_cast<const AttnItem*>(reinterpret_cast<const int32_t*>(ix.items) + 4 * h->ctx_cap);
+  ix.cta_first = reinterpret_cast<const int32_t*>(ix.attn_items) + 8 * h->max_attn_items;
+  ix.merges = reinterpret_cast<const AttnMerge*>(ix.cta_first + h->n_sms + 1);
+  return ix;
+}
+
+// Every decoder block for the Mi rows in h->resid (prefill: the new rows of the batch; decode: one row per
+// prompt): RMSNorm, QKV projection (rotation, pages, context), attention over the assembled context, output
+// projection, RMSNorm, SwiGLU FFN.  Layer l's attention first waits for ev_gather[l] when the fetch runs beside.
+bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_merges, bool overlap_gather,
+                bool use_ref, PhaseTimer& timer, cudaStream_t s) {
+  const ModelDims& D = h->dims;
+  const int d = D.d_model;
+  const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
+  const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
+  // CTA pairs pay off where the main loop is the bound: the two residual GEMMs (see umma_gemm_pick_shape)
+  const bool may_pair = !(h->flags & PERCACHE_FLAG_SINGLE_CTA_GEMM);
+  const int32_t *d_row_slot = ix.row_slot, *d_row_pos = ix.row_pos, *d_row_pool = ix.row_pool, *d_row_ctx0 = ix.row_ctx0;
+  const AttnItem* d_attn_items = ix.attn_items;
+  const int32_t* d_cta_first = ix.cta_first;
+  const AttnMerge* d_merges = ix.merges;
+  bool ok = true;
+  for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
+    LayerWeights& W = h->layers[l];
+    timer.begin(PERCACHE_PH_NORM);
+    launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
+    timer.end();
+
+    QkvEpilogue qe;
+    qe.rows = RowIndex{d_row_slot, d_row_pos, d_row_pool};
+    qe.rope = h->rope;
+    qe.q_out = h->qbuf;
+    qe.kpool = h->kpool + l * pool_layer;
+    qe.vpool = h->vpool + l * pool_layer;
+    qe.kctx = h->kctx + l * ctx_layer;
+    qe.vctx = h->vctx + l * ctx_layer;
+    qe.n_q_heads = D.n_q_heads;
+    qe.n_kv_heads = D.n_kv_heads;
+    timer.begin(PERCACHE_PH_QKV);
+    if (use_ref) {
+      launch_ref_gemm(h->xn, W.wqkv, h->cref, Mi, D.qkv_dim, d, s);
+      launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
+    } else {
+      {
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, false, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
+      }
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_ATTN);
+    if (overlap_gather) ok = ok && cudaStreamWaitEvent(s, h->ev_gather[l], 0) == cudaSuccess;
+    if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
+      launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
+    } else {
+      ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
+                                       h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s) == 0;
+      launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
+    }
+    timer.end();
+
+    ResidualEpilogue re{h->resid, d};
+    timer.begin(PERCACHE_PH_OPROJ);
+    if (use_ref) {
+      launch_ref_gemm(h->attn_out, W.wo, h->cref, Mi, d, D.q_dim, s);
+      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
+    } else {
+      {
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, d, D.q_dim, h->n_sms, true, may_pair, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_attn, (bn == 256 && !pr) ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
+      }
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_NORM);
+    launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
+    timer.end();
+
+    SwigluEpilogue se{h->act, D.d_ffn};
+    timer.begin(PERCACHE_PH_GATEUP);
+    if (use_ref) {
+      launch_ref_gemm(h->xn, W.wgu, h->cref, Mi, 2 * D.d_ffn, d, s);
+      launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
+    } else {
+      {
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, false, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
+      }
+    }
+    timer.end();
+
+    timer.begin(PERCACHE_PH_DOWN);
+    if (use_ref) {
+      launch_ref_gemm(h->act, W.wd, h->cref, Mi, d, D.d_ffn, s);
+      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
+    } else {
+      {
+        int bn, ks, pr;
+        umma_gemm_pick_shape(Mi, d, D.d_ffn, h->n_sms, true, may_pair, &bn, &ks, &pr);
+        ok = ok && launch_umma_gemm(h->m_act, (bn == 256 && !pr) ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
+                                    h->d_err, h->n_sms, s, ks, pr) == 0;
+      }
+    }
+    timer.end();
+  }
+  return ok;
 }
 
 }  // namespace
@@ -635,7 +767,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     if (results[b].out_capacity_rows < n_new || (n_new > 0 && !results[b].out_hidden)) return PERCACHE_E_CAPACITY;
     ctx_total += T;
     new_total += n_new;
-    if (ctx_total > h->ctx_cap || new_total > h->m_cap) return PERCACHE_E_CAPACITY;
+    if (ctx_total + static_cast<int64_t>(b + 1) * h->decode_reserve > h->ctx_cap || new_total > h->m_cap)
+      return PERCACHE_E_CAPACITY;
     plan.cu_ctx.push_back(static_cast<int32_t>(ctx_total));
     plan.cu_new.push_back(static_cast<int32_t>(new_total));
   }
@@ -685,7 +818,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   int64_t r = 0;
   for (int b = 0; b < n_prompts; ++b) {
     const percache_prompt_t& P = prompts[b];
-    const int32_t ctx0 = plan.cu_ctx[b];
+    const int32_t pbase = plan.cu_ctx[b];                              // index into the plan's per-slot arrays
+    const int32_t ctx0 = pbase + b * h->decode_reserve;                // slot in the device context
+    plan.ctx0.push_back(ctx0);
+    plan.dec_len.push_back(0);
     int32_t t = 0;
     for (int i = 0; i <= P.n_chunks; ++i) {
       const bool is_query = (i == P.n_chunks);
@@ -693,9 +829,9 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       if (len == 0) continue;
       const bool is_hit = !is_query && hit[b][i];
       for (int o = 0; o < len; ++o) {
-        plan.slot_chunk[ctx0 + t + o] = i;
-        plan.slot_offset[ctx0 + t + o] = o;
-        plan.slot_is_new[ctx0 + t + o] = is_hit ? 0 : 1;
+        plan.slot_chunk[pbase + t + o] = i;
+        plan.slot_offset[pbase + t + o] = o;
+        plan.slot_is_new[pbase + t + o] = is_hit ? 0 : 1;
       }
       if (is_hit) {
         const ChunkEntry& ent = h->table.find(keys[b][i])->second;
@@ -796,8 +932,6 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
   const int Mi = static_cast<int>(M);
-  // CTA pairs pay off where the main loop is the bound: the two residual GEMMs (see umma_gemm_pick_shape)
-  const bool may_pair = !(h->flags & PERCACHE_FLAG_SINGLE_CTA_GEMM);
   if (overlap_gather) {
     ok = ok && cudaEventRecord(h->ev_fork, s) == cudaSuccess && cudaStreamWaitEvent(h->side, h->ev_fork, 0) == cudaSuccess;
     for (int l = 0; l < D.n_layers && ok; ++l) {
@@ -811,95 +945,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
                          h->ctx_cap, D.kv_dim, h->rope, s);
     timer.end();
   }
-  for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
-    LayerWeights& W = h->layers[l];
-    timer.begin(PERCACHE_PH_NORM);
-    launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
-    timer.end();
-
-    QkvEpilogue qe;
-    qe.rows = RowIndex{d_row_slot, d_row_pos, d_row_pool};
-    qe.rope = h->rope;
-    qe.q_out = h->qbuf;
-    qe.kpool = h->kpool + l * pool_layer;
-    qe.vpool = h->vpool + l * pool_layer;
-    qe.kctx = h->kctx + l * ctx_layer;
-    qe.vctx = h->vctx + l * ctx_layer;
-    qe.n_q_heads = D.n_q_heads;
-    qe.n_kv_heads = D.n_kv_heads;
-    timer.begin(PERCACHE_PH_QKV);
-    if (use_ref) {
-      launch_ref_gemm(h->xn, W.wqkv, h->cref, Mi, D.qkv_dim, d, s);
-      launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
-    } else {
-      {
-        int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, false, &bn, &ks, &pr);
-        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
-                                    h->d_err, h->n_sms, s, ks, pr) == 0;
-      }
-    }
-    timer.end();
-
-    timer.begin(PERCACHE_PH_ATTN);
-    if (overlap_gather) ok = ok && cudaStreamWaitEvent(s, h->ev_gather[l], 0) == cudaSuccess;
-    if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
-      launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
-    } else {
-      ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
-                                       h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s) == 0;
-      launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
-    }
-    timer.end();
-
-    ResidualEpilogue re{h->resid, d};
-    timer.begin(PERCACHE_PH_OPROJ);
-    if (use_ref) {
-      launch_ref_gemm(h->attn_out, W.wo, h->cref, Mi, d, D.q_dim, s);
-      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
-    } else {
-      {
-        int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, d, D.q_dim, h->n_sms, true, may_pair, &bn, &ks, &pr);
-        ok = ok && launch_umma_gemm(h->m_attn, (bn == 256 && !pr) ? W.m_wo256 : W.m_wo, Mi, d, D.q_dim, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s, ks, pr) == 0;
-      }
-    }
-    timer.end();
-
-    timer.begin(PERCACHE_PH_NORM);
-    launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
-    timer.end();
-
-    SwigluEpilogue se{h->act, D.d_ffn};
-    timer.begin(PERCACHE_PH_GATEUP);
-    if (use_ref) {
-      launch_ref_gemm(h->xn, W.wgu, h->cref, Mi, 2 * D.d_ffn, d, s);
-      launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
-    } else {
-      {
-        int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, false, &bn, &ks, &pr);
-        ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
-                                    h->d_err, h->n_sms, s, ks, pr) == 0;
-      }
-    }
-    timer.end();
-
-    timer.begin(PERCACHE_PH_DOWN);
-    if (use_ref) {
-      launch_ref_gemm(h->act, W.wd, h->cref, Mi, d, D.d_ffn, s);
-      launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
-    } else {
-      {
-        int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, d, D.d_ffn, h->n_sms, true, may_pair, &bn, &ks, &pr);
-        ok = ok && launch_umma_gemm(h->m_act, (bn == 256 && !pr) ? W.m_wd256 : W.m_wd, Mi, d, D.d_ffn, bn, EPI_RESIDUAL, &re, nullptr,
-                                    h->d_err, h->n_sms, s, ks, pr) == 0;
-      }
-    }
-    timer.end();
-  }
+  ok = ok && (Mi <= 0 || run_layers(h, Mi, dev_index(h), n_attn_ctas, n_merges, overlap_gather, use_ref, timer, s));
   cudaEventRecord(h->ev_end, s);
   timer.begin(PERCACHE_PH_IO);
   for (int b = 0; b < n_prompts && ok; ++b) {
@@ -936,6 +982,106 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   refresh_page_stats(h);
   st.host_plan_us = plan_us;
   st.attn_visible_pairs = visible_pairs;
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
+  st.device_us = 1000.0 * ms;
+  timer.collect();
+  return PERCACHE_OK;
+}
+
+int percache_set_decode_reserve(percache_t* h, int32_t tokens_per_prompt) {
+  if (!h || tokens_per_prompt < 0) return PERCACHE_E_INVAL;
+  h->decode_reserve = tokens_per_prompt;
+  return PERCACHE_OK;
+}
+
+int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_t hidden_on_device, float* out_hidden,
+                    int32_t out_on_device) {
+  if (!h || !hidden || !out_hidden || n_prompts <= 0) return PERCACHE_E_INVAL;
+  Plan& plan = h->plan;
+  if (static_cast<size_t>(n_prompts) + 1 != plan.cu_ctx.size()) return PERCACHE_E_INVAL;   // not the last call's batch
+  if (n_prompts > h->m_cap) return PERCACHE_E_CAPACITY;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  const auto t_host0 = std::chrono::steady_clock::now();
+  const ModelDims& D = h->dims;
+  const int d = D.d_model;
+  int32_t* row_slot = h->h_index;
+  int32_t* row_pos = row_slot + h->m_cap;
+  int32_t* row_pool = row_pos + h->m_cap;
+  int32_t* row_ctx0 = row_pool + h->m_cap;
+  GatherItem* items = reinterpret_cast<GatherItem*>(row_ctx0 + h->m_cap);
+  AttnItem* attn_items = reinterpret_cast<AttnItem*>(reinterpret_cast<int32_t*>(items) + 4 * h->ctx_cap);
+  int32_t* cta_first = reinterpret_cast<int32_t*>(attn_items) + 8 * h->max_attn_items;
+  AttnMerge* merges = reinterpret_cast<AttnMerge*>(cta_first + h->n_sms + 1);
+  std::vector<AttnBaseTile> base_tiles;
+  int64_t visible_pairs = 0;
+  for (int b = 0; b < n_prompts; ++b) {
+    const int32_t T = plan.cu_ctx[b + 1] - plan.cu_ctx[b] + plan.dec_len[b];     // tokens so far = the new position
+    if (plan.dec_len[b] >= h->decode_reserve || T + 1 > h->cfg.max_prompt_tokens) return PERCACHE_E_CAPACITY;
+    row_slot[b] = plan.ctx0[b] + T;
+    row_pos[b] = T;
+    row_pool[b] = -1;                       // decoded tokens are not chunk content: nothing goes to the store
+    row_ctx0[b] = plan.ctx0[b];
+    base_tiles.push_back(AttnBaseTile{b, 1, plan.ctx0[b], (T + 1 + 127) / 128});
+    visible_pairs += T + 1;
+  }
+  std::vector<AttnItem> v_items;
+  std::vector<int32_t> v_first;
+  std::vector<AttnMerge> v_merges;
+  plan_attention(base_tiles, D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2), h->n_sms, h->partial_slots, &v_items,
+                 &v_first, &v_merges);
+  if (v_items.size() > h->max_attn_items || v_merges.size() > h->max_attn_merges ||
+      v_first.size() > static_cast<size_t>(h->n_sms) + 1)
+    return PERCACHE_E_CAPACITY;
+  std::copy(v_items.begin(), v_items.end(), attn_items);
+  std::fill(cta_first, cta_first + h->n_sms + 1, static_cast<int32_t>(v_items.size()));
+  std::copy(v_first.begin(), v_first.end(), cta_first);
+  std::copy(v_merges.begin(), v_merges.end(), merges);
+  const int n_attn_ctas = static_cast<int>(v_first.size()) - 1;
+  const int n_merges = static_cast<int>(v_merges.size());
+  const double plan_us =
+      std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
+
+  cudaStream_t s = h->stream;
+  percache_stats_t& st = h->stats;
+  std::memset(st.phase_us, 0, sizeof(st.phase_us));
+  std::memset(st.phase_launches, 0, sizeof(st.phase_launches));
+  PhaseTimer timer(h);
+  const bool use_ref = (h->flags & PERCACHE_FLAG_REFERENCE_KERNELS) != 0;
+  if (use_ref && !h->cref) {
+    const size_t wide = static_cast<size_t>(std::max(std::max(D.qkv_dim, 2 * D.d_ffn), d));
+    if (!dev_alloc(h, &h->cref, static_cast<size_t>(h->m_cap) * wide)) return PERCACHE_E_NOMEM;
+  }
+  bool ok = true;
+  const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(merges + n_merges) - h->h_index);
+  ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
+  timer.begin(PERCACHE_PH_IO);
+  ok = ok && cudaMemcpyAsync(h->xin, hidden, static_cast<size_t>(n_prompts) * d * 2,
+                             hidden_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s) == cudaSuccess;
+  cudaEventRecord(h->ev_begin, s);
+  launch_bf16_to_f32(h->xin, h->resid, static_cast<int64_t>(n_prompts) * d, s);
+  timer.end();
+  ok = ok && run_layers(h, n_prompts, dev_index(h), n_attn_ctas, n_merges, false, use_ref, timer, s);
+  cudaEventRecord(h->ev_end, s);
+  timer.begin(PERCACHE_PH_IO);
+  ok = ok && cudaMemcpyAsync(out_hidden, h->resid, static_cast<size_t>(n_prompts) * d * sizeof(float),
+                             out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  timer.end();
+  const cudaError_t sync_rc = cudaStreamSynchronize(s);
+  if (!ok || sync_rc != cudaSuccess || cudaGetLastError() != cudaSuccess) return PERCACHE_E_CUDA;
+  if (*h->h_err != 0) return PERCACHE_E_DEVICE_TIMEOUT;
+  for (int b = 0; b < n_prompts; ++b) plan.dec_len[b] += 1;      // the token's K/V now is part of the context
+  st.n_prompts = n_prompts;
+  st.chunks_hit = st.chunks_missed = 0;
+  st.hit_tokens = 0;
+  st.new_rows = n_prompts;
+  st.ctx_tokens = 0;
+  for (int b = 0; b < n_prompts; ++b) st.ctx_tokens += plan.cu_ctx[b + 1] - plan.cu_ctx[b] + plan.dec_len[b];
+  st.host_plan_us = plan_us;
+  st.attn_visible_pairs = visible_pairs;
+  st.evictions = 0;
   float ms = 0.f;
   cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
   st.device_us = 1000.0 * ms;
@@ -1002,8 +1148,9 @@ int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* 
     return PERCACHE_E_INVAL;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * h->dims.kv_dim;
-  const size_t off = layer * ctx_layer + static_cast<size_t>(h->plan.cu_ctx[prompt]) * h->dims.kv_dim;
-  const size_t bytes = static_cast<size_t>(h->plan.cu_ctx[prompt + 1] - h->plan.cu_ctx[prompt]) * h->dims.kv_dim * 2;
+  const size_t off = layer * ctx_layer + static_cast<size_t>(h->plan.ctx0[prompt]) * h->dims.kv_dim;
+  const size_t bytes = static_cast<size_t>(h->plan.cu_ctx[prompt + 1] - h->plan.cu_ctx[prompt] + h->plan.dec_len[prompt]) *
+                       h->dims.kv_dim * 2;
   if (cudaMemcpy(k_host, h->kctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemcpy(v_host, h->vctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
     return PERCACHE_E_CUDA;

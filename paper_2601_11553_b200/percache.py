@@ -30,7 +30,7 @@ PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
-           "percache_get_stats", "percache_set_flags", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx", "percache_debug_attn_plan",
+           "percache_get_stats", "percache_set_flags", "percache_decode", "percache_set_decode_reserve", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx", "percache_debug_attn_plan",
            "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_qa_top1", "percache_strerror")
 
 
@@ -88,6 +88,8 @@ def load_library() -> C.CDLL:
     lib.percache_destroy.argtypes = [vp]
     lib.percache_put_chunk_kv.argtypes = [vp, u64, i32, vp, vp, i32]
     lib.percache_prefill.argtypes = [vp, C.POINTER(PromptStruct), i32, C.POINTER(ResultStruct)]
+    lib.percache_decode.argtypes = [vp, i32, vp, i32, vp, i32]
+    lib.percache_set_decode_reserve.argtypes = [vp, i32]
     lib.percache_has_chunk.argtypes = [vp, u64, C.POINTER(i32)]
     lib.percache_drop_chunk.argtypes = [vp, u64]
     lib.percache_get_chunk_kv.argtypes = [vp, u64, vp, vp]
@@ -296,6 +298,23 @@ class PerCache:
                              int(rs[b].n_total)) for b in range(n)]
 
     # ------------------------------------------------------------------ introspection
+    def set_decode_reserve(self, tokens_per_prompt: int) -> None:
+        """Keep this many context slots free behind every prompt of later prefill calls (for decode)."""
+        _check(self._lib.percache_set_decode_reserve(self._h, int(tokens_per_prompt)), "percache_set_decode_reserve")
+
+    def decode(self, hidden: Any, out: Optional[Any] = None):
+        """percache_decode: one token per prompt of the last prefill call.
+
+        hidden: bf16 [n_prompts, d_model] as a uint16/bf16 numpy array (host) or a torch device tensor.
+        Returns fp32 [n_prompts, d_model] (numpy), or fills and returns `out` (host numpy or device tensor).
+        """
+        n = int(hidden.shape[0])
+        if out is None:
+            out = np.empty((n, self.d_model), dtype=np.float32)
+        _check(self._lib.percache_decode(self._h, n, _ptr(hidden), 1 if _is_device(hidden) else 0, _ptr(out),
+                                         1 if _is_device(out) else 0), "percache_decode")
+        return out
+
     def stats(self) -> Dict[str, Any]:
         s = StatsStruct()
         _check(self._lib.percache_get_stats(self._h, C.byref(s)), "percache_get_stats")

@@ -15,9 +15,9 @@ TOL_MEAN_ABS = 3e-3
 
 
 def make_handle(shape: wl.ModelShape, weights: List[dict], prompts: Sequence[wl.Prompt], pool_pages: int = 0,
-                flags: int = 0, slack_prompts: int = 0) -> pcb.PerCache:
-    max_t = max(p.n_total for p in prompts)
-    total = sum(p.n_total for p in prompts)
+                flags: int = 0, slack_prompts: int = 0, decode_reserve: int = 0) -> pcb.PerCache:
+    max_t = max(p.n_total for p in prompts) + decode_reserve
+    total = sum(p.n_total for p in prompts) + decode_reserve * len(prompts)
     if pool_pages <= 0:
         pool_pages = sum((l + 15) // 16 for p in prompts for l in p.chunk_len) + 64
     return pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
