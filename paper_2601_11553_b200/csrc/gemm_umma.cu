@@ -479,6 +479,8 @@ void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool
     const int workers = pr ? n_sms / 2 : n_sms;
     const int64_t clocks = shape == 0 ? 512 : (shape == 1 ? 768 : 600);
     const int64_t tiles = static_cast<int64_t>((M + tile_m - 1) / tile_m) * (N / bn);
+    // small problems (under half a round of pair tiles) are bound by ramp-up and tail, which pairs lengthen
+    if (pr && tiles * 2 < workers) continue;
     for (int sp = 1; sp <= (may_split_k ? 8 : 1); ++sp) {
       if (sp > 1 && n_kb / sp < 4) break;
       const int64_t rounds = (tiles * sp + workers - 1) / workers;
