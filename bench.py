@@ -421,7 +421,7 @@ def run_decode(args):
                for lw in weights_np]
     ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
     steps, warm = args.steps, max(args.warmup, 3)
-    reserve = warm + 2 * steps + 4
+    reserve = warm + 2 * steps + 8
     B = len(w.prompts)
     stream = torch.cuda.current_stream(dev)
     h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
@@ -432,6 +432,7 @@ def run_decode(args):
                      stream=stream.cuda_stream)
     del weights
     h.set_decode_reserve(reserve)
+    h.set_flags(args.flags)
     cached = set(w.cached_ids)
     for c in w.cached_ids:
         if w.cache_source == "integer_pool":
@@ -453,21 +454,33 @@ def run_decode(args):
 
     def timed(tok, out, n):
         ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
-        ctx = 0
+        ctx, dev_us = 0, 0.0
         for a, b in ev:
             a.record(stream)
             h.decode(tok, out=out)
             b.record(stream)
-            ctx += h.stats()["ctx_tokens"]
+            st = h.stats()
+            ctx += st["ctx_tokens"]
+            dev_us += st["device_us"]
         torch.cuda.synchronize(dev)
+        timed.device_ms = dev_us / 1000.0 / n
         return [a.elapsed_time(b) for a, b in ev], ctx
     timed(tok_dev, out_dev, warm)
     sampler = ClockSampler(local)
     sampler.start()
     ms, ctx_tokens = timed(tok_dev, out_dev, steps)
+    device_ms = timed.device_ms
     clocks = sampler.stop()
     ms_e2e, _ = timed(tok_host, out_host, steps)
     launches = sum(h.stats()["phase_launches"].values())
+    # per-kernel-class durations from a separate pass with events around every class
+    h.set_flags(args.flags | pcb.FLAG_PHASE_TIMING)
+    h.decode(tok_dev, out=out_dev)
+    h.decode(tok_dev, out=out_dev)
+    st = h.stats()
+    h.set_flags(args.flags)
+    per_phase = {k: {"us_per_launch": st["phase_us"][k] / st["phase_launches"][k], "launches_per_step": st["phase_launches"][k]}
+                 for k in pcb.PHASES if st["phase_launches"][k]}
     total_ms, e2e_ms = float(sum(ms)), float(sum(ms_e2e))
     peaks = load_peaks()
     weight_bytes = shape.params_per_layer * shape.n_layers * 2
@@ -479,6 +492,7 @@ def run_decode(args):
         "vs_baseline": None, "dtype": "f16", "data": "synthetic",
         "config": {"workload": args.workload, "description": "one decoded token per prompt and step after the prefill of "
                    + w.description, "prompts": B, "ctx_tokens": ctx_tokens / steps,
+                   "device_ms_per_step_kernels_only": device_ms,
                    "l2": f"weights ({weight_bytes / 1e6:.0f} MB) exceed L2"},
         "clocks": clocks,
         "e2e": {"value": B * steps / (e2e_ms / 1000.0), "unit": "tokens/s", "h2d_bytes_per_step": B * shape.d_model * 2,
@@ -486,7 +500,8 @@ def run_decode(args):
         "gpu_launches": launches * steps,
         "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
                      "traffic": None, "kernel": "whole decode step (weights + assembled K/V streamed once)",
-                     "peak_source": peaks["source"], "algorithmic_per_launch": weight_bytes + kv_bytes}}))
+                     "peak_source": peaks["source"], "algorithmic_per_launch": weight_bytes + kv_bytes},
+        "kernels": per_phase}))
     h.close()
 
 

@@ -65,6 +65,8 @@ extern "C" {
 #define PERCACHE_FLAG_PHASE_TIMING       2u  /* record CUDA events around every kernel class (see stats)       */
 #define PERCACHE_FLAG_REFERENCE_ATTENTION 4u /* debugging aid: plain attention kernel, tcgen05 GEMMs            */
 #define PERCACHE_FLAG_SINGLE_CTA_GEMM   16u  /* debugging aid: never run a GEMM on CTA pairs (256 x 256 tiles)     */
+#define PERCACHE_FLAG_NO_SMALL_ROW_KERNELS 32u /* debugging aid: calls with at most 8 rows (decode) use the tcgen05
+                                                GEMMs like any other instead of the weight-streaming kernels     */
 #define PERCACHE_FLAG_EVICT_LFU          8u  /* when the store is full, evict least-frequently-used chunks instead
                                                 of failing with PERCACHE_E_NOSPACE (see percache_set_store_limit)  */
 

@@ -375,10 +375,12 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
 }
 
 // Merge of the parts of a split unit: out[row][head] = sum_s 2^(m_s - M) O_s / sum_s 2^(m_s - M) l_s with
-// M = max_s m_s.  One warp per (row, head): lanes first take one part each for the (reference, sum) pairs,
-// then every lane owns four output columns and walks the parts with independent 16-byte loads.
+// M = max_s m_s.  A warp takes MERGE_ROWS rows of one (unit, head) at a time: for each row, lane s holds part s's
+// (reference, sum) pair and its weight, every lane owns four output columns, and the loads of up to four parts
+// of all the warp's rows are in flight together (the kernel is a chain of short dependent loads otherwise).
 namespace {
 constexpr int MERGE_WARPS = 8;
+constexpr int MERGE_ROWS = 2;
 __global__ void __launch_bounds__(MERGE_WARPS * 32)
 attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
                        const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads, int n_kv_heads) {
@@ -389,37 +391,62 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __rest
   const int i = blockIdx.y;
   const int head = (mg.unit / pairs) * group + 2 * (mg.unit % pairs) + i;
   const int lane = threadIdx.x & 31;
-  const int r = blockIdx.z * MERGE_WARPS + (threadIdx.x >> 5);
-  if (r >= mg.n_rows) return;
+  const int r0 = (blockIdx.z * MERGE_WARPS + (threadIdx.x >> 5)) * MERGE_ROWS;
+  if (r0 >= mg.n_rows) return;
   const size_t slot0 = static_cast<size_t>(mg.partial_slot0) * 2 + i;     // part s is two slots further each
-  float M = -INFINITY;
-  for (int s = lane; s < mg.n_parts; s += 32)
-    M = fmaxf(M, partial_ml[((slot0 + 2 * s) * BLK + r) * 2]);
+  float w[MERGE_ROWS], inv[MERGE_ROWS];
+  float4 acc[MERGE_ROWS];
 #pragma unroll
-  for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
-  float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-  float l = 0.f;
-#pragma unroll 4
-  for (int s = 0; s < mg.n_parts; ++s) {
-    const size_t slot = slot0 + 2 * s;
-    const float2 ml = *reinterpret_cast<const float2*>(partial_ml + (slot * BLK + r) * 2);
-    const float w = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;
-    const float4 o = *reinterpret_cast<const float4*>(partial_o + (slot * BLK + r) * HEAD_DIM + lane * 4);
-    acc.x = fmaf(w, o.x, acc.x); acc.y = fmaf(w, o.y, acc.y);
-    acc.z = fmaf(w, o.z, acc.z); acc.w = fmaf(w, o.w, acc.w);
-    l = fmaf(w, ml.y, l);
+  for (int k = 0; k < MERGE_ROWS; ++k) {
+    const int r = min(r0 + k, mg.n_rows - 1);
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < mg.n_parts) ml = *reinterpret_cast<const float2*>(partial_ml + ((slot0 + 2 * lane) * BLK + r) * 2);
+    float M = ml.y > 0.f ? ml.x : -INFINITY;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
+    w[k] = ml.y > 0.f ? exp2f(ml.x - M) : 0.f;
+    float l = w[k] * ml.y;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) l += __shfl_xor_sync(0xffffffffu, l, o);
+    inv[k] = 1.0f / l;
+    acc[k] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-  const float inv = 1.0f / l;
-  __half2 a = __floats2half2_rn(acc.x * inv, acc.y * inv), b = __floats2half2_rn(acc.z * inv, acc.w * inv);
-  *reinterpret_cast<uint2*>(out + (static_cast<size_t>(mg.row0 + r) * n_q_heads + head) * HEAD_DIM + lane * 4) =
-      make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+  for (int s0 = 0; s0 < mg.n_parts; s0 += 4) {          // n_parts <= 32: the weights live in lanes 0..n_parts-1
+    float4 o[MERGE_ROWS][4];
+#pragma unroll
+    for (int k = 0; k < MERGE_ROWS; ++k) {
+      const int r = min(r0 + k, mg.n_rows - 1);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        const int sp = min(s0 + q, mg.n_parts - 1);       // a repeated part gets weight zero below
+        o[k][q] = __ldg(reinterpret_cast<const float4*>(partial_o + ((slot0 + 2 * sp) * BLK + r) * HEAD_DIM + lane * 4));
+      }
+    }
+#pragma unroll
+    for (int k = 0; k < MERGE_ROWS; ++k)
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        float ws = __shfl_sync(0xffffffffu, w[k], (s0 + q) & 31);
+        if (s0 + q >= mg.n_parts) ws = 0.f;
+        acc[k].x = fmaf(ws, o[k][q].x, acc[k].x); acc[k].y = fmaf(ws, o[k][q].y, acc[k].y);
+        acc[k].z = fmaf(ws, o[k][q].z, acc[k].z); acc[k].w = fmaf(ws, o[k][q].w, acc[k].w);
+      }
+  }
+#pragma unroll
+  for (int k = 0; k < MERGE_ROWS; ++k) {
+    if (r0 + k >= mg.n_rows) break;
+    __half2 a = __floats2half2_rn(acc[k].x * inv[k], acc[k].y * inv[k]);
+    __half2 b = __floats2half2_rn(acc[k].z * inv[k], acc[k].w * inv[k]);
+    *reinterpret_cast<uint2*>(out + (static_cast<size_t>(mg.row0 + r0 + k) * n_q_heads + head) * HEAD_DIM + lane * 4) =
+        make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+  }
 }
 }  // namespace
 
 void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
                             __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s) {
   if (n_merges <= 0) return;
-  dim3 grid(n_merges, 2, BLK / MERGE_WARPS);
+  dim3 grid(n_merges, 2, BLK / (MERGE_WARPS * MERGE_ROWS));
   launch_pdl(attention_merge_kernel, grid, dim3(MERGE_WARPS * 32), 0, s, merges, partial_o, partial_ml, out, n_q_heads,
              n_kv_heads);
 }
@@ -430,9 +457,13 @@ int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int
   if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0) return -1;
-  if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
-      cudaSuccess)
-    return -1;
+  static bool smem_set = false;      // once per process: the call costs host time on every launch otherwise
+  if (!smem_set) {
+    if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
+        cudaSuccess)
+      return -1;
+    smem_set = true;
+  }
   AttnArgs a{};
   a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out;
   a.partial_o = partial_o; a.partial_ml = partial_ml;

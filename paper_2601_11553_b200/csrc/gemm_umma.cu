@@ -376,9 +376,13 @@ EncodeTiledFn g_encode = nullptr;
 template <int BN, int KIND, bool PAIR>
 int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, int n_sms, cudaStream_t s) {
   using Cfg = GemmCfg<BN, PAIR>;
-  if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           Cfg::SMEM_BYTES) != cudaSuccess)
-    return -1;
+  static bool smem_set = false;      // per kernel instantiation, once per process
+  if (!smem_set) {
+    if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             Cfg::SMEM_BYTES) != cudaSuccess)
+      return -1;
+    smem_set = true;
+  }
   constexpr int TILE_M = PAIR ? 2 * BM : BM;
   const int n_tiles = ((args.M + TILE_M - 1) / TILE_M) * (args.N / BN) * (args.k_splits > 0 ? args.k_splits : 1);
   if (n_tiles <= 0) return 0;

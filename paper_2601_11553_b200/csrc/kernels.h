@@ -125,6 +125,15 @@ int umma_gemm_pick_block_n(int M, int N, int n_sms);   // 128 or 256 for this pr
 void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
                           int* k_splits, int* pair);
 
+// ---- projections for at most SMALL_GEMM_MAX_ROWS rows on the CUDA cores, bound by reading W once (gemm_small.cu).
+// D[M][N] = A[M][K] * W[N][K]^T with the epilogue `kind` (EPI_QKV, EPI_RESIDUAL or EPI_SWIGLU, parameter block as
+// for the tcgen05 GEMM).  Input: x_f32 + gain (the RMSNorm of fp32 rows is applied on the way; QKV and SwiGLU) or
+// a_f16 (residual kind).  gu_blk: gate / up row interleave of W for EPI_SWIGLU.  K % 256 == 0.
+constexpr int SMALL_GEMM_MAX_ROWS = 8;
+int launch_small_gemm(GemmEpilogueKind kind, const void* epilogue, int M, int N, int K, const float* x_f32,
+                      const float* gain, float eps, const __half* a_f16, const __half* w, int gu_blk, int n_sms,
+                      cudaStream_t s);
+
 // rank-N fp16 tensor map with 128-byte swizzle; dims/strides innermost first (strides in bytes, from dim 1)
 int encode_f16_map(CUtensorMap* out, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                    const uint32_t* box);

@@ -260,12 +260,18 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   const AttnItem* d_attn_items = ix.attn_items;
   const int32_t* d_cta_first = ix.cta_first;
   const AttnMerge* d_merges = ix.merges;
+  // A handful of rows (decode) is a matter of reading the weights once: CUDA-core kernels bound by HBM, with the
+  // RMSNorm folded into the QKV and gate/up projections
+  const bool small_rows = !use_ref && !(h->flags & PERCACHE_FLAG_NO_SMALL_ROW_KERNELS) && Mi <= SMALL_GEMM_MAX_ROWS &&
+                          d % 256 == 0 && D.q_dim % 256 == 0 && D.d_ffn % 256 == 0;
   bool ok = true;
   for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
     LayerWeights& W = h->layers[l];
-    timer.begin(PERCACHE_PH_NORM);
-    launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
-    timer.end();
+    if (!small_rows) {
+      timer.begin(PERCACHE_PH_NORM);
+      launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
+      timer.end();
+    }
 
     QkvEpilogue qe;
     qe.rows = RowIndex{d_row_slot, d_row_pos, d_row_pool};
@@ -278,7 +284,10 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     qe.n_q_heads = D.n_q_heads;
     qe.n_kv_heads = D.n_kv_heads;
     timer.begin(PERCACHE_PH_QKV);
-    if (use_ref) {
+    if (small_rows) {
+      ok = ok && launch_small_gemm(EPI_QKV, &qe, Mi, D.qkv_dim, d, h->resid, W.g_attn, D.rms_eps, nullptr, W.wqkv, 0,
+                                   h->n_sms, s) == 0;
+    } else if (use_ref) {
       launch_ref_gemm(h->xn, W.wqkv, h->cref, Mi, D.qkv_dim, d, s);
       launch_ref_qkv_epilogue(h->cref, Mi, qe, s);
     } else {
@@ -304,7 +313,10 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
 
     ResidualEpilogue re{h->resid, d};
     timer.begin(PERCACHE_PH_OPROJ);
-    if (use_ref) {
+    if (small_rows) {
+      ok = ok && launch_small_gemm(EPI_RESIDUAL, &re, Mi, d, D.q_dim, nullptr, nullptr, 0.f, h->attn_out, W.wo, 0,
+                                   h->n_sms, s) == 0;
+    } else if (use_ref) {
       launch_ref_gemm(h->attn_out, W.wo, h->cref, Mi, d, D.q_dim, s);
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
@@ -317,13 +329,18 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     }
     timer.end();
 
-    timer.begin(PERCACHE_PH_NORM);
-    launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
-    timer.end();
+    if (!small_rows) {
+      timer.begin(PERCACHE_PH_NORM);
+      launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
+      timer.end();
+    }
 
     SwigluEpilogue se{h->act, D.d_ffn};
     timer.begin(PERCACHE_PH_GATEUP);
-    if (use_ref) {
+    if (small_rows) {
+      ok = ok && launch_small_gemm(EPI_SWIGLU, &se, Mi, 2 * D.d_ffn, d, h->resid, W.g_ffn, D.rms_eps, nullptr, W.wgu,
+                                   h->gu_blk, h->n_sms, s) == 0;
+    } else if (use_ref) {
       launch_ref_gemm(h->xn, W.wgu, h->cref, Mi, 2 * D.d_ffn, d, s);
       launch_ref_swiglu_epilogue(h->cref, Mi, D.d_ffn, h->gu_blk, se, s);
     } else {
@@ -337,7 +354,10 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     timer.end();
 
     timer.begin(PERCACHE_PH_DOWN);
-    if (use_ref) {
+    if (small_rows) {
+      ok = ok && launch_small_gemm(EPI_RESIDUAL, &re, Mi, d, D.d_ffn, nullptr, nullptr, 0.f, h->act, W.wd, 0, h->n_sms,
+                                   s) == 0;
+    } else if (use_ref) {
       launch_ref_gemm(h->act, W.wd, h->cref, Mi, d, D.d_ffn, s);
       launch_ref_residual_epilogue(h->cref, Mi, d, re, s);
     } else {
@@ -907,14 +927,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(merges + n_merges) - h->h_index);
   ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
-  const int32_t* d_row_slot = h->d_index;
-  const int32_t* d_row_pos = d_row_slot + h->m_cap;
-  const int32_t* d_row_pool = d_row_pos + h->m_cap;
-  const int32_t* d_row_ctx0 = d_row_pool + h->m_cap;
-  const GatherItem* d_items = reinterpret_cast<const GatherItem*>(d_row_ctx0 + h->m_cap);
-  const AttnItem* d_attn_items = reinterpret_cast<const AttnItem*>(reinterpret_cast<const int32_t*>(d_items) + 4 * h->ctx_cap);
-  const int32_t* d_cta_first = reinterpret_cast<const int32_t*>(d_attn_items) + 8 * h->max_attn_items;
-  const AttnMerge* d_merges = reinterpret_cast<const AttnMerge*>(d_cta_first + h->n_sms + 1);
+  const DevIndex dix = dev_index(h);
+  const GatherItem* d_items = dix.items;
 
   if (use_ref && !h->cref) {
     const size_t wide = static_cast<size_t>(std::max(std::max(D.qkv_dim, 2 * D.d_ffn), d));
@@ -945,7 +959,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
                          h->ctx_cap, D.kv_dim, h->rope, s);
     timer.end();
   }
-  ok = ok && (Mi <= 0 || run_layers(h, Mi, dev_index(h), n_attn_ctas, n_merges, overlap_gather, use_ref, timer, s));
+  ok = ok && (Mi <= 0 || run_layers(h, Mi, dix, n_attn_ctas, n_merges, overlap_gather, use_ref, timer, s));
   cudaEventRecord(h->ev_end, s);
   timer.begin(PERCACHE_PH_IO);
   for (int b = 0; b < n_prompts && ok; ++b) {

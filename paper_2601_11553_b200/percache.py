@@ -26,6 +26,7 @@ E_INVAL, E_NOMEM, E_NOSPACE, E_EXISTS, E_LEN_MISMATCH = -1, -2, -3, -4, -5
 E_MISS_NO_INPUT, E_CAPACITY, E_DEVICE_TIMEOUT, E_CUDA, E_NOTFOUND = -6, -7, -8, -9, -10
 FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION, FLAG_EVICT_LFU = 1, 2, 4, 8
 FLAG_SINGLE_CTA_GEMM = 16
+FLAG_NO_SMALL_ROW_KERNELS = 32
 PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",

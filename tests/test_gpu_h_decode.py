@@ -12,7 +12,7 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve):
+def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve, flags=0):
     """prompts_spec: list of (chunk_lens, n_query, hit_idx).  Returns nothing; asserts parity at every step."""
     ws = [wl.small_workload(seed=seed, n_layers=n_layers, chunk_lens=cl, n_query=nq, hit_idx=hi, id_base=100 + 50 * b)
           for b, (cl, nq, hi) in enumerate(prompts_spec)]
@@ -27,7 +27,7 @@ def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve):
                                             for p in prompts], keep_ctx=True, commit=False)
     states = [dec.begin_decode(r) for r in want]
     toks = [wl.make_hidden(seed, (9, j), len(prompts), shape.d_model) for j in range(n_steps)]   # bf16 bits [B, d]
-    with G.make_handle(shape, weights, prompts, decode_reserve=reserve) as h:
+    with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=flags) as h:
         h.set_decode_reserve(reserve)
         G.push_store(h, store, cached)
         got = h.prefill(G.specs_for(prompts, cached))
@@ -72,6 +72,22 @@ def test_decode_crosses_a_context_block_boundary():
 def test_decode_batch_of_ragged_prompts():
     _decode_case(seed=63, n_layers=2, prompts_spec=[([64, 37], 9, [1]), ([300], 17, []), ([16, 16, 16], 1, [0, 1, 2])],
                  n_steps=2, reserve=2)
+
+
+def test_decode_six_prompts():
+    # five to eight rows take the eight-row variant of the weight-streaming kernels
+    spec = [([48], 3 + b, [0] if b % 2 else []) for b in range(6)]
+    _decode_case(seed=65, n_layers=2, prompts_spec=spec, n_steps=2, reserve=2)
+
+
+def test_decode_ten_prompts_uses_the_tensor_core_path():
+    spec = [([32 + 16 * (b % 3)], 2 + b, [0] if b % 3 == 0 else []) for b in range(10)]
+    _decode_case(seed=66, n_layers=2, prompts_spec=spec, n_steps=2, reserve=2)
+
+
+def test_decode_single_prompt_on_the_tensor_core_path():
+    _decode_case(seed=61, n_layers=2, prompts_spec=[([128, 100, 160], 40, [0, 2])], n_steps=2, reserve=2,
+                 flags=pcb.FLAG_NO_SMALL_ROW_KERNELS)
 
 
 def test_decode_needs_the_batch_of_the_last_prefill():
