@@ -32,6 +32,7 @@ struct SmallArgs {
   ResidualEpilogue res;
   SwigluEpilogue swi;
   int32_t gu_blk;            // SwiGLU: gate / up rows are interleaved in blocks of this many rows
+  int32_t k_parts;           // residual kind: pieces a row pair's K range is cut into (K / 8 / k_parts % 32 == 0)
 };
 
 __device__ __forceinline__ void half8_to_float(const uint4& v, float (&f)[8]) {
@@ -83,16 +84,30 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
 
   // ---- stage the input rows (rows >= M are zero)
   if constexpr (NORM) {
-    for (int m = warp; m < MR; m += SM_THREADS / 32) {
-      float ss = 0.f;
-      if (m < M)
-        for (int k = lane * 4; k < K; k += 128) {
-          const float4 v = *reinterpret_cast<const float4*>(a.x_f32 + static_cast<size_t>(m) * K + k);
-          ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
-        }
+    // sum of squares of every row: all threads load at once (one round trip), then warp and block reduction
+    __shared__ float part_ss[SM_THREADS / 32][MR];
+    float ss[MR];
 #pragma unroll
-      for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
-      if (lane == 0) row_scale[m] = rsqrtf(ss / static_cast<float>(K) + a.eps);
+    for (int m = 0; m < MR; ++m) {
+      ss[m] = 0.f;
+      if (m < M)
+        for (int k = tid * 4; k < K; k += SM_THREADS * 4) {
+          const float4 v = *reinterpret_cast<const float4*>(a.x_f32 + static_cast<size_t>(m) * K + k);
+          ss[m] += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < MR; ++m) {
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) ss[m] += __shfl_xor_sync(0xffffffffu, ss[m], o);
+      if (lane == 0) part_ss[warp][m] = ss[m];
+    }
+    __syncthreads();
+    if (tid < MR) {
+      float t = 0.f;
+#pragma unroll
+      for (int w8 = 0; w8 < SM_THREADS / 32; ++w8) t += part_ss[w8][tid];
+      row_scale[tid] = rsqrtf(t / static_cast<float>(K) + a.eps);
     }
     __syncthreads();
     for (int i = tid * 4; i < MR * K; i += SM_THREADS * 4) {
@@ -119,9 +134,14 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
   QkvRow rw{0, 0, -1};
   if (KIND == EPI_QKV && lane < M) rw = load_qkv_row(a.qkv, lane);
 
-  const int n_units = a.N / 2;
+  // Residual kind: N is small (d_model), so a row pair's K range is cut into a.k_parts pieces for as many warps,
+  // which add their partial sums atomically (as the tcgen05 residual GEMM does when it splits K).
+  const int k_parts = KIND == EPI_RESIDUAL ? a.k_parts : 1;
+  const int n_units = (a.N / 2) * k_parts;
+  const int vecs = K / 8 / k_parts;            // 16-byte vectors of a row per part
   const int warps_total = gridDim.x * (SM_THREADS / 32);
-  for (int unit = blockIdx.x * (SM_THREADS / 32) + warp; unit < n_units; unit += warps_total) {
+  for (int wu = blockIdx.x * (SM_THREADS / 32) + warp; wu < n_units; wu += warps_total) {
+    const int unit = wu / k_parts, v_begin = (wu % k_parts) * vecs;
     int r0, r1;
     if (KIND == EPI_QKV) {                 // columns c and c + 64 of head block hb
       r0 = (unit / ROPE_HALF) * HEAD_DIM + unit % ROPE_HALF;
@@ -139,7 +159,7 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
 #pragma unroll
     for (int m = 0; m < MR; ++m) { acc0[m] = 0.f; acc1[m] = 0.f; }
 #pragma unroll 4
-    for (int v = lane; v < K / 8; v += 32) {
+    for (int v = v_begin + lane; v < v_begin + vecs; v += 32) {
       float f0[8], f1[8];
       half8_to_float(__ldg(w0 + v), f0);
       half8_to_float(__ldg(w1 + v), f1);
@@ -171,11 +191,16 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
       } else if (KIND == EPI_SWIGLU) {
         a.swi.act[static_cast<size_t>(lane) * a.swi.ld + unit] = __float2half_rn(silu_f(s0) * s1);
       } else {
-        float2* p = reinterpret_cast<float2*>(a.res.resid + static_cast<size_t>(lane) * a.res.ld + r0);
-        float2 v = *p;
-        v.x += s0;
-        v.y += s1;
-        *p = v;
+        float* p = a.res.resid + static_cast<size_t>(lane) * a.res.ld + r0;
+        if (k_parts > 1) {
+          atomicAdd(p, s0);
+          atomicAdd(p + 1, s1);
+        } else {
+          float2 v = *reinterpret_cast<float2*>(p);
+          v.x += s0;
+          v.y += s1;
+          *reinterpret_cast<float2*>(p) = v;
+        }
       }
     }
   }
@@ -192,7 +217,7 @@ int launch_small_mr(const SmallArgs& a, int n_sms, cudaStream_t s) {
       return -1;
     smem_set = smem;
   }
-  const int units = a.N / 2;
+  const int units = (a.N / 2) * (a.k_parts > 0 ? a.k_parts : 1);
   const int per_sm = smem > 100 * 1024 ? 1 : 2;
   const int blocks = std::min((units + SM_THREADS / 32 - 1) / (SM_THREADS / 32), n_sms * per_sm);
   return launch_pdl(small_gemm_kernel<KIND, MR, NORM>, dim3(blocks), dim3(SM_THREADS), smem, s, a) == cudaSuccess ? 0 : -1;
@@ -214,6 +239,7 @@ int launch_small_gemm(GemmEpilogueKind kind, const void* epilogue, int M, int N,
   if (M > SMALL_GEMM_MAX_ROWS || K % 256 != 0 || N % 2 != 0) return -1;
   SmallArgs a{};
   a.M = M; a.N = N; a.K = K; a.x_f32 = x_f32; a.gain = gain; a.eps = eps; a.a_f16 = a_f16; a.w = w; a.gu_blk = gu_blk;
+  a.k_parts = 1;
   const bool norm = x_f32 != nullptr;
   switch (kind) {
     case EPI_QKV:
@@ -227,6 +253,9 @@ int launch_small_gemm(GemmEpilogueKind kind, const void* epilogue, int M, int N,
     case EPI_RESIDUAL:
       if (norm) return -1;
       a.res = *static_cast<const ResidualEpilogue*>(epilogue);
+      // enough warps to keep every SM streaming (sixteen per SM), pieces of whole 256-element strides
+      a.k_parts = 1;
+      while (a.k_parts < 8 && (N / 2) * a.k_parts < 16 * n_sms && (K / 256) % (2 * a.k_parts) == 0) a.k_parts *= 2;
       return launch_small<EPI_RESIDUAL, false>(a, n_sms, s);
     default:
       return -1;

@@ -102,3 +102,31 @@ def test_decode_needs_the_batch_of_the_last_prefill():
         with pytest.raises(pcb.PerCacheError):           # two rows for a batch of one prompt
             h.decode(np.ascontiguousarray(tok))
         h.decode(np.ascontiguousarray(tok[:1]))
+
+
+def test_decode_after_the_28_layer_workload_at_full_size():
+    """Two decode steps behind the full-depth, 2112-token prompt (three of eight chunks cached), in the launch
+    configuration the benchmark's decode workload times."""
+    w = wl.config1()
+    weights = wl.make_weights(w.shape, w.seed)
+    model = H.oracle_model(w.shape, weights)
+    p = w.prompts[0]
+    lens = dict(zip(p.chunk_ids, p.chunk_len))
+    store = G.oracle_store_alone(model, w.seed, [(c, lens[c]) for c in w.cached_ids])
+    cached = set(w.cached_ids)
+    want = orc.reuse_prefill(model, store, [H.oracle_prompt(p, [i for i, c in enumerate(p.chunk_ids) if c in cached])],
+                             keep_ctx=True, commit=False)[0]
+    st = dec.begin_decode(want)
+    toks = wl.make_hidden(w.seed, (9, 0), 2, w.shape.d_model)
+    with G.make_handle(w.shape, weights, w.prompts, decode_reserve=2) as h:
+        h.set_decode_reserve(2)
+        G.push_store(h, store, w.cached_ids)
+        got = h.prefill(G.specs_for(w.prompts, w.cached_ids))[0]
+        c = G.compare_hidden(got.out_hidden, want.out_hidden)
+        assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
+        for j in range(2):
+            out = h.decode(np.ascontiguousarray(toks[j:j + 1]))
+            ref = dec.decode_step(model, st, orc.bf16_bits_to_f64(toks[j]))
+            c = G.compare_hidden(out[0], ref)
+            print("decode step", j, c)
+            assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, (j, c)
