@@ -220,6 +220,29 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           nv1[it] = p0[4];
         }
       }
+      // EPI_QKV: everything the epilogue needs besides the accumulator depends on the tile alone, so it is
+      // requested while the main loop still runs.  Every lane keeps the index entries of row (row_base + lane);
+      // the four rows a lane stores in a pass (it * 8 + lane / 4) are fetched by shuffle.  The rotation depends on
+      // the column inside a head, not on the head, so the two column groups a warp handles need two sets of table
+      // entries per tile.
+      QkvRow rws[4];
+      RopeCs cs_all[2][4];
+      if constexpr (KIND == EPI_QKV) {
+        const QkvRow mine = load_qkv_row(args.qkv, min(m_idx * BM + quarter * 32 + lane, args.M - 1));
+#pragma unroll
+        for (int it4 = 0; it4 < 4; ++it4) {
+          const int rl = it4 * 8 + (lane >> 2);
+          rws[it4].pos = __shfl_sync(0xffffffffu, mine.pos, rl);
+          rws[it4].slot = __shfl_sync(0xffffffffu, mine.slot, rl);
+          rws[it4].pool_tok = __shfl_sync(0xffffffffu, mine.pool_tok, rl);
+        }
+#pragma unroll
+        for (int p16 = 0; p16 < 2; ++p16)
+#pragma unroll
+          for (int it4 = 0; it4 < 4; ++it4)
+            cs_all[p16][it4] = qkv_load_cs(args.qkv, rws[it4].pos, n_idx * (BN / HEAD_DIM),
+                                           cgroup * 32 + p16 * 16 + (lane & 3) * 4);
+      }
       bool ok = mbar_wait(&tmem_full_bar[acc], acc_phase, args.err_word, DEV_ERR_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
       if (!ok) break;
@@ -305,31 +328,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           });
         }
       } else if constexpr (KIND == EPI_QKV) {
-        // every lane keeps the index entries of row (row_base + lane); the four rows a lane stores in a pass
-        // (it * 8 + lane / 4) are fetched by shuffle once per tile.  The rotation table entries of a pass are
-        // requested before the accumulator is read, so their latency is not paid once per row.
-        const QkvRow mine = load_qkv_row(args.qkv, min(row_base + lane, args.M - 1));
-        QkvRow rws[4];
-#pragma unroll
-        for (int it4 = 0; it4 < 4; ++it4) {
-          const int rl = it4 * 8 + (lane >> 2);
-          rws[it4].pos = __shfl_sync(0xffffffffu, mine.pos, rl);
-          rws[it4].slot = __shfl_sync(0xffffffffu, mine.slot, rl);
-          rws[it4].pool_tok = __shfl_sync(0xffffffffu, mine.pool_tok, rl);
-        }
 #pragma unroll 1
         for (int hl = 0; hl < BN / HEAD_DIM; ++hl) {
           const int hb = n_idx * (BN / HEAD_DIM) + hl;
-#pragma unroll 1
+#pragma unroll
           for (int p16 = 0; p16 < 2; ++p16) {
             const int c0 = cgroup * 32 + p16 * 16;                       // low-half column of this pass
-            RopeCs cs[4];
-#pragma unroll
-            for (int it4 = 0; it4 < 4; ++it4) cs[it4] = qkv_load_cs(args.qkv, rws[it4].pos, hb, c0 + (lane & 3) * 4);
             int it_ctr = 0;
             pass(hl * HEAD_DIM + c0, hl * HEAD_DIM + ROPE_HALF + c0, [&](int rl, int c4, bool valid, float4 lo, float4 hi) {
               const int it4 = it_ctr++;
-              if (valid) qkv_store4_cs(args.qkv, row_base + rl, rws[it4], hb, c0 + c4, lo, hi, cs[it4]);
+              if (valid) qkv_store4_cs(args.qkv, row_base + rl, rws[it4], hb, c0 + c4, lo, hi, cs_all[p16][it4]);
             });
           }
         }
