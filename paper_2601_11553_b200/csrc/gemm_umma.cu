@@ -342,16 +342,50 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           }
         }
       } else {   // EPI_SWIGLU: every 128-column block holds 64 gate columns, then the matching 64 up columns
-#pragma unroll 1
-        for (int hl = 0; hl < BN / 128; ++hl) {
-#pragma unroll 1
-          for (int p16 = 0; p16 < 2; ++p16) {
-            const int c0 = cgroup * 32 + p16 * 16;
-            pass(hl * 128 + c0, hl * 128 + 64 + c0, [&](int rl, int c4, bool valid, float4 g, float4 u) {
-              if (valid) swiglu_store4(args.swi, row_base + rl, (n_idx * (BN / 128) + hl) * 64 + c0 + c4, g, u);
-            });
+        // A thread has gate and up of the same (row, column) in hand as they come from TMEM, so silu(g) * u is
+        // formed and rounded to fp16 first and only the result crosses shared memory: 32 bytes per row instead of
+        // 128 (the staging competes with the MMA's operand reads for shared-memory bandwidth and was the largest
+        // part of this epilogue).
+        // The way through shared memory has a long latency while the MMA is reading operands, so the passes are
+        // software-pipelined over the warp's two staging buffers: pass p is written, then pass p - 1 (written one
+        // step earlier) is read back and stored.
+        constexpr int PITCH = 48;               // 32 bytes of a row + 16: lanes land on distinct 16-byte slots
+        constexpr int N_PASS = 2 * (BN / 128);
+        auto out_col = [&](int p) { return (n_idx * (BN / 128) + (p >> 1)) * 64 + cgroup * 32 + (p & 1) * 16; };
+        auto drain = [&](int p) {               // read pass p back, four lanes per row, and store it
+          const uint8_t* buf = stg + (p & 1) * STG_BUF_BYTES;
+#pragma unroll
+          for (int it = 0; it < 4; ++it) {
+            const int rl = it * 8 + (lane >> 2);
+            const uint2 v = *reinterpret_cast<const uint2*>(buf + rl * PITCH + (lane & 3) * 8);
+            if (row_base + rl < args.M)
+              *reinterpret_cast<uint2*>(args.swi.act + static_cast<size_t>(row_base + rl) * args.swi.ld + out_col(p) +
+                                        (lane & 3) * 4) = v;
+          }
+        };
+#pragma unroll
+        for (int p = 0; p < N_PASS; ++p) {
+          const int c0 = (p >> 1) * 128 + cgroup * 32 + (p & 1) * 16;
+          uint32_t rg[16], ru[16];
+          tmem_ld_32x16(t_acc + c0, rg);
+          tmem_ld_32x16(t_acc + 64 + c0, ru);
+          tmem_wait_ld();
+          uint32_t o[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i)
+            o[i] = pack_half2(silu_f(__uint_as_float(rg[2 * i])) * __uint_as_float(ru[2 * i]),
+                              silu_f(__uint_as_float(rg[2 * i + 1])) * __uint_as_float(ru[2 * i + 1]));
+          uint4* w = reinterpret_cast<uint4*>(stg + (p & 1) * STG_BUF_BYTES + lane * PITCH);
+          w[0] = make_uint4(o[0], o[1], o[2], o[3]);
+          w[1] = make_uint4(o[4], o[5], o[6], o[7]);
+          __syncwarp();                          // pass p is visible to the whole warp
+          if (p > 0) {
+            drain(p - 1);
+            __syncwarp();                        // all lanes have read that buffer before pass p + 1 rewrites it
           }
         }
+        drain(N_PASS - 1);
+        __syncwarp();
       }
       tc_fence_before_sync();
       __syncwarp();
