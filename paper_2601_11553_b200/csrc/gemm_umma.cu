@@ -114,7 +114,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   }
   tc_fence_after_sync();
   const uint32_t tmem_base = tmem_base_slot;
-  pdl_wait();                 // operands and the residual stream come from earlier kernels
+  // The A operand, the index arrays and the residual stream come from earlier kernels: nothing that touches them
+  // runs before pdl_wait().  The weights do not, so the producer thread requests its first B tiles before it waits:
+  // when this CTA starts while the previous kernel still runs on other SMs (programmatic launch), the first
+  // DRAM round trip of the weights is over by the time the dependency resolves.
+  const bool is_producer_thread = warp == 0 && lane == 0;
+  if (!is_producer_thread) pdl_wait();
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -122,22 +127,48 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       int stage = 0;
       uint32_t phase = 0;
       bool ok = true;
+      // rank 0's barrier counts the bytes of both CTAs of a pair; each CTA loads its rows of A and its half of B
+      auto expect = [&](int st) {
+        if constexpr (PAIR) { if (rank == 0) mbar_arrive_expect_tx(&full_bar[st], 2 * Cfg::STAGE_BYTES); }
+        else mbar_arrive_expect_tx(&full_bar[st], Cfg::STAGE_BYTES);
+      };
+      auto load_b = [&](int st, int kb, int n_idx) {
+        uint8_t* b_dst = ring + st * Cfg::STAGE_BYTES + A_STAGE_BYTES;
+        if constexpr (PAIR)
+          tma_load_2d_pair(b_dst, &tmB, mapa_shared(smem_u32(&full_bar[st]), 0), kb * BK,
+                           n_idx * BN + static_cast<int>(rank) * Cfg::B_ROWS);
+        else tma_load_2d(b_dst, &tmB, &full_bar[st], kb * BK, n_idx * BN);
+      };
+      auto load_a = [&](int st, int kb, int m_idx) {
+        uint8_t* a_dst = ring + st * Cfg::STAGE_BYTES;
+        if constexpr (PAIR)
+          tma_load_2d_pair(a_dst, &tmA, mapa_shared(smem_u32(&full_bar[st]), 0), kb * BK,
+                           m_idx * TILE_M + static_cast<int>(rank) * BM);
+        else tma_load_2d(a_dst, &tmA, &full_bar[st], kb * BK, m_idx * BM);
+      };
+      // weights of the first tile's first steps, into the still untouched stages
+      int early = 0;
+      if (worker < n_tiles) {
+        const int n_idx = (worker / k_splits) % n_n_tiles;
+        const int kb0 = kb_begin(worker);
+        early = min(STAGES, kb_end(worker) - kb0);
+        for (int i = 0; i < early; ++i) {
+          expect(i);
+          load_b(i, kb0 + i, n_idx);
+        }
+      }
+      pdl_wait();
       for (int tile = worker; tile < n_tiles && ok; tile += n_workers) {
         const int m_idx = (tile / k_splits) / n_n_tiles, n_idx = (tile / k_splits) % n_n_tiles;
         for (int kb = kb_begin(tile); kb < kb_end(tile); ++kb) {
-          if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
-          uint8_t* a_dst = ring + stage * Cfg::STAGE_BYTES;
-          uint8_t* b_dst = a_dst + A_STAGE_BYTES;
-          if constexpr (PAIR) {
-            // rank 0's barrier counts the bytes of both CTAs; each CTA loads its rows of A and its half of B
-            if (rank == 0) mbar_arrive_expect_tx(&full_bar[stage], 2 * Cfg::STAGE_BYTES);
-            const uint32_t bar0 = mapa_shared(smem_u32(&full_bar[stage]), 0);
-            tma_load_2d_pair(a_dst, &tmA, bar0, kb * BK, m_idx * TILE_M + static_cast<int>(rank) * BM);
-            tma_load_2d_pair(b_dst, &tmB, bar0, kb * BK, n_idx * BN + static_cast<int>(rank) * Cfg::B_ROWS);
+          if (early > 0) {            // this stage's barrier is armed and its B tile is on the way (or there)
+            --early;
+            load_a(stage, kb, m_idx);
           } else {
-            mbar_arrive_expect_tx(&full_bar[stage], Cfg::STAGE_BYTES);
-            tma_load_2d(a_dst, &tmA, &full_bar[stage], kb * BK, m_idx * BM);
-            tma_load_2d(b_dst, &tmB, &full_bar[stage], kb * BK, n_idx * BN);
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
+            expect(stage);
+            load_a(stage, kb, m_idx);
+            load_b(stage, kb, n_idx);
           }
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
