@@ -80,6 +80,26 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int K = a.K, M = a.M;
   pdl_launch_dependents();
+  // The weights do not depend on the previous kernel: every warp asks L2 for the row pair of its first unit before
+  // it waits for that kernel, so the DRAM round trip overlaps the previous kernel's tail.
+  {
+    const int kp = KIND == EPI_RESIDUAL ? a.k_parts : 1;
+    const int wu = blockIdx.x * (SM_THREADS / 32) + warp;
+    if (wu < (a.N / 2) * kp) {
+      const int unit = wu / kp;
+      int r0, r1;
+      if (KIND == EPI_QKV) { r0 = (unit / ROPE_HALF) * HEAD_DIM + unit % ROPE_HALF; r1 = r0 + ROPE_HALF; }
+      else if (KIND == EPI_SWIGLU) { r0 = (2 * (unit / a.gu_blk)) * a.gu_blk + unit % a.gu_blk; r1 = r0 + a.gu_blk; }
+      else { r0 = 2 * unit; r1 = r0 + 1; }
+      const int part_bytes = K * 2 / kp;
+      const char* p0 = reinterpret_cast<const char*>(a.w + static_cast<size_t>(r0) * K) + (wu % kp) * part_bytes;
+      const char* p1 = reinterpret_cast<const char*>(a.w + static_cast<size_t>(r1) * K) + (wu % kp) * part_bytes;
+      for (int off = lane * 128; off < part_bytes; off += 32 * 128) {
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p0 + off));
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p1 + off));
+      }
+    }
+  }
   pdl_wait();
 
   // ---- stage the input rows (rows >= M are zero)
