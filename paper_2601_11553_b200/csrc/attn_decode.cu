@@ -1,0 +1,231 @@
+// Attention of a decode step: one new row per prompt against that prompt's whole assembled context.
+//
+// With a single query row per (prompt, KV head) the work is reading K and V once: 512 bytes per context slot and
+// KV head for 2 * Hq / Hkv * 128 multiply-adds each, so the kernel is bound by HBM and runs on the CUDA cores (a
+// 128-row MMA tile would use one row in 128).  The host cuts every (prompt, KV head) into chunks of context slots,
+// one block per chunk; a block keeps the query heads that share the KV head in registers, streams the chunk's K
+// and V with 16-byte loads (eight lanes per slot, four slots per warp and step), keeps a running maximum, sum and
+// output per slot group (online softmax), folds the groups and warps together, and writes an unnormalised partial
+// result; a second kernel merges the chunks of a (prompt, head).  The row at position p sees slots 0..p.
+#include <algorithm>
+
+#include "kernels.h"
+#include "ptx.cuh"
+
+namespace pc {
+
+namespace {
+
+constexpr int DEC_THREADS = 128;          // 4 warps
+constexpr int DEC_WARPS = DEC_THREADS / 32;
+constexpr int MAX_GROUP = 4;              // query heads per KV head handled by one block
+
+__device__ __forceinline__ void half8_to_f32(const uint4& v, float (&f)[8]) {
+  const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const float2 t = __half22float2(h[i]);
+    f[2 * i] = t.x;
+    f[2 * i + 1] = t.y;
+  }
+}
+
+// partial_o: [item][group][128] fp32; partial_ml: [item][group][2] (reference maximum in log2 units, sum)
+template <int GROUP>
+__global__ void __launch_bounds__(DEC_THREADS)
+decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* __restrict__ q,
+                        const __half* __restrict__ kctx, const __half* __restrict__ vctx, float* __restrict__ partial_o,
+                        float* __restrict__ partial_ml, int n_q_heads, int n_kv_heads, float scale_log2) {
+  __shared__ float sm_o[DEC_WARPS][GROUP][HEAD_DIM];
+  __shared__ float sm_ml[DEC_WARPS][GROUP][2];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int l8 = lane & 7;                  // which 16 of the 128 dimensions this lane holds
+  const int grp = lane >> 3;                // which of the warp's four slots per step
+  pdl_launch_dependents();
+  pdl_wait();
+  const DecodeAttnItem it = items[blockIdx.x];
+  const int kv_dim = n_kv_heads * HEAD_DIM;
+  const int g = it.kv_head;
+  // the query heads of this KV head, 16 dimensions per lane, pre-scaled so that scores come out in log2 units
+  float qv[GROUP][16];
+#pragma unroll
+  for (int h = 0; h < GROUP; ++h) {
+    const __half* qp = q + (static_cast<size_t>(it.row) * n_q_heads + g * GROUP + h) * HEAD_DIM + l8 * 16;
+    float f[8];
+    half8_to_f32(*reinterpret_cast<const uint4*>(qp), f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qv[h][e] = f[e] * scale_log2;
+    half8_to_f32(*reinterpret_cast<const uint4*>(qp + 8), f);
+#pragma unroll
+    for (int e = 0; e < 8; ++e) qv[h][8 + e] = f[e] * scale_log2;
+  }
+  float m[GROUP], l[GROUP], o[GROUP][16];
+#pragma unroll
+  for (int h = 0; h < GROUP; ++h) {
+    m[h] = -INFINITY;
+    l[h] = 0.f;
+#pragma unroll
+    for (int e = 0; e < 16; ++e) o[h][e] = 0.f;
+  }
+  const size_t base = static_cast<size_t>(it.ctx0) * kv_dim + g * HEAD_DIM + l8 * 16;
+  // Loads run three steps ahead of the arithmetic (three register buffers), so that every warp keeps 6 KB in flight.
+  constexpr int STEP = DEC_WARPS * 4;
+  auto fetch = [&](int s0, uint4 (&r)[4]) {
+    const int slot = s0 + grp;
+    if (slot < it.slot_end) {
+      const size_t off = base + static_cast<size_t>(slot) * kv_dim;
+      r[0] = __ldg(reinterpret_cast<const uint4*>(kctx + off));
+      r[1] = __ldg(reinterpret_cast<const uint4*>(kctx + off + 8));
+      r[2] = __ldg(reinterpret_cast<const uint4*>(vctx + off));
+      r[3] = __ldg(reinterpret_cast<const uint4*>(vctx + off + 8));
+    }
+  };
+  auto consume = [&](int s0, const uint4 (&r)[4]) {
+    const bool live = s0 + grp < it.slot_end;
+    float kf[16], vf[16];
+    half8_to_f32(r[0], *reinterpret_cast<float(*)[8]>(&kf[0]));
+    half8_to_f32(r[1], *reinterpret_cast<float(*)[8]>(&kf[8]));
+    half8_to_f32(r[2], *reinterpret_cast<float(*)[8]>(&vf[0]));
+    half8_to_f32(r[3], *reinterpret_cast<float(*)[8]>(&vf[8]));
+#pragma unroll
+    for (int h = 0; h < GROUP; ++h) {
+      float sc = 0.f;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) sc = fmaf(qv[h][e], kf[e], sc);
+      sc += __shfl_xor_sync(0xffffffffu, sc, 1);
+      sc += __shfl_xor_sync(0xffffffffu, sc, 2);
+      sc += __shfl_xor_sync(0xffffffffu, sc, 4);          // all eight lanes of the slot hold its score
+      if (!live) sc = -INFINITY;
+      const float m_new = fmaxf(m[h], sc);
+      if (m_new > -INFINITY) {
+        const float alpha = exp2f(m[h] - m_new);            // 0 when m was -inf
+        const float p = exp2f(sc - m_new);
+        l[h] = l[h] * alpha + p;
+#pragma unroll
+        for (int e = 0; e < 16; ++e) o[h][e] = fmaf(p, live ? vf[e] : 0.f, o[h][e] * alpha);
+        m[h] = m_new;
+      }
+    }
+  };
+  uint4 ra[4] = {}, rb[4] = {}, rc[4] = {};
+  int s0 = it.slot_begin + warp * 4;
+  fetch(s0, ra);
+  fetch(s0 + STEP, rb);
+  fetch(s0 + 2 * STEP, rc);
+  while (s0 < it.slot_end) {
+    {
+      const uint4 c[4] = {ra[0], ra[1], ra[2], ra[3]};
+      fetch(s0 + 3 * STEP, ra);
+      consume(s0, c);
+    }
+    s0 += STEP;
+    if (s0 >= it.slot_end) break;
+    {
+      const uint4 c[4] = {rb[0], rb[1], rb[2], rb[3]};
+      fetch(s0 + 3 * STEP, rb);
+      consume(s0, c);
+    }
+    s0 += STEP;
+    if (s0 >= it.slot_end) break;
+    {
+      const uint4 c[4] = {rc[0], rc[1], rc[2], rc[3]};
+      fetch(s0 + 3 * STEP, rc);
+      consume(s0, c);
+    }
+    s0 += STEP;
+  }
+  // fold the warp's four slot groups (lanes l8, l8 + 8, l8 + 16, l8 + 24 hold the same dimensions)
+#pragma unroll
+  for (int h = 0; h < GROUP; ++h) {
+#pragma unroll
+    for (int x = 8; x <= 16; x <<= 1) {
+      const float m_o = __shfl_xor_sync(0xffffffffu, m[h], x);
+      const float l_o = __shfl_xor_sync(0xffffffffu, l[h], x);
+      const float m_n = fmaxf(m[h], m_o);
+      const float a = m[h] > -INFINITY ? exp2f(m[h] - m_n) : 0.f;
+      const float b = m_o > -INFINITY ? exp2f(m_o - m_n) : 0.f;
+#pragma unroll
+      for (int e = 0; e < 16; ++e) {
+        const float o_o = __shfl_xor_sync(0xffffffffu, o[h][e], x);
+        o[h][e] = o[h][e] * a + o_o * b;
+      }
+      l[h] = l[h] * a + l_o * b;
+      m[h] = m_n;
+    }
+    if (grp == 0) {
+#pragma unroll
+      for (int e = 0; e < 16; ++e) sm_o[warp][h][l8 * 16 + e] = o[h][e];
+      if (l8 == 0) { sm_ml[warp][h][0] = m[h]; sm_ml[warp][h][1] = l[h]; }
+    }
+  }
+  __syncthreads();
+  // fold the warps: thread d owns dimension d
+  const int d = threadIdx.x;
+#pragma unroll
+  for (int h = 0; h < GROUP; ++h) {
+    float M = -INFINITY;
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) M = fmaxf(M, sm_ml[w][h][0]);
+    float acc = 0.f, L = 0.f;
+#pragma unroll
+    for (int w = 0; w < DEC_WARPS; ++w) {
+      const float wgt = sm_ml[w][h][0] > -INFINITY ? exp2f(sm_ml[w][h][0] - M) : 0.f;
+      acc = fmaf(wgt, sm_o[w][h][d], acc);
+      L = fmaf(wgt, sm_ml[w][h][1], L);
+    }
+    const size_t slot = static_cast<size_t>(it.partial_slot) * GROUP + h;
+    partial_o[slot * HEAD_DIM + d] = acc;
+    if (d == 0) { partial_ml[slot * 2] = M; partial_ml[slot * 2 + 1] = L; }
+  }
+}
+
+// out[row][head][:] = sum_c w_c O_c / sum_c w_c l_c over the chunks of (row, KV head), w_c = 2^(m_c - max m).
+template <int GROUP>
+__global__ void __launch_bounds__(HEAD_DIM)
+decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
+                    const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const DecodeAttnMerge mg = merges[blockIdx.x];
+  const int h = blockIdx.y, d = threadIdx.x;
+  float M = -INFINITY;
+  for (int c = 0; c < mg.n_parts; ++c) M = fmaxf(M, partial_ml[(static_cast<size_t>(mg.partial_slot0 + c) * GROUP + h) * 2]);
+  float acc = 0.f, L = 0.f;
+  for (int c = 0; c < mg.n_parts; ++c) {
+    const size_t slot = static_cast<size_t>(mg.partial_slot0 + c) * GROUP + h;
+    const float mc = partial_ml[slot * 2];
+    const float wgt = mc > -INFINITY ? exp2f(mc - M) : 0.f;
+    acc = fmaf(wgt, partial_o[slot * HEAD_DIM + d], acc);
+    L = fmaf(wgt, partial_ml[slot * 2 + 1], L);
+  }
+  out[(static_cast<size_t>(mg.row) * n_q_heads + mg.kv_head * GROUP + h) * HEAD_DIM + d] = __float2half_rn(acc / L);
+}
+
+}  // namespace
+
+int launch_decode_attention(const DecodeAttnItem* items, int n_items, const DecodeAttnMerge* merges, int n_merges,
+                            const __half* q, const __half* kctx_layer, const __half* vctx_layer, float* partial_o,
+                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s) {
+  if (n_items <= 0) return 0;
+  const int group = n_q_heads / n_kv_heads;
+  const float scale_log2 = 1.4426950408889634f * 0.08838834764831845f;      // log2(e) / sqrt(128)
+  cudaError_t rc;
+  if (group == 2) {
+    rc = launch_pdl(decode_attention_kernel<2>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer, vctx_layer,
+                    partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
+    if (rc == cudaSuccess)
+      rc = launch_pdl(decode_merge_kernel<2>, dim3(n_merges, 2), dim3(HEAD_DIM), 0, s, merges, partial_o, partial_ml, out,
+                      n_q_heads);
+  } else if (group == 4) {
+    rc = launch_pdl(decode_attention_kernel<4>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer, vctx_layer,
+                    partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
+    if (rc == cudaSuccess)
+      rc = launch_pdl(decode_merge_kernel<4>, dim3(n_merges, 4), dim3(HEAD_DIM), 0, s, merges, partial_o, partial_ml, out,
+                      n_q_heads);
+  } else {
+    return -1;
+  }
+  return rc == cudaSuccess ? 0 : -1;
+}
+
+}  // namespace pc

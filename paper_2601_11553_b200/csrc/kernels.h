@@ -54,6 +54,26 @@ struct AttnMerge {
   int32_t pad0, pad1, pad2;
 };
 
+// Decode-step attention (attn_decode.cu): one block per (row, KV head, chunk of context slots).
+struct DecodeAttnItem {
+  int32_t row;           // new row (= prompt index in a decode step)
+  int32_t ctx0;          // global context slot of the prompt's slot 0
+  int32_t slot_begin;    // first slot of the chunk (slot inside the prompt)
+  int32_t slot_end;      // one past its last slot (at most position + 1)
+  int32_t kv_head;
+  int32_t partial_slot;  // where the chunk's unnormalised result goes
+  int32_t pad0, pad1;
+};
+struct DecodeAttnMerge {   // the chunks of one (row, KV head) are in slots partial_slot0 .. + n_parts - 1
+  int32_t row, kv_head, partial_slot0, n_parts;
+  int32_t pad0, pad1, pad2, pad3;
+};
+// partial_o: fp32 [items][query heads per KV head][128]; partial_ml: fp32 [items][query heads per KV head][2].
+// Query heads per KV head must be 2 or 4.
+int launch_decode_attention(const DecodeAttnItem* items, int n_items, const DecodeAttnMerge* merges, int n_merges,
+                            const __half* q, const __half* kctx_layer, const __half* vctx_layer, float* partial_o,
+                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
+
 // A tile before scheduling: its rows and the number of 128-slot context blocks its last row can see.
 struct AttnBaseTile { int32_t row0, n_rows, ctx0, n_blocks; };
 // Deals (tile, unit, block range) items to at most n_sms CTAs (attn_plan.cu).  cta_first gets one entry per

@@ -248,8 +248,9 @@ DevIndex dev_index(const percache* h) {
 // Every decoder block for the Mi rows in h->resid (prefill: the new rows of the batch; decode: one row per
 // prompt): RMSNorm, QKV projection (rotation, pages, context), attention over the assembled context, output
 // projection, RMSNorm, SwiGLU FFN.  Layer l's attention first waits for ev_gather[l] when the fetch runs beside.
+// n_decode_items > 0: the attention work is a decode step's list of DecodeAttnItem / DecodeAttnMerge records.
 bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_merges, bool overlap_gather,
-                bool use_ref, PhaseTimer& timer, cudaStream_t s) {
+                bool use_ref, PhaseTimer& timer, cudaStream_t s, int n_decode_items = 0) {
   const ModelDims& D = h->dims;
   const int d = D.d_model;
   const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
@@ -304,6 +305,11 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     if (overlap_gather) ok = ok && cudaStreamWaitEvent(s, h->ev_gather[l], 0) == cudaSuccess;
     if (use_ref || (h->flags & PERCACHE_FLAG_REFERENCE_ATTENTION)) {
       launch_ref_attention(h->qbuf, qe.kctx, qe.vctx, h->attn_out, d_row_pos, d_row_ctx0, Mi, D.n_q_heads, D.n_kv_heads, s);
+    } else if (n_decode_items > 0) {
+      ok = ok && launch_decode_attention(reinterpret_cast<const DecodeAttnItem*>(d_attn_items), n_decode_items,
+                                         reinterpret_cast<const DecodeAttnMerge*>(d_merges), n_merges, h->qbuf, qe.kctx,
+                                         qe.vctx, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads,
+                                         s) == 0;
     } else {
       ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
                                        h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s) == 0;
@@ -452,7 +458,8 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   const size_t units_per_tile = static_cast<size_t>(D.n_kv_heads) * (D.n_q_heads / D.n_kv_heads / 2);
   h->partial_slots = 2 * h->n_sms + 2;
   h->max_attn_items = max_tiles * units_per_tile + 2 * static_cast<size_t>(h->n_sms);
-  h->max_attn_merges = static_cast<size_t>(h->n_sms) + 1;
+  h->max_attn_merges = std::max(static_cast<size_t>(h->n_sms) + 1,      // prefill: at most one cut unit per CTA
+                                static_cast<size_t>(cfg->max_batch_prompts) * D.n_kv_heads);   // decode: (prompt, KV head)
   h->index_ints = 4 * static_cast<size_t>(h->m_cap) + 4 * static_cast<size_t>(h->ctx_cap) + 8 * h->max_attn_items +
                   static_cast<size_t>(h->n_sms) + 1 + 8 * h->max_attn_merges;
   ok = ok && dev_alloc(h, &h->partial_o, static_cast<size_t>(h->partial_slots) * 2 * 128 * HEAD_DIM);
@@ -1039,20 +1046,58 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
     base_tiles.push_back(AttnBaseTile{b, 1, plan.ctx0[b], (T + 1 + 127) / 128});
     visible_pairs += T + 1;
   }
-  std::vector<AttnItem> v_items;
-  std::vector<int32_t> v_first;
-  std::vector<AttnMerge> v_merges;
-  plan_attention(base_tiles, D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2), h->n_sms, h->partial_slots, &v_items,
-                 &v_first, &v_merges);
-  if (v_items.size() > h->max_attn_items || v_merges.size() > h->max_attn_merges ||
-      v_first.size() > static_cast<size_t>(h->n_sms) + 1)
-    return PERCACHE_E_CAPACITY;
-  std::copy(v_items.begin(), v_items.end(), attn_items);
-  std::fill(cta_first, cta_first + h->n_sms + 1, static_cast<int32_t>(v_items.size()));
-  std::copy(v_first.begin(), v_first.end(), cta_first);
-  std::copy(v_merges.begin(), v_merges.end(), merges);
-  const int n_attn_ctas = static_cast<int>(v_first.size()) - 1;
-  const int n_merges = static_cast<int>(v_merges.size());
+  // One query row per prompt: the attention is a matter of reading every prompt's K and V once, which the
+  // weight-streaming style kernel of attn_decode.cu does on the CUDA cores; (prompt, KV head) pairs are cut into
+  // chunks of context slots so that a few hundred blocks per SM-full are in flight.
+  const int group = D.n_q_heads / D.n_kv_heads;
+  const bool stream_attention = !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION |
+                                              PERCACHE_FLAG_NO_SMALL_ROW_KERNELS)) && (group == 2 || group == 4);
+  int n_attn_ctas = 0, n_merges = 0, n_decode_items = 0;
+  if (stream_attention) {
+    int64_t total_slots = 0;
+    for (int b = 0; b < n_prompts; ++b) total_slots += row_pos[b] + 1;
+    int chunk = static_cast<int>(std::min<int64_t>(1024, std::max<int64_t>(64, (total_slots * D.n_kv_heads / (4 * h->n_sms) + 63) / 64 * 64)));
+    const size_t scratch_items = static_cast<size_t>(h->partial_slots) * 2 * 128 * HEAD_DIM / (static_cast<size_t>(group) * HEAD_DIM);
+    auto count_items = [&](int ch) {
+      int64_t n = 0;
+      for (int b = 0; b < n_prompts; ++b) n += static_cast<int64_t>((row_pos[b] + 1 + ch - 1) / ch) * D.n_kv_heads;
+      return n;
+    };
+    while (static_cast<size_t>(count_items(chunk)) > std::min(h->max_attn_items, scratch_items)) chunk *= 2;
+    if (static_cast<size_t>(n_prompts) * D.n_kv_heads > h->max_attn_merges) return PERCACHE_E_CAPACITY;
+    DecodeAttnItem* ditems = reinterpret_cast<DecodeAttnItem*>(attn_items);
+    DecodeAttnMerge* dmerges = reinterpret_cast<DecodeAttnMerge*>(merges);
+    // Items are ordered (prompt, chunk, KV head): the blocks of the KV heads of one chunk run side by side and
+    // together read whole 2 KB context rows, which keeps DRAM pages open; the results of a (prompt, KV head) still
+    // go to consecutive slots for the merge.
+    int next_slot = 0;
+    for (int b = 0; b < n_prompts; ++b) {
+      const int n_slots = row_pos[b] + 1;
+      const int n_chunks = (n_slots + chunk - 1) / chunk;
+      for (int g = 0; g < D.n_kv_heads; ++g)
+        dmerges[n_merges++] = DecodeAttnMerge{b, g, next_slot + g * n_chunks, n_chunks, 0, 0, 0, 0};
+      for (int c = 0; c < n_chunks; ++c)
+        for (int g = 0; g < D.n_kv_heads; ++g)
+          ditems[n_decode_items++] = DecodeAttnItem{b, plan.ctx0[b], c * chunk, std::min(n_slots, (c + 1) * chunk), g,
+                                                    next_slot + g * n_chunks + c, 0, 0};
+      next_slot += n_chunks * D.n_kv_heads;
+    }
+  } else {
+    std::vector<AttnItem> v_items;
+    std::vector<int32_t> v_first;
+    std::vector<AttnMerge> v_merges;
+    plan_attention(base_tiles, D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2), h->n_sms, h->partial_slots, &v_items,
+                   &v_first, &v_merges);
+    if (v_items.size() > h->max_attn_items || v_merges.size() > h->max_attn_merges ||
+        v_first.size() > static_cast<size_t>(h->n_sms) + 1)
+      return PERCACHE_E_CAPACITY;
+    std::copy(v_items.begin(), v_items.end(), attn_items);
+    std::fill(cta_first, cta_first + h->n_sms + 1, static_cast<int32_t>(v_items.size()));
+    std::copy(v_first.begin(), v_first.end(), cta_first);
+    std::copy(v_merges.begin(), v_merges.end(), merges);
+    n_attn_ctas = static_cast<int>(v_first.size()) - 1;
+    n_merges = static_cast<int>(v_merges.size());
+  }
   const double plan_us =
       std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
 
@@ -1076,7 +1121,7 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   cudaEventRecord(h->ev_begin, s);
   launch_bf16_to_f32(h->xin, h->resid, static_cast<int64_t>(n_prompts) * d, s);
   timer.end();
-  ok = ok && run_layers(h, n_prompts, dev_index(h), n_attn_ctas, n_merges, false, use_ref, timer, s);
+  ok = ok && run_layers(h, n_prompts, dev_index(h), n_attn_ctas, n_merges, false, use_ref, timer, s, n_decode_items);
   cudaEventRecord(h->ev_end, s);
   timer.begin(PERCACHE_PH_IO);
   ok = ok && cudaMemcpyAsync(out_hidden, h->resid, static_cast<size_t>(n_prompts) * d * sizeof(float),
