@@ -537,10 +537,10 @@ int umma_gemm_block_n(GemmEpilogueKind kind) {
 // a 128 x 256 x 64 step (48 KB) about 768; a CTA pair on a 256 x 256 tile loads 32 KB per CTA and step and its
 // step costs about 600 clocks.  A work item also pays about three steps of ramp-up and tail.  The cost of a
 // choice is (rounds of items over the workers) x (steps per item + 3) x (clocks per step).
-// Measured on B200 (M = 33 024, d = 1024): pairs raise the two residual GEMMs from 990 to 1183 TFLOP/s (K = 2048)
-// and from 1059 to 1280 (K = 3072); the QKV and gate/up GEMMs (K = 1024, rotation / SwiGLU epilogues) are
-// bound by their epilogues at 128 x 256 per CTA either way and lose a few percent to the pair's
-// synchronisation, so callers allow pairs for the residual epilogue only.
+// Measured on B200 (M = 33 024, d = 1024), single CTAs -> pairs: O-projection 990 -> 1183 TFLOP/s (K = 2048), down-
+// projection 1059 -> 1280 (K = 3072), and, once their epilogues had been shortened, QKV 1103 -> 1149 and gate/up
+// 1269 -> 1392 (K = 1024); at M = 2176, d = 2048: QKV 886 -> 966, gate/up 1037 -> 1213.  At M = 1344 pairs made the
+// whole step 0.8 % slower (three runs each), hence the thresholds below.
 void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
                           int* k_splits, int* pair) {
   const int n_kb = K / BK;
@@ -556,8 +556,9 @@ void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool
     const int workers = pr ? n_sms / 2 : n_sms;
     const int64_t clocks = shape == 0 ? 512 : (shape == 1 ? 768 : 600);
     const int64_t tiles = static_cast<int64_t>((M + tile_m - 1) / tile_m) * (N / bn);
-    // small problems (under half a round of pair tiles) are bound by ramp-up and tail, which pairs lengthen
-    if (pr && tiles * 2 < workers) continue;
+    // small problems are bound by ramp-up and tail, which pairs lengthen: the residual GEMMs (long K) take pairs
+    // from half a round of pair tiles, the others (K = d_model, epilogue-heavy) from one and a half rounds
+    if (pr && tiles * 2 < (may_split_k ? 1 : 3) * workers) continue;
     for (int sp = 1; sp <= (may_split_k ? 8 : 1); ++sp) {
       if (sp > 1 && n_kb / sp < 4) break;
       const int64_t rounds = (tiles * sp + workers - 1) / workers;

@@ -255,7 +255,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   const int d = D.d_model;
   const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * D.kv_dim;
-  // CTA pairs pay off where the main loop is the bound: the two residual GEMMs (see umma_gemm_pick_shape)
+  // CTA pairs: chosen per GEMM by size (see umma_gemm_pick_shape)
   const bool may_pair = !(h->flags & PERCACHE_FLAG_SINGLE_CTA_GEMM);
   const int32_t *d_row_slot = ix.row_slot, *d_row_pos = ix.row_pos, *d_row_pool = ix.row_pool, *d_row_ctx0 = ix.row_ctx0;
   const AttnItem* d_attn_items = ix.attn_items;
@@ -294,7 +294,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     } else {
       {
         int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, false, &bn, &ks, &pr);
+        umma_gemm_pick_shape(Mi, D.qkv_dim, d, h->n_sms, false, may_pair, &bn, &ks, &pr);
         ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wqkv256 : W.m_wqkv, Mi, D.qkv_dim, d, bn, EPI_QKV, &qe, nullptr,
                                     h->d_err, h->n_sms, s, ks, pr) == 0;
       }
@@ -352,7 +352,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     } else {
       {
         int bn, ks, pr;
-        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, false, &bn, &ks, &pr);
+        umma_gemm_pick_shape(Mi, 2 * D.d_ffn, d, h->n_sms, false, may_pair, &bn, &ks, &pr);
         ok = ok && launch_umma_gemm(h->m_xn, (bn == 256 && !pr) ? W.m_wgu256 : W.m_wgu, Mi, 2 * D.d_ffn, d, bn, EPI_SWIGLU, &se, nullptr,
                                     h->d_err, h->n_sms, s, ks, pr) == 0;
       }
