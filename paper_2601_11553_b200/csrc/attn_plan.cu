@@ -19,10 +19,10 @@ namespace pc {
 namespace {
 // costs in quarter blocks (one block = the two heads' work on 128 context slots)
 constexpr int64_t BLOCK_COST = 4;
-constexpr int64_t ITEM_COST = 6;        // Q load, pipeline fill, output rows
+constexpr int64_t ITEM_COST = 12;       // Q load, pipeline fill, output rows (measured: 6 and 16 are both slower)
 constexpr int64_t PARTIAL_COST = 2;     // fp32 partial output instead of fp16 rows
 constexpr int64_t MERGE_COST = 16;      // the merge kernel behind the attention kernel
-constexpr int MIN_PART = 2;             // blocks; shorter parts are not worth an item
+constexpr int MIN_PART = 3;             // blocks; shorter parts are not worth an item
 }  // namespace
 
 int64_t plan_attention(const std::vector<AttnBaseTile>& tiles, int units_per_tile, int n_sms, int max_partial_slots,

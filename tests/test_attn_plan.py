@@ -30,7 +30,7 @@ def check_plan(n_blocks, units, n_ctas=148, max_slots=298):
             s = [p[2] for p in parts]
             assert s == list(range(s[0], s[0] + len(parts))) and s[0] >= 0
             slots_seen += s
-            assert all(p[1] - p[0] >= 2 for p in parts)   # no part shorter than two blocks
+            assert all(p[1] - p[0] >= 3 for p in parts)   # no part shorter than three blocks
     assert split_units == n_split
     assert sorted(slots_seen) == list(range(len(slots_seen))) and len(slots_seen) <= max_slots
     load = np.zeros(max(ctas_used, 1), dtype=np.int64)
