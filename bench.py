@@ -179,6 +179,22 @@ def run_reference(args):
         "gpu_launches": 0}))
 
 
+# --------------------------------------------------------------------------- replicas
+def max_over_ranks(values, dist, device):
+    """Every rank runs an independent replica; the job's time is the slowest rank's (max over ranks of each value)."""
+    if dist is None:
+        return [float(v) for v in values]
+    import torch
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def aggregate_tokens_per_s(world: int, tokens_per_step: int, steps: int, total_ms: float) -> float:
+    """Whole-job throughput of `world` replicas that each did `steps` steps within total_ms (the slowest rank's)."""
+    return world * tokens_per_step * steps / (total_ms / 1000.0)
+
+
 # --------------------------------------------------------------------------- GPU leg
 def run_gpu(args):
     import torch
@@ -291,18 +307,15 @@ def run_gpu(args):
     ms_e2e, _, _, _, _ = timed(specs_host, out_host, args.steps)
     barrier()
     e2e_ms = float(sum(ms_e2e))
-    if dist is not None:
-        t = torch.tensor([total_ms, e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
     if rank != 0:
         return
 
     peaks = load_peaks()
     tokens = w.total_tokens
     new_rows = int(st["new_rows"])
-    value = world * tokens * args.steps / (total_ms / 1000.0)
-    e2e_value = world * tokens * args.steps / (e2e_ms / 1000.0)
+    value = aggregate_tokens_per_s(world, tokens, args.steps, total_ms)
+    e2e_value = aggregate_tokens_per_s(world, tokens, args.steps, e2e_ms)
     fl = flops_per_step(w, new_rows, int(st["attn_visible_pairs"]))
     gather_bytes = int(st["hit_tokens"]) * shape.n_layers * shape.kv_dim * 2 * 2 * 2
     per_phase = {}

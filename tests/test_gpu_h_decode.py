@@ -12,9 +12,10 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve, flags=0):
+def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve, flags=0, **model_kw):
     """prompts_spec: list of (chunk_lens, n_query, hit_idx).  Returns nothing; asserts parity at every step."""
-    ws = [wl.small_workload(seed=seed, n_layers=n_layers, chunk_lens=cl, n_query=nq, hit_idx=hi, id_base=100 + 50 * b)
+    ws = [wl.small_workload(seed=seed, n_layers=n_layers, chunk_lens=cl, n_query=nq, hit_idx=hi, id_base=100 + 50 * b,
+                            **model_kw)
           for b, (cl, nq, hi) in enumerate(prompts_spec)]
     shape = ws[0].shape
     weights = wl.make_weights(shape, seed)
@@ -88,6 +89,12 @@ def test_decode_ten_prompts_uses_the_tensor_core_path():
 def test_decode_single_prompt_on_the_tensor_core_path():
     _decode_case(seed=61, n_layers=2, prompts_spec=[([128, 100, 160], 40, [0, 2])], n_steps=2, reserve=2,
                  flags=pcb.FLAG_NO_SMALL_ROW_KERNELS)
+
+
+def test_decode_four_query_heads_per_kv_head():
+    # two head pairs per KV head in the prefill attention, the four-head variant of the decode attention
+    _decode_case(seed=67, n_layers=2, prompts_spec=[([200, 90], 21, [0]), ([130], 7, [])], n_steps=2, reserve=2,
+                 n_q_heads=8, n_kv_heads=2, d_model=512)
 
 
 def test_decode_needs_the_batch_of_the_last_prefill():
