@@ -18,7 +18,6 @@ namespace {
 
 constexpr int DEC_THREADS = 128;          // 4 warps
 constexpr int DEC_WARPS = DEC_THREADS / 32;
-constexpr int MAX_GROUP = 4;              // query heads per KV head handled by one block
 
 __device__ __forceinline__ void half8_to_f32(const uint4& v, float (&f)[8]) {
   const __half2* h = reinterpret_cast<const __half2*>(&v);

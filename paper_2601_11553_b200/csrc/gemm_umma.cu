@@ -569,12 +569,6 @@ void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool
     }
   }
 }
-int umma_gemm_pick_block_n(int M, int N, int n_sms) {
-  int bn, sp, pr;
-  umma_gemm_pick_shape(M, N, 64 * 16, n_sms, false, false, &bn, &sp, &pr);
-  return bn;
-}
-
 template <int BN, bool PAIR>
 static int launch_bn(const GemmOperand& A, const GemmOperand& B, GemmArgs& args, GemmEpilogueKind kind,
                      const void* epilogue, int n_sms, cudaStream_t s) {

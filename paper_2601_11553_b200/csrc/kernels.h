@@ -139,7 +139,6 @@ int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, i
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
                      cudaStream_t s, int k_splits = 1, int pair = 0);
 int umma_gemm_block_n(GemmEpilogueKind kind);    // narrowest N tile (a B operand map needs box_rows = the tile used)
-int umma_gemm_pick_block_n(int M, int N, int n_sms);   // 128 or 256 for this problem
 // tile width, number of K parts (parts > 1 only if may_split_k: the residual epilogue then adds atomically) and
 // whether CTA pairs are used (only if may_pair)
 void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
