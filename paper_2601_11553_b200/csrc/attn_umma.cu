@@ -75,6 +75,17 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint8_t* k_smem = base + 2 * TILE_BYTES;                  // [stages][2 halves][128][64]
   uint8_t* v_smem = k_smem + KV_STAGES * TILE_BYTES;
 
+  // The work list and the row positions are written by the host before the first kernel of the call, not by the
+  // kernel this one depends on: they are read ahead of the dependency wait, while the prologue runs.
+  const int w_begin = args.cta_first[blockIdx.x], w_end = args.cta_first[blockIdx.x + 1];
+  AttnItem first_item{};
+  if (w_begin < w_end) first_item = args.items[w_begin];
+  int first_pos = 0;
+  if (warp < 8 && w_begin < w_end) {
+    const int r = (warp & 3) * 32 + lane;
+    first_pos = args.row_pos[first_item.row0 + (r < first_item.n_rows ? r : first_item.n_rows - 1)];
+  }
+
   if (threadIdx.x == 0) {
     mbar_init(&q_full, 1);
     mbar_init(&q_empty, 1);
@@ -103,7 +114,6 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   const int group = args.n_q_heads / args.n_kv_heads;      // query heads per KV head (even)
   // An item's `unit` = g * pairs + pair covers query heads (g * group + 2 * pair, +1) and KV head g.
   const int pairs = group / 2;
-  const int w_begin = args.cta_first[blockIdx.x], w_end = args.cta_first[blockIdx.x + 1];
 
   if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
@@ -111,7 +121,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       uint32_t unit_it = 0, kvit = 0;
       bool ok = true;
       for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
-        const AttnItem t = args.items[w];
+        const AttnItem t = w == w_begin ? first_item : args.items[w];
         const int gp = t.unit;
         const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
         const int nb = t.blk_end - t.blk_begin;
@@ -161,7 +171,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         umma_commit(&s_full[i]);
       };
       for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
-        const AttnItem t = args.items[w];
+        const AttnItem t = w == w_begin ? first_item : args.items[w];
         const int nb = t.blk_end - t.blk_begin;
         const uint32_t kv0 = kvit;
         if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
@@ -214,14 +224,14 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     uint32_t unit_it = 0, kvit = 0;
     bool ok = true;
     for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
-      const AttnItem t = args.items[w];
+      const AttnItem t = w == w_begin ? first_item : args.items[w];
       const int gp = t.unit;
       const int head = (gp / pairs) * group + 2 * (gp % pairs) + i;
       const int nb = t.blk_end - t.blk_begin;
       const uint32_t kv0 = kvit;
       const bool valid = r_in_tile < t.n_rows;
       const int row = t.row0 + (valid ? r_in_tile : t.n_rows - 1);
-      const int pos = args.row_pos[row];
+      const int pos = w == w_begin ? first_pos : args.row_pos[row];
       float m = -INFINITY, l = 0.f;
       for (int j = 0; j < nb; ++j) {
         const uint32_t kvidx = kv0 + j;
@@ -385,8 +395,8 @@ __global__ void __launch_bounds__(MERGE_WARPS * 32)
 attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
                        const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads, int n_kv_heads) {
   pdl_launch_dependents();
+  const AttnMerge mg = merges[blockIdx.x];      // host-written before the call's first kernel: read ahead of the wait
   pdl_wait();
-  const AttnMerge mg = merges[blockIdx.x];
   const int group = n_q_heads / n_kv_heads, pairs = group / 2;
   const int i = blockIdx.y;
   const int head = (mg.unit / pairs) * group + 2 * (mg.unit % pairs) + i;
