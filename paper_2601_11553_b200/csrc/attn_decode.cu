@@ -41,8 +41,8 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
   const int l8 = lane & 7;                  // which 16 of the 128 dimensions this lane holds
   const int grp = lane >> 3;                // which of the warp's four slots per step
   pdl_launch_dependents();
+  const DecodeAttnItem it = items[blockIdx.x];     // host-written before the step's first kernel: read ahead of the wait
   pdl_wait();
-  const DecodeAttnItem it = items[blockIdx.x];
   const int kv_dim = n_kv_heads * HEAD_DIM;
   const int g = it.kv_head;
   // the query heads of this KV head, 16 dimensions per lane, pre-scaled so that scores come out in log2 units
@@ -184,8 +184,8 @@ __global__ void __launch_bounds__(HEAD_DIM)
 decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
                     const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads) {
   pdl_launch_dependents();
+  const DecodeAttnMerge mg = merges[blockIdx.x];   // host-written, as above
   pdl_wait();
-  const DecodeAttnMerge mg = merges[blockIdx.x];
   const int h = blockIdx.y, d = threadIdx.x;
   float M = -INFINITY;
   for (int c = 0; c < mg.n_parts; ++c) M = fmaxf(M, partial_ml[(static_cast<size_t>(mg.partial_slot0 + c) * GROUP + h) * 2]);

@@ -76,12 +76,19 @@ template <int VPL>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
                                                       __half* __restrict__ out, int M, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int lane = threadIdx.x & 31;
+  const int nv = d >> 2;
   pdl_launch_dependents();
+  // the gain is a weight: it is requested before the wait for the kernel that writes x
+  float4 g[VPL];
+#pragma unroll
+  for (int k = 0; k < VPL; ++k) {
+    const int i = lane + 32 * k;
+    g[k] = i < nv ? __ldg(reinterpret_cast<const float4*>(gain) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+  }
   pdl_wait();
   if (row >= M) return;
-  const int lane = threadIdx.x & 31;
   const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
-  const int nv = d >> 2;
   float4 v[VPL];
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
@@ -94,15 +101,13 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, o);
   const float inv = rsqrtf(ss / static_cast<float>(d) + eps);
-  const float4* g4 = reinterpret_cast<const float4*>(gain);
   uint2* o2 = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
     const int i = lane + 32 * k;
     if (i < nv) {
-      const float4 g = __ldg(g4 + i);
-      __half2 a = __floats2half2_rn(v[k].x * inv * g.x, v[k].y * inv * g.y);
-      __half2 b = __floats2half2_rn(v[k].z * inv * g.z, v[k].w * inv * g.w);
+      __half2 a = __floats2half2_rn(v[k].x * inv * g[k].x, v[k].y * inv * g[k].y);
+      __half2 b = __floats2half2_rn(v[k].z * inv * g[k].z, v[k].w * inv * g[k].w);
       o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
     }
   }
