@@ -32,8 +32,8 @@ __device__ __forceinline__ void half8_to_f32(const uint4& v, float (&f)[8]) {
 // partial_o: [item][group][128] fp32; partial_ml: [item][group][2] (reference maximum in log2 units, sum)
 template <int GROUP>
 __global__ void __launch_bounds__(DEC_THREADS)
-decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* __restrict__ q,
-                        const __half* __restrict__ kctx, const __half* __restrict__ vctx, float* __restrict__ partial_o,
+decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* q, const __half* kctx,
+                        const __half* vctx, float* __restrict__ partial_o,
                         float* __restrict__ partial_ml, int n_q_heads, int n_kv_heads, float scale_log2) {
   __shared__ float sm_o[DEC_WARPS][GROUP][HEAD_DIM];
   __shared__ float sm_ml[DEC_WARPS][GROUP][2];
@@ -51,10 +51,10 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
   for (int h = 0; h < GROUP; ++h) {
     const __half* qp = q + (static_cast<size_t>(it.row) * n_q_heads + g * GROUP + h) * HEAD_DIM + l8 * 16;
     float f[8];
-    half8_to_f32(*reinterpret_cast<const uint4*>(qp), f);
+    half8_to_f32(ld_dep_v4(qp), f);
 #pragma unroll
     for (int e = 0; e < 8; ++e) qv[h][e] = f[e] * scale_log2;
-    half8_to_f32(*reinterpret_cast<const uint4*>(qp + 8), f);
+    half8_to_f32(ld_dep_v4(qp + 8), f);
 #pragma unroll
     for (int e = 0; e < 8; ++e) qv[h][8 + e] = f[e] * scale_log2;
   }
@@ -73,10 +73,10 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
     const int slot = s0 + grp;
     if (slot < it.slot_end) {
       const size_t off = base + static_cast<size_t>(slot) * kv_dim;
-      r[0] = __ldg(reinterpret_cast<const uint4*>(kctx + off));
-      r[1] = __ldg(reinterpret_cast<const uint4*>(kctx + off + 8));
-      r[2] = __ldg(reinterpret_cast<const uint4*>(vctx + off));
-      r[3] = __ldg(reinterpret_cast<const uint4*>(vctx + off + 8));
+      r[0] = ld_dep_v4(kctx + off);          // the newest slot was written by the kernel before this one
+      r[1] = ld_dep_v4(kctx + off + 8);
+      r[2] = ld_dep_v4(vctx + off);
+      r[3] = ld_dep_v4(vctx + off + 8);
     }
   };
   auto consume = [&](int s0, const uint4 (&r)[4]) {
@@ -181,21 +181,40 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
 // out[row][head][:] = sum_c w_c O_c / sum_c w_c l_c over the chunks of (row, KV head), w_c = 2^(m_c - max m).
 template <int GROUP>
 __global__ void __launch_bounds__(HEAD_DIM)
-decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
-                    const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads) {
+decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* partial_o, const float* partial_ml,
+                    __half* __restrict__ out, int n_q_heads) {
   pdl_launch_dependents();
   const DecodeAttnMerge mg = merges[blockIdx.x];   // host-written, as above
   pdl_wait();
   const int h = blockIdx.y, d = threadIdx.x;
+  // eight parts at a time, all their loads issued before the first is used (a part index past the end repeats the
+  // last part and gets weight zero)
+  constexpr int U = 8;
+  auto slot_of = [&](int c) { return static_cast<size_t>(mg.partial_slot0 + min(c, mg.n_parts - 1)) * GROUP + h; };
   float M = -INFINITY;
-  for (int c = 0; c < mg.n_parts; ++c) M = fmaxf(M, partial_ml[(static_cast<size_t>(mg.partial_slot0 + c) * GROUP + h) * 2]);
+  for (int c0 = 0; c0 < mg.n_parts; c0 += U) {
+    float mv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) mv[u] = ld_dep_f32(partial_ml + slot_of(c0 + u) * 2);
+#pragma unroll
+    for (int u = 0; u < U; ++u) M = fmaxf(M, mv[u]);
+  }
   float acc = 0.f, L = 0.f;
-  for (int c = 0; c < mg.n_parts; ++c) {
-    const size_t slot = static_cast<size_t>(mg.partial_slot0 + c) * GROUP + h;
-    const float mc = partial_ml[slot * 2];
-    const float wgt = mc > -INFINITY ? exp2f(mc - M) : 0.f;
-    acc = fmaf(wgt, partial_o[slot * HEAD_DIM + d], acc);
-    L = fmaf(wgt, partial_ml[slot * 2 + 1], L);
+  for (int c0 = 0; c0 < mg.n_parts; c0 += U) {
+    float mv[U], ov[U], lv[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const size_t slot = slot_of(c0 + u);
+      mv[u] = ld_dep_f32(partial_ml + slot * 2);
+      lv[u] = ld_dep_f32(partial_ml + slot * 2 + 1);
+      ov[u] = ld_dep_f32(partial_o + slot * HEAD_DIM + d);
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const float wgt = (c0 + u < mg.n_parts && mv[u] > -INFINITY) ? exp2f(mv[u] - M) : 0.f;
+      acc = fmaf(wgt, ov[u], acc);
+      L = fmaf(wgt, lv[u], L);
+    }
   }
   out[(static_cast<size_t>(mg.row) * n_q_heads + mg.kv_head * GROUP + h) * HEAD_DIM + d] = __float2half_rn(acc / L);
 }

@@ -392,8 +392,8 @@ namespace {
 constexpr int MERGE_WARPS = 8;
 constexpr int MERGE_ROWS = 2;
 __global__ void __launch_bounds__(MERGE_WARPS * 32)
-attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __restrict__ partial_o,
-                       const float* __restrict__ partial_ml, __half* __restrict__ out, int n_q_heads, int n_kv_heads) {
+attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* partial_o, const float* partial_ml,
+                       __half* __restrict__ out, int n_q_heads, int n_kv_heads) {
   pdl_launch_dependents();
   const AttnMerge mg = merges[blockIdx.x];      // host-written before the call's first kernel: read ahead of the wait
   pdl_wait();
@@ -410,7 +410,7 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __rest
   for (int k = 0; k < MERGE_ROWS; ++k) {
     const int r = min(r0 + k, mg.n_rows - 1);
     float2 ml = make_float2(-INFINITY, 0.f);
-    if (lane < mg.n_parts) ml = *reinterpret_cast<const float2*>(partial_ml + ((slot0 + 2 * lane) * BLK + r) * 2);
+    if (lane < mg.n_parts) ml = ld_dep_f32x2(partial_ml + ((slot0 + 2 * lane) * BLK + r) * 2);
     float M = ml.y > 0.f ? ml.x : -INFINITY;
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) M = fmaxf(M, __shfl_xor_sync(0xffffffffu, M, o));
@@ -429,7 +429,7 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* __rest
 #pragma unroll
       for (int q = 0; q < 4; ++q) {
         const int sp = min(s0 + q, mg.n_parts - 1);       // a repeated part gets weight zero below
-        o[k][q] = __ldg(reinterpret_cast<const float4*>(partial_o + ((slot0 + 2 * sp) * BLK + r) * HEAD_DIM + lane * 4));
+        o[k][q] = ld_dep_f32x4(partial_o + ((slot0 + 2 * sp) * BLK + r) * HEAD_DIM + lane * 4);
       }
     }
 #pragma unroll

@@ -73,7 +73,7 @@ void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStr
 // The row stays in registers between the two passes (VPL float4 per lane, d <= 128 * VPL); all loads of a row
 // are issued before the first is used.
 template <int VPL>
-__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+__global__ void __launch_bounds__(256) rmsnorm_kernel(const float* x, const float* __restrict__ gain,
                                                       __half* __restrict__ out, int M, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
@@ -93,7 +93,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
     const int i = lane + 32 * k;
-    v[k] = i < nv ? xr[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+    v[k] = i < nv ? ld_dep_f32x4(xr + i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
   float ss = 0.f;
 #pragma unroll
@@ -113,7 +113,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* __restrict__ 
   }
 }
 // Rows of any length: two passes over global memory.
-__global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* __restrict__ x, const float* __restrict__ gain,
+__global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* x, const float* __restrict__ gain,
                                                            __half* __restrict__ out, int M, int d, float eps) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   pdl_launch_dependents();
@@ -124,7 +124,7 @@ __global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* __restri
   const int nv = d >> 2;
   float ss = 0.f;
   for (int i = lane; i < nv; i += 32) {
-    const float4 v = xr[i];
+    const float4 v = ld_dep_f32x4(xr + i);
     ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
   }
 #pragma unroll
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* __restri
   const float4* g4 = reinterpret_cast<const float4*>(gain);
   uint2* o2 = reinterpret_cast<uint2*>(out + static_cast<size_t>(row) * d);
   for (int i = lane; i < nv; i += 32) {
-    const float4 v = xr[i];
+    const float4 v = ld_dep_f32x4(xr + i);
     const float4 g = g4[i];
     __half2 a = __floats2half2_rn(v.x * inv * g.x, v.y * inv * g.y);
     __half2 b = __floats2half2_rn(v.z * inv * g.z, v.w * inv * g.w);
