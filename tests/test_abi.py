@@ -70,3 +70,21 @@ def test_no_cpu_fallback(lib):
     with pytest.raises(pcb.PerCacheError) as e:
         pcb.debug_gemm(a, a, use_reference=True)
     assert e.value.code == pcb.E_CUDA
+
+
+def test_dependent_data_is_not_read_through_read_only_loads():
+    """Kernels run beside their producer (programmatic launch), so what the producer writes must not be read with
+    __ldg or through a const __restrict__ pointer: such a load may be scheduled above griddepcontrol.wait.  The
+    buffers that are written by one kernel of a step and read by the next are checked by name."""
+    src_dir = os.path.join(os.path.dirname(pcb.__file__), "csrc")
+    produced = ["partial_o", "partial_ml", "kctx", "vctx", "attn_out", "resid", "qbuf"]
+    for name in ("attn_umma.cu", "attn_decode.cu", "gemm_small.cu", "gemm_umma.cu"):
+        text = open(os.path.join(src_dir, name)).read()
+        for buf in produced:
+            assert not re.search(r"__ldg\([^;]*\b%s\b" % buf, text), (name, buf)
+            assert not re.search(r"const\s+\w+\s*\*\s*__restrict__\s+%s\b" % buf, text), (name, buf)
+    norm = open(os.path.join(src_dir, "kernels_mem.cu")).read()
+    for kernel in ("rmsnorm_kernel", "rmsnorm_long_kernel"):
+        sig = norm[norm.index("%s(" % kernel):]
+        sig = sig[:sig.index(")")]
+        assert "__restrict__ x" not in sig, kernel
