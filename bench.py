@@ -1,12 +1,15 @@
 #!/usr/bin/env python
 """Benchmark of reuse-prefill on B200: one step = one percache_prefill call of the workload.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg1] [--impl reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg4_50] [--impl reference] [--no-table]
 
 Prints ONE JSON line.  `value` is context tokens per second (prompt tokens served / time) with inputs
 resident in HBM; `e2e` is the same through host buffers (pinned input hidden states copied in, output
 rows copied out inside the timed call).  Between steps the chunks the call stored are dropped again
-(host-only bookkeeping, untimed) so that every step sees the same cache state.
+(host-only bookkeeping, untimed) so that every step sees the same cache state.  The line is about the named
+workload (default: the long context with half of its chunks cached); at one GPU its key `workloads` also holds one
+compact record for each of the other workloads (time per step, tokens/s, per-kernel-class throughput and fraction
+of the measured peak, clocks, and the oracle's extrapolated throughput on the host).
 
 With N > 1 every rank runs an independent replica of the workload on its own GPU (the path does not
 shard: no collective), and the aggregate is N x tokens / slowest rank.
@@ -32,6 +35,8 @@ from paper_2601_11553_b200 import workloads as wl
 
 METRIC = "reuse_prefill_tokens_per_s"
 UNIT = "tokens/s"
+DEFAULT_WORKLOAD = "cfg4_50"      # the largest single-GPU workload that uses both halves of the method
+TABLE_WORKLOADS = ("cfg0", "cfg1", "cfg2", "cfg3", "cfg4_100", "cfg4_90", "cfg4_50", "cfg4_0")
 
 
 def load_peaks():
@@ -119,20 +124,28 @@ def flops_per_step(w: wl.Workload, new_rows: int, visible_pairs: int):
 
 
 # --------------------------------------------------------------------------- CPU oracle leg
+def _oracle_cores():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
+    except Exception:
+        return os.cpu_count() or 1
+
+
+def _oracle_model(shape, weights):
+    from oracle import reuse_prefill as orc
+    return orc.Model(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                     n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn,
+                     rope_theta=shape.rope_theta, rms_eps=shape.rms_eps, layers=weights)
+
+
 def oracle_sample(w: wl.Workload, n_layers_sample: int):
     """Time the oracle on the first `n_layers_sample` layers of the workload's model (all rows, same prompts)."""
     from oracle import reuse_prefill as orc
-    try:
-        from threadpoolctl import threadpool_info
-        cores = max([p.get("num_threads", 1) for p in threadpool_info()] or [1])
-    except Exception:
-        cores = os.cpu_count() or 1
+    cores = _oracle_cores()
     shape = wl.ModelShape(n_layers=n_layers_sample, **{k: getattr(w.shape, k) for k in
                                                        ("d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn")})
-    weights = wl.make_weights(shape, w.seed)
-    model = orc.Model(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
-                      n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn,
-                      rope_theta=shape.rope_theta, rms_eps=shape.rms_eps, layers=weights)
+    model = _oracle_model(shape, wl.make_weights(shape, w.seed))
     store = orc.Store()
     ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
     for c in w.cached_ids:     # cached content: seeded integer values (timing does not depend on them)
@@ -155,20 +168,111 @@ def oracle_sample(w: wl.Workload, n_layers_sample: int):
     return step, cores
 
 
+class OracleBlockSample:
+    """The oracle on a bounded sample of a large workload: block 0 of the model through oracle.block_rows, which
+    forms K and V for every new row of a prompt (they are the block's context) and the rest of the block for a few
+    sampled rows.  Timed at two sample sizes; the time is linear in the number of sampled rows, so the line through
+    the two points gives the time of the block for all rows, and the depth multiplies it.  For a batch only every
+    `prompt_stride`-th prompt is timed.  Cached K/V are zeros here (their values do not change the time)."""
+
+    def __init__(self, w: wl.Workload, rows=(32, 288), max_prompts: int = 8):
+        from oracle import reuse_prefill as orc
+        self.orc, self.w, self.rows = orc, w, rows
+        shape1 = wl.ModelShape(n_layers=1, **{k: getattr(w.shape, k) for k in
+                                              ("d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn")})
+        self.model = _oracle_model(shape1, wl.make_weights(shape1, w.seed))
+        self.cores = _oracle_cores()
+        cached = set(w.cached_ids)
+        stride = max(1, -(-len(w.prompts) // max_prompts))
+        self.stride = stride
+        self.cases = []
+        hkv, hd = w.shape.n_kv_heads, w.shape.head_dim
+        for p in w.prompts[::stride]:
+            new, segs, xs, start = [], [], [], 0
+            for i, (c, n) in enumerate(zip(p.chunk_ids, p.chunk_len)):
+                if c in cached:
+                    z = np.zeros((n, hkv, hd))
+                    segs.append((start, z, z))
+                else:
+                    new.append(np.arange(start, start + n))
+                    xs.append(orc.bf16_bits_to_f64(p.chunk_hidden[i]))
+                start += n
+            new.append(np.arange(start, start + p.n_query))
+            xs.append(orc.bf16_bits_to_f64(p.query_hidden))
+            self.cases.append((np.concatenate(xs), np.concatenate(new), start + p.n_query, segs))
+        self.m_sampled = sum(c[0].shape[0] for c in self.cases)
+        self.slope = None
+
+    def _time(self, n_rows: int) -> float:
+        t0 = time.perf_counter()
+        for x, new, T, segs in self.cases:
+            m = x.shape[0]
+            rows = np.unique(np.linspace(0, m - 1, min(n_rows, m)).astype(np.int64))
+            self.orc.block_rows(self.model, 0, x, new, T, segs, rows)
+        return time.perf_counter() - t0
+
+    def step(self) -> float:
+        """One bounded sample; returns the extrapolated seconds of one whole step of the workload."""
+        if self.slope is None:
+            self._time(self.rows[0])    # untimed first pass: pages in the weights and the BLAS threads
+        t_small = self._time(self.rows[0])
+        if self.slope is None:          # seconds per sampled row and case, measured once
+            t_big = self._time(self.rows[1])
+            self.slope = max(0.0, (t_big - t_small) / (self.rows[1] - self.rows[0]) / len(self.cases))
+        per_case_rows = [c[0].shape[0] for c in self.cases]
+        full_block = t_small + self.slope * sum(max(0, m - min(self.rows[0], m)) for m in per_case_rows)
+        return full_block * (self.w.new_rows() / max(self.m_sampled, 1)) * self.w.shape.n_layers
+
+    def describe(self, t_step: float) -> str:
+        return (f"block 0 of {self.w.shape.n_layers} of {self.w.name} via oracle.block_rows: K/V of all new rows of "
+                f"{len(self.cases)} of {len(self.w.prompts)} prompts + {self.rows[0]} (and once {self.rows[1]}) sampled "
+                f"rows each; linear in rows -> all {self.w.new_rows()} new rows, x {self.w.shape.n_layers} blocks: "
+                f"EXTRAPOLATED to {t_step:.0f} s per step")
+
+
+def cpu_baseline_for(w: wl.Workload):
+    """Oracle tokens/s on the host for workload w: a whole run where it takes seconds, else the bounded block sample."""
+    tokens = w.total_tokens
+    if w.new_rows() * w.shape.n_layers <= 3000:            # cfg0-sized: the whole call
+        step, cores = oracle_sample(w, w.shape.n_layers)
+        t = step()
+        return {"value": tokens / t, "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"the whole {w.name} call ({t:.2f} s)", "extrapolated": False}
+    if w.new_rows() <= 1500 and len(w.prompts) == 1:       # cfg1-sized: a few layers of the real call
+        n_sample = max(1, min(w.shape.n_layers, 4))
+        step, cores = oracle_sample(w, n_sample)
+        t = step()
+        scale = w.shape.n_layers / n_sample
+        return {"value": tokens / (t * scale), "unit": UNIT, "cores": cores, "kind": "oracle",
+                "sample": f"first {n_sample} of {w.shape.n_layers} layers of {w.name}, all new rows, one call "
+                          f"({t:.1f} s), time x {scale:g}", "extrapolated": True}
+    smp = OracleBlockSample(w)
+    t = smp.step()
+    return {"value": tokens / t, "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": smp.describe(t),
+            "extrapolated": True}
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     w = wl.by_name(args.workload)
-    n_sample = 1
-    step, cores = oracle_sample(w, n_sample)
+    big = not (w.new_rows() <= 1500 and len(w.prompts) == 1)
+    if big:
+        smp = OracleBlockSample(w)
+        step = smp.step
+        cores = smp.cores
+    else:
+        n_sample = 1
+        raw, cores = oracle_sample(w, n_sample)
+        step = lambda: raw() * (w.shape.n_layers / n_sample)
     for _ in range(min(args.warmup, 1)):
         step()
     times = [step() for _ in range(args.steps)]
-    scale = w.shape.n_layers / n_sample
-    ms = 1000.0 * float(np.mean(times)) * scale
+    ms = 1000.0 * float(np.mean(times))
     value = w.total_tokens / (ms / 1000.0)
-    sample = f"layer 0 of {w.shape.n_layers} of {w.name} (all prompts, all new rows), time x {scale:g}"
+    sample = smp.describe(ms / 1000.0) if big else \
+        f"layer 0 of {w.shape.n_layers} of {w.name} (all prompts, all new rows), time x {w.shape.n_layers:g}"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -195,7 +299,197 @@ def aggregate_tokens_per_s(world: int, tokens_per_step: int, steps: int, total_m
     return world * tokens_per_step * steps / (total_ms / 1000.0)
 
 
+def replica_launch_command(args, port: int):
+    """The command that starts one rank per GPU of this node when bench.py itself is asked for N > 1 GPUs without a
+    launcher around it (no WORLD_SIZE in the environment)."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)]
+    return cmd + list(args.forward)
+
+
 # --------------------------------------------------------------------------- GPU leg
+KERNEL_OF = {"attn": "umma_attention_kernel", "gather": "gather_rerope_kernel"}
+
+
+def pick_peak(peaks, timed_s: float, reasons):
+    """The tensor-core denominator for a run: the sustained figure when the timed region lasts seconds or the power
+    cap was active while it ran, else the burst figure."""
+    if timed_s >= 1.0 or "sw_power_cap" in reasons:
+        return peaks["tflops_sustained"], "sustained"
+    return peaks["tflops_burst"], "burst"
+
+
+class Bench:
+    """One model on one GPU and the workloads that run on it."""
+
+    def __init__(self, shape, seed, workloads, local, torch, pcb):
+        self.torch, self.pcb = torch, pcb
+        self.dev = torch.device("cuda", local)
+        self.local = local
+        self.shape = shape
+        self.stream = torch.cuda.current_stream(self.dev)
+        weights_np = wl.make_weights(shape, seed)
+        weights = [{k: torch.from_numpy(v.view(np.int16)).to(self.dev).view(torch.bfloat16) for k, v in lw.items()}
+                   for lw in weights_np]
+        ids_lens = {}
+        for w in workloads:
+            ids_lens.update({c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)})
+        self.ids_lens = ids_lens
+        max_tokens = max(w.total_tokens for w in workloads)
+        self.h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                              n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
+                              pool_pages=sum((l + 15) // 16 for l in ids_lens.values()) + 64,
+                              max_prompt_tokens=max(p.n_total for w in workloads for p in w.prompts),
+                              max_batch_prompts=max(len(w.prompts) for w in workloads),
+                              max_batch_ctx_tokens=max_tokens, max_batch_new_rows=max_tokens, device=local,
+                              stream=self.stream.cuda_stream)
+
+    def close(self):
+        self.h.close()
+
+    def set_cache_state(self, w: wl.Workload):
+        """Exactly w.cached_ids of the workload's chunks are stored: missing ones are produced (a prefill of the chunk
+        alone through the library itself, or the seeded integer pool), others of the workload are dropped."""
+        h, pcb = self.h, self.pcb
+        cached = set(w.cached_ids)
+        for c in w.cached_ids:
+            if h.has_chunk(c) is not None:
+                continue
+            if w.cache_source == "integer_pool":
+                h.put_chunk_synthetic(c, self.ids_lens[c], w.seed)
+            else:
+                hid = wl.chunk_hidden_for(w.seed, c, self.ids_lens[c], self.shape.d_model)
+                h.prefill([pcb.PromptSpec([c], [self.ids_lens[c]], [hid], None, 0)])
+        for p in w.prompts:
+            for c in p.chunk_ids:
+                if c not in cached and h.has_chunk(c) is not None:
+                    h.drop_chunk(c)
+
+    def measure(self, w: wl.Workload, steps: int, warmup: int, flags: int, full: bool, barrier, dist):
+        """Times the workload.  full: also the end-to-end pass through host buffers."""
+        torch, pcb, h, dev, stream, shape = self.torch, self.pcb, self.h, self.dev, self.stream, self.shape
+        self.set_cache_state(w)
+        cached = set(w.cached_ids)
+        missed = sorted({c for p in w.prompts for c in p.chunk_ids if c not in cached})
+
+        def to_dev(a):
+            return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+        def to_pinned(a):
+            return torch.from_numpy(a.view(np.int16)).pin_memory().view(torch.bfloat16)
+
+        def specs(conv):
+            out = []
+            for p in w.prompts:
+                hid = [None if c in cached else conv(hh) for c, hh in zip(p.chunk_ids, p.chunk_hidden)] \
+                    if p.chunk_hidden else None
+                out.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, conv(p.query_hidden), p.n_query))
+            return out
+
+        n_new = [p.n_query + sum(l for c, l in zip(p.chunk_ids, p.chunk_len) if c not in cached) for p in w.prompts]
+        specs_dev = specs(to_dev)
+        out_dev = [torch.empty((n, shape.d_model), dtype=torch.float32, device=dev) for n in n_new]
+
+        def timed(spec_list, outs, n):
+            ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+            phases = {k: 0.0 for k in pcb.PHASES}
+            launches = {k: 0 for k in pcb.PHASES}
+            dev_us, st = 0.0, None
+            for i in range(n):
+                ev[i][0].record(stream)
+                h.prefill(spec_list, out=outs)
+                ev[i][1].record(stream)
+                st = h.stats()
+                dev_us += st["device_us"]
+                for k in pcb.PHASES:
+                    phases[k] += st["phase_us"][k]
+                    launches[k] += st["phase_launches"][k]
+                for c in missed:           # host-only bookkeeping, untimed: every step starts from the same cache state
+                    h.drop_chunk(c)
+            torch.cuda.synchronize(dev)
+            return [a.elapsed_time(b) for a, b in ev], phases, launches, dev_us, st
+
+        h.set_flags(flags)
+        timed(specs_dev, out_dev, max(warmup, 3))
+        sampler = ClockSampler(self.local)
+        barrier()
+        sampler.start()
+        ms, _, launches, dev_us, st = timed(specs_dev, out_dev, steps)
+        barrier()
+        clocks = sampler.stop()
+        total_ms = float(sum(ms))
+        # the same steps with CUDA events around every kernel class (a separate pass: the events cost a few per cent)
+        h.set_flags(flags | pcb.FLAG_PHASE_TIMING)
+        timed(specs_dev, out_dev, 2)
+        ph_steps = steps if full else max(2, min(steps, 5))
+        ms_ph, phases, launches_ph, _, _ = timed(specs_dev, out_dev, ph_steps)
+        h.set_flags(flags)
+        e2e_ms = None
+        if full:     # end to end: pinned host hidden states in, host rows out, inside the timed call
+            specs_host = specs(to_pinned)
+            out_host = [torch.empty((n, shape.d_model), dtype=torch.float32).pin_memory() for n in n_new]
+            timed(specs_host, out_host, 3)
+            barrier()
+            ms_e2e, _, _, _, _ = timed(specs_host, out_host, steps)
+            barrier()
+            e2e_ms = float(sum(ms_e2e))
+        vals = max_over_ranks([total_ms] + ([e2e_ms] if full else []), dist, dev)
+        total_ms = vals[0]
+        if full:
+            e2e_ms = vals[1]
+
+        peaks = load_peaks()
+        new_rows = int(st["new_rows"])
+        fl = flops_per_step(w, new_rows, int(st["attn_visible_pairs"]))
+        gather_bytes = int(st["hit_tokens"]) * shape.n_layers * shape.kv_dim * 2 * 2 * 2
+        tensor_peak, which_peak = pick_peak(peaks, total_ms / 1000.0, clocks["reasons"])
+        weight_bytes_layer = shape.params_per_layer * 2
+        per_phase = {}
+        for k in ("qkv", "attn", "oproj", "gateup", "down"):
+            n = launches_ph[k]
+            if n:
+                us = phases[k] / n
+                tf = fl[k] / shape.n_layers / us / 1e6
+                per_phase[k] = {"us_per_launch": us, "launches_per_step": n // ph_steps, "tflops": tf,
+                                "frac_of_tensor_peak": tf / tensor_peak}
+        if launches_ph["gather"]:
+            us = phases["gather"] / launches_ph["gather"]
+            gbs = gather_bytes / us / 1e3
+            per_phase["gather"] = {"us_per_launch": us, "launches_per_step": 1, "gbs": gbs,
+                                   "frac_of_hbm_peak": gbs / peaks["hbm_gbs"]}
+        if launches_ph["norm"]:
+            per_phase["norm"] = {"us_per_launch": phases["norm"] / launches_ph["norm"],
+                                 "launches_per_step": launches_ph["norm"] // ph_steps}
+        return {"w": w, "ms": ms, "total_ms": total_ms, "e2e_ms": e2e_ms, "clocks": clocks, "st": st, "phases": phases,
+                "launches": launches, "launches_ph": launches_ph, "per_phase": per_phase, "fl": fl, "dev_us": dev_us,
+                "gather_bytes": gather_bytes, "new_rows": new_rows, "tensor_peak": tensor_peak, "which_peak": which_peak,
+                "peaks": peaks, "ms_ph": ms_ph, "ph_steps": ph_steps, "weight_bytes_layer": weight_bytes_layer}
+
+
+def table_row(r, world, steps):
+    """Compact record of one workload for the per-workload table."""
+    w = r["w"]
+    row = {"workload": w.name, "ms_per_step": r["total_ms"] / steps,
+           "tokens_per_s": aggregate_tokens_per_s(world, w.total_tokens, steps, r["total_ms"]),
+           "new_rows": r["new_rows"], "hit_tokens": int(r["st"]["hit_tokens"]), "steps": steps,
+           "tensor_peak": {"tflops": r["tensor_peak"], "which": r["which_peak"]},
+           "clocks": {k: r["clocks"][k] for k in ("sm_mhz", "sm_max_mhz", "reasons")}, "kernels": {}}
+    for k, v in r["per_phase"].items():
+        if "tflops" in v:
+            row["kernels"][k] = {"tflops": round(v["tflops"], 1), "frac": round(v["frac_of_tensor_peak"], 3)}
+        elif "gbs" in v:
+            row["kernels"][k] = {"gbs": round(v["gbs"], 1), "frac": round(v["frac_of_hbm_peak"], 3)}
+    # whole step against the roofline of its algorithmic work: tensor flops, or weight + gather bytes when the call has
+    # too few rows to reach the tensor roof (the ridge is ~210 flops per byte)
+    flops = sum(r["fl"].values())
+    t_s = r["total_ms"] / steps / 1000.0
+    row["step_tflops"] = flops / t_s / 1e12
+    row["step_frac_of_tensor_peak"] = row["step_tflops"] / r["tensor_peak"]
+    hbm_bytes = r["weight_bytes_layer"] * w.shape.n_layers + r["gather_bytes"]
+    row["step_hbm_floor_ms"] = hbm_bytes / r["peaks"]["hbm_gbs"] / 1e6
+    return row
+
+
 def run_gpu(args):
     import torch
     from paper_2601_11553_b200 import percache as pcb
@@ -213,170 +507,94 @@ def run_gpu(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     dev = torch.device("cuda", local)
 
-    w = wl.by_name(args.workload)
-    shape = w.shape
-    weights_np = wl.make_weights(shape, w.seed)
-    weights = [{k: torch.from_numpy(v.view(np.int16)).to(dev).view(torch.bfloat16) for k, v in lw.items()}
-               for lw in weights_np]
-    ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
-    pool_pages = sum((l + 15) // 16 for l in ids_lens.values()) + 64
-    stream = torch.cuda.current_stream(dev)
-    h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
-                     n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
-                     pool_pages=pool_pages, max_prompt_tokens=max(p.n_total for p in w.prompts),
-                     max_batch_prompts=len(w.prompts), max_batch_ctx_tokens=w.total_tokens,
-                     max_batch_new_rows=w.total_tokens, device=local, stream=stream.cuda_stream)
-    del weights
-    # ---- cache state before every step
-    cached = set(w.cached_ids)
-    if w.cache_source == "integer_pool":
-        for c in w.cached_ids:
-            h.put_chunk_synthetic(c, ids_lens[c], w.seed)
-    else:   # prefill every cached chunk alone through the library itself
-        for c in w.cached_ids:
-            hid = wl.chunk_hidden_for(w.seed, c, ids_lens[c], shape.d_model)
-            h.prefill([pcb.PromptSpec([c], [ids_lens[c]], [hid], None, 0)])
-    missed = sorted({c for p in w.prompts for c in p.chunk_ids if c not in cached})
-
-    def to_dev(a):
-        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
-
-    def to_pinned(a):
-        return torch.from_numpy(a.view(np.int16)).pin_memory().view(torch.bfloat16)
-
-    def specs(conv):
-        out = []
-        for p in w.prompts:
-            hid = [None if c in cached else conv(hh) for c, hh in zip(p.chunk_ids, p.chunk_hidden)] \
-                if p.chunk_hidden else None
-            out.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, conv(p.query_hidden), p.n_query))
-        return out
-
-    specs_dev, specs_host = specs(to_dev), specs(to_pinned)
-    n_new = [p.n_query + sum(l for c, l in zip(p.chunk_ids, p.chunk_len) if c not in cached) for p in w.prompts]
-    out_dev = [torch.empty((n, shape.d_model), dtype=torch.float32, device=dev) for n in n_new]
-    out_host = [torch.empty((n, shape.d_model), dtype=torch.float32).pin_memory() for n in n_new]
-
-    def restore():
-        for c in missed:
-            h.drop_chunk(c)
-
-    def timed(spec_list, outs, steps, collect_phases=False):
-        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
-        phases = {k: 0.0 for k in pcb.PHASES}
-        launches = {k: 0 for k in pcb.PHASES}
-        dev_us = 0.0
-        for i in range(steps):
-            ev[i][0].record(stream)
-            h.prefill(spec_list, out=outs)
-            ev[i][1].record(stream)
-            st = h.stats()
-            dev_us += st["device_us"]
-            for k in pcb.PHASES:
-                phases[k] += st["phase_us"][k]
-                launches[k] += st["phase_launches"][k]
-            restore()
-        torch.cuda.synchronize(dev)
-        ms = [a.elapsed_time(b) for a, b in ev]
-        return ms, phases, launches, dev_us, st
-
     def barrier():
         torch.cuda.synchronize(dev)
         if dist is not None:
             dist.barrier()
         torch.cuda.synchronize(dev)
 
-    # ---- warm-up, then the timed region (device-resident inputs), max over ranks
-    h.set_flags(args.flags)
-    timed(specs_dev, out_dev, max(args.warmup, 3))
-    sampler = ClockSampler(local)
-    barrier()
-    sampler.start()
-    ms, _, launches, dev_us, st = timed(specs_dev, out_dev, args.steps)
-    barrier()
-    clocks = sampler.stop()
-    total_ms = float(sum(ms))
-    # ---- same steps with per-kernel-class events (separate pass: the extra events cost a few percent)
-    h.set_flags(args.flags | pcb.FLAG_PHASE_TIMING)
-    timed(specs_dev, out_dev, 2)
-    ms_ph, phases, launches_ph, _, _ = timed(specs_dev, out_dev, args.steps)
-    h.set_flags(args.flags)
-    # ---- end to end through host buffers
-    timed(specs_host, out_host, 3)
-    barrier()
-    ms_e2e, _, _, _, _ = timed(specs_host, out_host, args.steps)
-    barrier()
-    e2e_ms = float(sum(ms_e2e))
-    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], dist, dev)
+    main_w = wl.by_name(args.workload)
+    # Workloads that share the main one's model run on the same handle (the long-context sweep: one model, four hit
+    # rates with nested hit sets, run from the fullest cache to the emptiest); the others get a handle each.
+    table_names = [] if (args.no_table or world > 1) else [n for n in TABLE_WORKLOADS if n != main_w.name]
+    groups = {}
+    for name in [main_w.name] + table_names:
+        w = main_w if name == main_w.name else wl.by_name(name)
+        groups.setdefault((w.seed, w.shape), []).append(w)
+    rows, main = [], None
+    for (seed, shape), ws in groups.items():
+        ws.sort(key=lambda w: -len(w.cached_ids))
+        b = Bench(shape, seed, ws, local, torch, pcb)
+        for w in ws:
+            is_main = w.name == main_w.name
+            steps = args.steps if is_main else max(3, min(args.steps, 10))
+            r = b.measure(w, steps, args.warmup, args.flags, is_main, barrier, dist)
+            if is_main:
+                main = r
+            elif rank == 0:
+                row = table_row(r, world, steps)
+                if not args.no_cpu_baseline:
+                    row["cpu_baseline"] = cpu_baseline_for(w)
+                rows.append(row)
+        b.close()
+        del b
+        torch.cuda.empty_cache()
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
     if rank != 0:
         return
 
-    peaks = load_peaks()
-    tokens = w.total_tokens
-    new_rows = int(st["new_rows"])
-    value = aggregate_tokens_per_s(world, tokens, args.steps, total_ms)
-    e2e_value = aggregate_tokens_per_s(world, tokens, args.steps, e2e_ms)
-    fl = flops_per_step(w, new_rows, int(st["attn_visible_pairs"]))
-    gather_bytes = int(st["hit_tokens"]) * shape.n_layers * shape.kv_dim * 2 * 2 * 2
-    per_phase = {}
-    for k in ("qkv", "attn", "oproj", "gateup", "down"):
-        n = launches_ph[k]
-        if n:
-            us = phases[k] / n
-            per_phase[k] = {"us_per_launch": us, "launches_per_step": n // args.steps,
-                            "tflops": fl[k] / shape.n_layers / us / 1e6}
-    if launches_ph["gather"]:
-        us = phases["gather"] / launches_ph["gather"]
-        per_phase["gather"] = {"us_per_launch": us, "launches_per_step": 1, "gbs": gather_bytes / us / 1e3}
-    if launches_ph["norm"]:
-        per_phase["norm"] = {"us_per_launch": phases["norm"] / launches_ph["norm"],
-                             "launches_per_step": launches_ph["norm"] // args.steps}
-    dom = max(("qkv", "attn", "oproj", "gateup", "down", "gather"), key=lambda k: phases[k])
+    r, w, shape = main, main_w, main_w.shape
+    peaks, st, per_phase, fl = r["peaks"], r["st"], r["per_phase"], r["fl"]
+    tokens, new_rows = w.total_tokens, r["new_rows"]
+    value = aggregate_tokens_per_s(world, tokens, args.steps, r["total_ms"])
+    e2e_value = aggregate_tokens_per_s(world, tokens, args.steps, r["e2e_ms"])
+    dom = max(("qkv", "attn", "oproj", "gateup", "down", "gather"), key=lambda k: r["phases"][k])
     if dom == "gather":
         roof = {"bound": "hbm", "achieved": per_phase[dom]["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                "frac": per_phase[dom]["gbs"] / peaks["hbm_gbs"], "traffic": None, "kernel": "gather_rerope_kernel"}
+                "frac": per_phase[dom]["gbs"] / peaks["hbm_gbs"], "traffic": None, "kernel": "gather_rerope_kernel",
+                "peak_source": f"{peaks['source']} copy bandwidth"}
     else:
-        roof = {"bound": "tensor", "achieved": per_phase[dom]["tflops"], "peak": peaks["tflops_sustained"],
-                "unit": "TFLOP/s", "frac": per_phase[dom]["tflops"] / peaks["tflops_sustained"], "traffic": None,
-                "kernel": {"attn": "umma_attention_kernel"}.get(dom, f"umma_gemm_kernel<{dom}>")}
-    roof["peak_source"] = f"{peaks['source']} (sustained bf16 figure x 1.0 nominal fp16/bf16 ratio)" \
-        if roof["bound"] == "tensor" else peaks["source"]
-    roof["share_of_step"] = phases[dom] / max(sum(phases.values()), 1e-9)
-    roof["traffic"] = kernel_traffic(roof["kernel"], w.name)
-    roof["algorithmic_per_launch"] = gather_bytes if dom == "gather" else fl[dom] / shape.n_layers
-    kernels_per_step = (sum(launches[k] for k in pcb.PHASES if k != "io") // args.steps) + 1
+        roof = {"bound": "tensor", "achieved": per_phase[dom]["tflops"], "peak": r["tensor_peak"], "unit": "TFLOP/s",
+                "frac": per_phase[dom]["tflops"] / r["tensor_peak"], "traffic": None,
+                "kernel": KERNEL_OF.get(dom, f"umma_gemm_kernel<{dom}>"),
+                "peak_source": f"{peaks['source']} {r['which_peak']} bf16 figure x 1.0 (nominal fp16 : bf16 ratio); "
+                               f"{r['which_peak']} because the timed region lasted {r['total_ms'] / 1000.0:.2f} s with "
+                               f"throttle reasons {r['clocks']['reasons']}"}
+    roof["share_of_step"] = r["phases"][dom] / max(sum(r["phases"].values()), 1e-9)
+    traffic = kernel_traffic(roof["kernel"], w.name)
+    roof["traffic"] = traffic
+    roof["traffic_source"] = None if traffic is None else "stored: one ncu capture of this kernel (profiles/dram_traffic.json), not this run"
+    roof["algorithmic_per_launch"] = r["gather_bytes"] if dom == "gather" else fl[dom] / shape.n_layers
+    kernels_per_step = (sum(r["launches"][k] for k in pcb.PHASES if k != "io") // args.steps) + 1
+    main_row = table_row(r, world, args.steps)
 
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
-        n_sample = max(1, min(shape.n_layers, 7))
-        step, cores = oracle_sample(w, n_sample)
-        t = step()
-        scale = shape.n_layers / n_sample
-        cpu = {"value": tokens / (t * scale), "unit": UNIT, "cores": cores, "kind": "oracle",
-               "sample": f"first {n_sample} of {shape.n_layers} layers of {w.name}, all new rows, one call "
-                         f"({t:.1f} s), time x {scale:g}"}
+        cpu = cpu_baseline_for(w)
+        main_row["cpu_baseline"] = cpu
 
     print(json.dumps({
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
-        "ms_per_step": total_ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "ms_per_step": r["total_ms"] / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
         "config": {"workload": w.name, "description": w.description, "tokens_per_step": tokens,
                    "new_rows_per_step": new_rows, "hit_tokens_per_step": int(st["hit_tokens"]),
-                   "prompts_per_step": len(w.prompts), "ms_per_prompt": total_ms / args.steps / len(w.prompts),
-                   "computed_rows_per_s": world * new_rows * args.steps / (total_ms / 1000.0),
+                   "prompts_per_step": len(w.prompts), "ms_per_prompt": r["total_ms"] / args.steps / len(w.prompts),
+                   "computed_rows_per_s": world * new_rows * args.steps / (r["total_ms"] / 1000.0),
                    "l2": f"inputs exceed L2: {shape.params_per_layer * shape.n_layers * 2 / 1e6:.0f} MB of weights are "
                          "streamed every step", "multi_gpu": "independent replicas, no collective",
                    "cache_state": "chunks stored by a step are dropped again before the next (untimed host bookkeeping)",
-                   "device_ms_per_step_kernels_only": dev_us / args.steps / 1000.0,
-                   "host_plan_us": st["host_plan_us"], "phase_pass_ms_per_step": float(sum(ms_ph)) / args.steps},
-        "clocks": clocks,
+                   "device_ms_per_step_kernels_only": r["dev_us"] / args.steps / 1000.0,
+                   "host_plan_us": st["host_plan_us"], "phase_pass_ms_per_step": float(sum(r["ms_ph"])) / r["ph_steps"]},
+        "clocks": r["clocks"],
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": new_rows * shape.d_model * 2,
-                "d2h_bytes_per_step": new_rows * shape.d_model * 4, "ms_per_step": e2e_ms / args.steps},
+                "d2h_bytes_per_step": new_rows * shape.d_model * 4, "ms_per_step": r["e2e_ms"] / args.steps},
         "gpu_launches": kernels_per_step * args.steps,
-        "roofline": roof, "kernels": per_phase, "cpu_baseline": cpu}))
-    h.close()
-    if dist is not None:
-        dist.destroy_process_group()
+        "roofline": roof, "kernels": per_phase, "cpu_baseline": cpu,
+        "step_tflops": main_row["step_tflops"], "step_frac_of_tensor_peak": main_row["step_frac_of_tensor_peak"],
+        "workloads": rows}))
 
 
 def run_qa_bank(args):
@@ -521,13 +739,24 @@ def run_decode(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--workload", default="cfg1")
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="percache", choices=["percache", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-table", action="store_true", help="time the named workload only, not the per-workload table")
     ap.add_argument("--flags", type=int, default=0, help="PERCACHE_FLAG_* bits kept set during the timed passes")
     args = ap.parse_args()
+    args.forward = sys.argv[1:]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":
+        # asked for N GPUs without a launcher around us: start one rank per GPU ourselves (independent replicas;
+        # the only thing they exchange is the maximum of their times)
+        import socket
+        import subprocess
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        raise SystemExit(subprocess.call(replica_launch_command(args, port)))
     if args.workload == "qa_bank":
         run_qa_bank(args)
     elif args.workload.startswith("decode_"):

@@ -23,7 +23,17 @@
  *    throws or aborts across this boundary.  percache_strerror() names a code.
  *  - A handle is not thread-safe.  All device work of a handle runs on the stream
  *    given at creation; calls return after that work has finished.
- *  - A call that fails leaves the store exactly as it was.
+ *  - A call that is refused before its device work starts (every argument, capacity and space check) leaves the
+ *    store exactly as it was, also when eviction is on: victims are chosen first but dropped only when the kernels
+ *    are about to write.  A call whose device work fails (PERCACHE_E_CUDA, PERCACHE_E_DEVICE_TIMEOUT) stores
+ *    nothing and leaves the store consistent, but chunks it evicted to make room stay evicted, and the assembled
+ *    context of the previous call is forgotten (percache_decode then returns PERCACHE_E_INVAL).
+ *  - Number formats: the store is bf16, the residual stream fp32, every operand of a projection or of the attention
+ *    is fp16 with fp32 accumulation.  fp16 carries magnitudes up to 65504; every conversion to fp16 inside the
+ *    library saturates (a larger value becomes +-65504, never infinity), so out-of-range weights, cached values or
+ *    activations (a SwiGLU product, a rotated key) are clipped and the call stays finite.  Results are only
+ *    meaningful while normed activations, projections and SwiGLU products stay within that range; bf16 values below
+ *    2^-24 in magnitude flush to zero as operands.
  *  - The library never frees or keeps caller memory: every caller buffer may be
  *    released as soon as the call returns.
  *  - There is no CPU fallback: without a CUDA device every call that needs one fails
@@ -233,7 +243,7 @@ typedef struct {
 
 PERCACHE_API int percache_get_stats(percache_t* h, percache_stats_t* out);
 
-/* Switch PERCACHE_FLAG_PHASE_TIMING / PERCACHE_FLAG_REFERENCE_KERNELS after creation. */
+/* Replace the handle's flags (any PERCACHE_FLAG_* bits) after creation. */
 PERCACHE_API int percache_set_flags(percache_t* h, uint32_t flags);
 
 /* Integer plan of the last successful percache_prefill (host int32 arrays, caller-allocated).
@@ -255,9 +265,29 @@ PERCACHE_API int percache_debug_attn_plan(const int32_t* n_blocks, int32_t n_til
                              int32_t max_partial_slots, int32_t* items_out, int64_t items_capacity,
                              int64_t* counts_out);
 
+/* Debugging aid for parity checks at full size and depth: while host_buf is set, every percache_prefill (and
+ * percache_decode) call also copies the fp32 residual stream of its rows as it enters each decoder block, and once
+ * more after the last block, to host_buf laid out [n_layers + 1][rows of the call][d_model] (entry l = input of
+ * block l, entry n_layers = the call's output).  A checker can then feed block l's input to a reference
+ * implementation and compare single blocks, which keeps the check affordable where a whole reference run is not.
+ * host_buf: caller-owned host memory of capacity_floats floats that must stay valid until it is unset with NULL; a
+ * prefill that needs more than the capacity fails with PERCACHE_E_CAPACITY before anything runs.  The copies
+ * serialise the call's kernels: never leave this on while timing. */
+PERCACHE_API int percache_debug_capture_layers(percache_t* h, float* host_buf, int64_t capacity_floats);
+
 /* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
  * [n_total + tokens decoded since][n_kv_heads][head_dim], copied to host buffers. */
 PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
+
+/* Failure-path check that is safe to run: one tiny kernel waits, through the very wait function every tcgen05
+ * kernel of this library uses, on a shared-memory barrier nobody arrives at.  The first waiter's limit is limit_us
+ * (1..2000): its wait runs out and it records a code in the error word; a second waiter with a 1000 times longer
+ * limit must leave as soon as it sees that code.  Nothing is in flight (no bulk copy, no tensor memory), the kernel
+ * returns normally and the device stays usable.  Returns PERCACHE_E_DEVICE_TIMEOUT when the wait ran out as
+ * designed (the mapping percache_prefill applies to a non-zero error word), PERCACHE_OK if the error word stayed
+ * zero.  code_out: the recorded code (901 = the probe); waited_ns [2]: how long the two waiters waited.  Either
+ * pointer may be NULL. */
+PERCACHE_API int percache_debug_wait_probe(int32_t device, uint32_t limit_us, int32_t* code_out, uint64_t* waited_ns);
 
 /* C[M][N] (fp32, host) = A[M][K] * B[N][K]^T with fp16 inputs (host), through the tcgen05 GEMM
  * (use_reference = 0), the plain kernel (1), or the tcgen05 GEMM on CTA pairs with 256 x 256 tiles (2; needs

@@ -339,6 +339,57 @@ def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit:
 
 
 # --------------------------------------------------------------------------- #
+# one block, some rows: the unit of a teacher-forced check
+# --------------------------------------------------------------------------- #
+def block_rows(model: Model, layer: int, x: np.ndarray, new_slots: np.ndarray, n_total: int,
+               hit_segments: Sequence[Tuple[int, np.ndarray, np.ndarray]], rows: np.ndarray,
+               round_kv: bool = True) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """One transformer block of reuse-prefill for one prompt, with the block's output formed for some rows only.
+
+    The same steps as the loop body of reuse_prefill (Appendix B.1: projection and position encoding on the rows
+    that are not covered by loaded tensors, computed and loaded tensors concatenated on the sequence axis, the rest
+    of the block as usual), arranged so that a full-size case can be checked block by block: the K and V of a
+    block depend on the block's input for *every* new row, but attention, output projection and FFN are row-wise,
+    so they are evaluated for the chosen rows alone.
+
+    x            float64 [m, d]: the block's input for all m new rows of the prompt, in slot order
+    new_slots    int [m]: their slots (= positions), ascending
+    n_total      context length T of the prompt
+    hit_segments [(first slot, K [n, Hkv, hd], V [n, Hkv, hd])]: this layer's stored (unrotated, bf16-valued)
+                 tensors of the chunks that hit, each with the slot its first token occupies
+    rows         indices into the m new rows
+    Returns (block output of the chosen rows [len(rows), d], unrotated K of all new rows, V of all new rows).
+    """
+    hq, hkv, hd = model.n_q_heads, model.n_kv_heads, model.head_dim
+    new = np.asarray(new_slots)
+    rows = np.asarray(rows)
+    m = x.shape[0]
+    xn = rmsnorm(x, model.w(layer, "attn_norm"), model.rms_eps)
+    k = (xn @ model.w(layer, "wk").T).reshape(m, hkv, hd)
+    v = (xn @ model.w(layer, "wv").T).reshape(m, hkv, hd)
+    if round_kv:
+        k, v = round_to_bf16(k), round_to_bf16(v)
+    k_pre = np.zeros((n_total, hkv, hd), dtype=np.float64)
+    v_all = np.zeros((n_total, hkv, hd), dtype=np.float64)
+    k_pre[new] = k
+    v_all[new] = v
+    for start, ck, cv in hit_segments:
+        k_pre[start:start + ck.shape[0]] = ck
+        v_all[start:start + cv.shape[0]] = cv
+    pos_r = new[rows]
+    t_hi = int(pos_r.max()) + 1 if rows.size else 0          # no chosen row sees a slot beyond this one
+    k_rot = rope(k_pre[:t_hi], np.arange(t_hi), model.rope_theta)
+    q = (xn[rows] @ model.w(layer, "wq").T).reshape(rows.size, hq, hd)
+    q_rot = rope(q, pos_r, model.rope_theta)
+    att = attention_rows(q_rot, pos_r, k_rot, v_all[:t_hi])
+    xr = x[rows] + att @ model.w(layer, "wo").T
+    yn = rmsnorm(xr, model.w(layer, "ffn_norm"), model.rms_eps)
+    act = silu(yn @ model.w(layer, "w_gate").T) * (yn @ model.w(layer, "w_up").T)
+    xr = xr + act @ model.w(layer, "w_down").T
+    return xr, k, v
+
+
+# --------------------------------------------------------------------------- #
 # the plain definition without any cache: every row goes through every block
 # --------------------------------------------------------------------------- #
 def dense_prefill(model: Model, hidden: np.ndarray, round_kv: bool = True):

@@ -15,7 +15,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 OBJ_DIR = os.path.join(HERE, "_build")
 LIB_PATH = os.path.join(HERE, "libpercache.so")
-SOURCES = ["percache_api.cu", "kernels_mem.cu", "kernels_ref.cu", "gemm_umma.cu", "gemm_small.cu", "attn_umma.cu", "attn_decode.cu", "attn_plan.cu", "gemm_noalloc.cu", "qa_bank.cu"]
+SOURCES = ["percache_api.cu", "kernels_mem.cu", "kernels_ref.cu", "gemm_umma.cu", "gemm_small.cu", "attn_umma.cu", "attn_decode.cu", "attn_plan.cu", "gemm_noalloc.cu", "qa_bank.cu", "wait_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]
 

@@ -67,6 +67,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   __shared__ __align__(8) uint64_t k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ __align__(8) uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
   __shared__ uint32_t tmem_base_slot;
+  __shared__ int cta_failed;       // set by any role whose bounded wait ran out (or saw another role's error)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -87,6 +88,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   }
 
   if (threadIdx.x == 0) {
+    cta_failed = 0;
     mbar_init(&q_full, 1);
     mbar_init(&q_empty, 1);
     for (int s = 0; s < KV_STAGES; ++s) {
@@ -125,7 +127,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const int gp = t.unit;
         const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
         const int nb = t.blk_end - t.blk_begin;
-        if (!mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+        if (!mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; cta_failed = 1; break; }
         mbar_arrive_expect_tx(&q_full, 2 * TILE_BYTES);
         for (int i = 0; i < 2; ++i)
           for (int hf = 0; hf < 2; ++hf)
@@ -134,22 +136,19 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         for (int j = 0; j < nb; ++j, ++kvit) {
           const int st = kvit & 1;
           const uint32_t ph = (kvit >> 1) & 1u;
-          if (!mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+          if (!mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; cta_failed = 1; break; }
           mbar_arrive_expect_tx(&k_full[st], TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
             tma_load_2d(k_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmK, &k_full[st], g * HEAD_DIM + hf * 64,
                         t.ctx0 + (t.blk_begin + j) * BLK);
-          if (!mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; break; }
+          if (!mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER)) { ok = false; cta_failed = 1; break; }
           mbar_arrive_expect_tx(&v_full[st], TILE_BYTES);
           for (int hf = 0; hf < 2; ++hf)
             tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES, &tmV, &v_full[st], g * HEAD_DIM + hf * 64,
                         t.ctx0 + (t.blk_begin + j) * BLK);
         }
       }
-      if (!ok) {   // error path only: let copies already issued land before shared memory is released
-        const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
-      }
+      (void)ok;
     }
   } else if (warp == 9) {
     // ---------------------------------------------------------------- MMA issuer
@@ -174,8 +173,8 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const AttnItem t = w == w_begin ? first_item : args.items[w];
         const int nb = t.blk_end - t.blk_begin;
         const uint32_t kv0 = kvit;
-        if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
-        if (!mbar_wait(&k_full[kv0 & 1], (kv0 >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+        if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
+        if (!mbar_wait(&k_full[kv0 & 1], (kv0 >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
         tc_fence_after_sync();
         issue_s(0, kv0);
         issue_s(1, kv0);
@@ -185,9 +184,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           const uint32_t kvidx = kv0 + j;
           const int st = kvidx & 1;
           for (int i = 0; i < 2; ++i) {
-            if (!mbar_wait(&p_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
-            if (j == 0 && !mbar_wait(&o_free[i], (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
-            if (i == 0 && !mbar_wait(&v_full[st], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+            if (!mbar_wait(&p_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
+            if (j == 0 && !mbar_wait(&o_free[i], (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
+            if (i == 0 && !mbar_wait(&v_full[st], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
             tc_fence_after_sync();
             const uint32_t va = smem_u32(v_smem + st * TILE_BYTES);
 #pragma unroll
@@ -200,7 +199,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             if (i == 1) umma_commit(&v_empty[st]);
             if (j + 1 < nb) {
               const uint32_t nxt = kvidx + 1;
-              if (i == 0 && !mbar_wait(&k_full[nxt & 1], (nxt >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; break; }
+              if (i == 0 && !mbar_wait(&k_full[nxt & 1], (nxt >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
               tc_fence_after_sync();
               issue_s(i, nxt);
               if (i == 1) {
@@ -237,7 +236,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         const uint32_t kvidx = kv0 + j;
         ok = mbar_wait(&s_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_SOFTMAX);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;
+        if (!ok) { cta_failed = 1; break; }
         tc_fence_after_sync();
         uint32_t s[128];
 #pragma unroll
@@ -270,7 +269,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             // O_i must be complete up to the previous block before it is rescaled in place
             ok = mbar_wait(&o_done[i], (kvidx - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
             ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            if (!ok) { cta_failed = 1; break; }
             tc_fence_after_sync();
             float alpha = 1.0f;
             if (need) { alpha = fast_exp2(m - m_blk); m = m_blk; l *= alpha; }
@@ -311,7 +310,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       // ---- final: O_i / l -> fp16 -> out, or the unnormalised part -> scratch
       ok = mbar_wait(&o_done[i], (kv0 + nb - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+      if (!ok) { cta_failed = 1; break; }
       tc_fence_after_sync();
       if (t.partial_slot < 0) {
         const float inv_l = 1.0f / l;
@@ -361,6 +360,15 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // ---------------------------------------------------------------- teardown
   tc_fence_before_sync();
   __syncthreads();
+  if (cta_failed) {
+    // Error path only (the flag was written before the barrier, so the branch is uniform): let bulk copies this CTA
+    // issued land before its shared memory is released, whichever role it was that gave up.
+    if (threadIdx.x == 0) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
+    }
+    __syncthreads();
+  }
   if (warp == 9) {
     tc_fence_after_sync();
     tmem_dealloc<512>(tmem_base);
@@ -467,12 +475,13 @@ int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int
   if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0) return -1;
-  static bool smem_set = false;      // once per process: the call costs host time on every launch otherwise
-  if (!smem_set) {
+  static bool smem_set[MAX_DEVICES] = {};      // once per device: the call costs host time on every launch otherwise
+  const int dev = current_device_slot();
+  if (!smem_set[dev]) {
     if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
         cudaSuccess)
       return -1;
-    smem_set = true;
+    smem_set[dev] = true;
   }
   AttnArgs a{};
   a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out;

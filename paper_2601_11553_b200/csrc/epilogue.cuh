@@ -10,9 +10,18 @@ namespace pc {
 // rounded to fp16 right after, and the division was a third of the SwiGLU epilogue's time
 __device__ __forceinline__ float silu_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 
+// Two floats to packed fp16 (a in the low half), round to nearest even, SATURATING: a magnitude beyond the
+// largest finite fp16 value (65504) becomes +-65504 instead of infinity (NaN stays NaN).  Every fp16 operand the
+// library forms goes through this conversion, so an out-of-range activation or cached bf16 value clips instead
+// of turning into inf and, one masked product later, NaN.
 __device__ __forceinline__ uint32_t pack_half2(float a, float b) {
-  __half2 h = __floats2half2_rn(a, b);
-  return *reinterpret_cast<uint32_t*>(&h);
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));   // first source -> upper half
+  return r;
+}
+__device__ __forceinline__ __half to_half_sat(float a) {
+  const uint32_t r = pack_half2(a, 0.f);
+  return __ushort_as_half(static_cast<unsigned short>(r & 0xffffu));
 }
 __device__ __forceinline__ uint32_t pack_bf162(__nv_bfloat16 a, __nv_bfloat16 b) {
   __nv_bfloat162 h(a, b);

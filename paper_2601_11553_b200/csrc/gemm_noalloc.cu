@@ -48,7 +48,7 @@ extern "C" int percache_debug_gemm_noalloc(int32_t device, int32_t M, int32_t N,
   if (M <= 0 || N <= 0 || K <= 0 || !a_f16 || !b_f16 || !c) return PERCACHE_E_INVAL;
   if (K % 64 != 0 || N % 128 != 0) return PERCACHE_E_INVAL;
   // layout of the scratch: [error word | A padded to whole 128-row tiles | B | C], each 256-byte aligned
-  const size_t m_pad = static_cast<size_t>((M + 127) / 128) * 128;
+  const size_t m_pad = (static_cast<size_t>(M) + 127) / 128 * 128;     // in size_t: M may be close to INT32_MAX
   const size_t a_bytes = round256(m_pad * K * 2), b_bytes = round256(static_cast<size_t>(N) * K * 2);
   const size_t c_bytes = round256(static_cast<size_t>(M) * N * 4);
   if (256 + a_bytes + b_bytes + c_bytes > NOALLOC_SCRATCH_BYTES) return PERCACHE_E_CAPACITY;

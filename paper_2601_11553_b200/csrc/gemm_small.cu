@@ -54,8 +54,8 @@ __device__ __forceinline__ void qkv_store1(const QkvEpilogue& e, int row, const 
   if (is_q || is_k) cs = __ldg(e.rope + static_cast<size_t>(rw.pos) * ROPE_HALF + c);
   if (is_q) {
     __half* dst = e.q_out + static_cast<size_t>(row) * (e.n_q_heads * HEAD_DIM) + hb * HEAD_DIM + c;
-    dst[0] = __float2half_rn(lo * cs.x - hi * cs.y);
-    dst[ROPE_HALF] = __float2half_rn(hi * cs.x + lo * cs.y);
+    dst[0] = to_half_sat(lo * cs.x - hi * cs.y);
+    dst[ROPE_HALF] = to_half_sat(hi * cs.x + lo * cs.y);
     return;
   }
   const int kvh = is_k ? hb - e.n_q_heads : hb - e.n_q_heads - e.n_kv_heads;
@@ -68,8 +68,8 @@ __device__ __forceinline__ void qkv_store1(const QkvEpilogue& e, int row, const 
   }
   const float l = __bfloat162float(bl), h = __bfloat162float(bh);
   __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(rw.slot) * kv_dim + kvh * HEAD_DIM + c;
-  dst[0] = __float2half_rn(is_k ? l * cs.x - h * cs.y : l);
-  dst[ROPE_HALF] = __float2half_rn(is_k ? h * cs.x + l * cs.y : h);
+  dst[0] = to_half_sat(is_k ? l * cs.x - h * cs.y : l);
+  dst[ROPE_HALF] = to_half_sat(is_k ? h * cs.x + l * cs.y : h);
 }
 
 template <int KIND, int MR, bool NORM>
@@ -209,7 +209,7 @@ __global__ void __launch_bounds__(SM_THREADS) small_gemm_kernel(SmallArgs a) {
       if (KIND == EPI_QKV) {
         qkv_store1(a.qkv, lane, rw, unit / ROPE_HALF, unit % ROPE_HALF, s0, s1);
       } else if (KIND == EPI_SWIGLU) {
-        a.swi.act[static_cast<size_t>(lane) * a.swi.ld + unit] = __float2half_rn(silu_f(s0) * s1);
+        a.swi.act[static_cast<size_t>(lane) * a.swi.ld + unit] = to_half_sat(silu_f(s0) * s1);
       } else {
         float* p = a.res.resid + static_cast<size_t>(lane) * a.res.ld + r0;
         if (k_parts > 1) {
@@ -230,7 +230,8 @@ template <int KIND, bool NORM, int MR>
 int launch_small_mr(const SmallArgs& a, int n_sms, cudaStream_t s) {
   const size_t smem = static_cast<size_t>(MR) * a.K * sizeof(__half);
   if (smem > 200 * 1024) return -1;
-  static size_t smem_set = 0;        // per kernel instantiation: raised when a call needs more than any before
+  static size_t smem_set_of[MAX_DEVICES] = {};   // per kernel instantiation and device: raised when a call needs more
+  size_t& smem_set = smem_set_of[current_device_slot()];
   if (smem > smem_set) {
     if (cudaFuncSetAttribute(small_gemm_kernel<KIND, MR, NORM>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem)) != cudaSuccess)

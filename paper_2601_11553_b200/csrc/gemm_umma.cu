@@ -73,6 +73,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   __shared__ __align__(8) uint64_t tmem_full_bar[2];
   __shared__ __align__(8) uint64_t tmem_empty_bar[2];
   __shared__ uint32_t tmem_base_slot;
+  __shared__ int cta_failed;       // set by any role whose bounded wait ran out (or saw another role's error)
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -88,6 +89,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   auto kb_end = [&](int item) { return ((item % k_splits + 1) * n_kb_total) / k_splits; };
 
   if (threadIdx.x == 0) {
+    cta_failed = 0;
     for (int s = 0; s < STAGES; ++s) { mbar_init(&full_bar[s], 1); mbar_init(&empty_bar[s], 1); }
     for (int s = 0; s < 2; ++s) { mbar_init(&tmem_full_bar[s], 1); mbar_init(&tmem_empty_bar[s], PAIR ? 16 : 8); }
     fence_mbar_init();
@@ -165,7 +167,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
             --early;
             load_a(stage, kb, m_idx);
           } else {
-            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; break; }
+            if (!mbar_wait(&empty_bar[stage], phase ^ 1u, args.err_word, DEV_ERR_GEMM_PRODUCER)) { ok = false; cta_failed = 1; break; }
             expect(stage);
             load_a(stage, kb, m_idx);
             load_b(stage, kb, n_idx);
@@ -173,11 +175,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
           if (++stage == STAGES) { stage = 0; phase ^= 1u; }
         }
       }
-      if (!ok) {
-        // Error path only: give copies already issued time to land before shared memory is released.
-        const unsigned long long t0 = globaltimer_ns();
-        while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
-      }
+      (void)ok;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -190,12 +188,12 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       for (int tile = worker; tile < n_tiles && ok; tile += n_workers, ++it) {
         const int acc = it & 1;
         const uint32_t acc_phase = (it >> 1) & 1u;
-        if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
+        if (!mbar_wait(&tmem_empty_bar[acc], acc_phase ^ 1u, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; cta_failed = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
         const int kb0 = kb_begin(tile), kb1 = kb_end(tile);
         for (int kb = kb0; kb < kb1; ++kb) {
-          if (!mbar_wait(&full_bar[stage], phase, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; break; }
+          if (!mbar_wait(&full_bar[stage], phase, args.err_word, DEV_ERR_GEMM_MMA)) { ok = false; cta_failed = 1; break; }
           tc_fence_after_sync();
           const uint32_t a_addr = smem_u32(ring + stage * Cfg::STAGE_BYTES);
           const uint32_t b_addr = a_addr + A_STAGE_BYTES;
@@ -276,7 +274,7 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
       }
       bool ok = mbar_wait(&tmem_full_bar[acc], acc_phase, args.err_word, DEV_ERR_GEMM_EPILOGUE);
       ok = __all_sync(0xffffffffu, ok);
-      if (!ok) break;
+      if (!ok) { cta_failed = 1; break; }
       tc_fence_after_sync();
       const uint32_t t_acc = tmem_base + lane_base + static_cast<uint32_t>(acc * BN);
       const int row_base = m_idx * BM + quarter * 32;          // first of this warp's 32 rows
@@ -430,6 +428,16 @@ umma_gemm_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant_
   // ------------------------------------------------------------------ teardown (every thread gets here)
   tc_fence_before_sync();
   __syncthreads();
+  if (cta_failed) {
+    // Error path only (the flag was written before the barrier, so every thread takes the same branch): whichever
+    // role gave up, bulk copies this CTA issued may still be on their way into its shared memory; give them time to
+    // land before the memory is released.
+    if (threadIdx.x == 0) {
+      const unsigned long long t0 = globaltimer_ns();
+      while (globaltimer_ns() - t0 < DRAIN_LIMIT_NS) { }
+    }
+    __syncthreads();
+  }
   if constexpr (PAIR) {       // neither CTA may leave while the other can still read its memory or signal it
     cluster_arrive();
     cluster_wait();
@@ -449,12 +457,13 @@ EncodeTiledFn g_encode = nullptr;
 template <int BN, int KIND, bool PAIR>
 int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args, int n_sms, cudaStream_t s) {
   using Cfg = GemmCfg<BN, PAIR>;
-  static bool smem_set = false;      // per kernel instantiation, once per process
-  if (!smem_set) {
+  static bool smem_set[MAX_DEVICES] = {};      // per kernel instantiation and device
+  const int dev = current_device_slot();
+  if (!smem_set[dev]) {
     if (cudaFuncSetAttribute(umma_gemm_kernel<BN, KIND, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              Cfg::SMEM_BYTES) != cudaSuccess)
       return -1;
-    smem_set = true;
+    smem_set[dev] = true;
   }
   constexpr int TILE_M = PAIR ? 2 * BM : BM;
   const int n_tiles = ((args.M + TILE_M - 1) / TILE_M) * (args.N / BN) * (args.k_splits > 0 ? args.k_splits : 1);
@@ -477,7 +486,8 @@ int launch_one(const GemmOperand& A, const GemmOperand& B, const GemmArgs& args,
     cfg.numAttrs = 2;
     // SMs pair up inside a GPC only, so fewer than n_sms / 2 clusters may be resident at once; a persistent
     // grid larger than that would run its last clusters after all the others
-    static int max_clusters = 0;                // per kernel instantiation (one device model per process)
+    static int max_clusters_of[MAX_DEVICES] = {};      // per kernel instantiation and device
+    int& max_clusters = max_clusters_of[dev];
     if (max_clusters == 0) {
       cfg.gridDim = dim3((n_sms / 2) * 2);
       int n = 0;
@@ -525,11 +535,6 @@ int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t c
   const uint64_t strides[1] = {static_cast<uint64_t>(cols) * 2};
   const uint32_t box[2] = {static_cast<uint32_t>(BK), static_cast<uint32_t>(box_rows)};
   return encode_f16_map(&out->map, base, 2, dims, strides, box);
-}
-
-int umma_gemm_block_n(GemmEpilogueKind kind) {
-  (void)kind;
-  return 128;
 }
 
 // Tile shape (and, for the residual GEMMs, the number of K parts) for a problem.  The main loop of a single

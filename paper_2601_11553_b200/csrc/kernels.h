@@ -138,7 +138,7 @@ int make_operand_map(GemmOperand* out, const void* base, int64_t rows, int64_t c
 int launch_umma_gemm(const GemmOperand& A, const GemmOperand& B, int M, int N, int K, int block_n,
                      GemmEpilogueKind kind, const void* epilogue, float* c_f32, int* err_word, int n_sms,
                      cudaStream_t s, int k_splits = 1, int pair = 0);
-int umma_gemm_block_n(GemmEpilogueKind kind);    // narrowest N tile (a B operand map needs box_rows = the tile used)
+constexpr int UMMA_GEMM_MIN_BLOCK_N = 128;       // narrowest N tile (a B operand map needs box_rows = the tile used)
 // tile width, number of K parts (parts > 1 only if may_split_k: the residual epilogue then adds atomically) and
 // whether CTA pairs are used (only if may_pair)
 void umma_gemm_pick_shape(int M, int N, int K, int n_sms, bool may_split_k, bool may_pair, int* block_n,
@@ -170,6 +170,15 @@ void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* 
                             __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
 
 int init_driver_api();   // resolves cuTensorMapEncodeTiled once; 0 on success
+
+// Kernel attributes (dynamic shared memory limit) and cluster occupancy belong to a device, not to the process:
+// launch helpers remember what they have set per device ordinal.
+constexpr int MAX_DEVICES = 64;
+inline int current_device_slot() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return 0;
+  return dev;
+}
 
 // Launch with programmatic stream serialisation (see pdl_wait() in ptx.cuh).
 template <typename... KArgs, typename... Args>

@@ -1,5 +1,6 @@
 // Memory-bound kernels: gather + re-RoPE of cached pages, RMSNorm, format conversions, page copies.
 #include <algorithm>
+#include "epilogue.cuh"
 #include "kernels.h"
 #include "ptx.cuh"
 
@@ -29,7 +30,7 @@ void launch_build_rope_table(float2* table, int max_pos, double theta, cudaStrea
 __global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int64_t n) {
   int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
   const int64_t stride = static_cast<int64_t>(gridDim.x) * blockDim.x;
-  for (; i < n; i += stride) dst[i] = __float2half_rn(__bfloat162float(src[i]));
+  for (; i < n; i += stride) dst[i] = to_half_sat(__bfloat162float(src[i]));
 }
 void launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, int64_t n, cudaStream_t s) {
   if (n <= 0) return;
@@ -45,8 +46,8 @@ __global__ void interleave_rows_kernel(const __nv_bfloat16* __restrict__ gate, c
   for (; i < n; i += stride) {
     const int r = static_cast<int>(i / cols), c = static_cast<int>(i % cols);
     const int b = r / blk, rr = r % blk;
-    dst[(static_cast<int64_t>(2 * b) * blk + rr) * cols + c] = __float2half_rn(__bfloat162float(gate[i]));
-    dst[(static_cast<int64_t>(2 * b + 1) * blk + rr) * cols + c] = __float2half_rn(__bfloat162float(up[i]));
+    dst[(static_cast<int64_t>(2 * b) * blk + rr) * cols + c] = to_half_sat(__bfloat162float(gate[i]));
+    dst[(static_cast<int64_t>(2 * b + 1) * blk + rr) * cols + c] = to_half_sat(__bfloat162float(up[i]));
   }
 }
 void launch_interleave_rows_bf16_to_f16(const __nv_bfloat16* gate, const __nv_bfloat16* up, __half* dst, int rows,
@@ -106,9 +107,7 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* x, const floa
   for (int k = 0; k < VPL; ++k) {
     const int i = lane + 32 * k;
     if (i < nv) {
-      __half2 a = __floats2half2_rn(v[k].x * inv * g[k].x, v[k].y * inv * g[k].y);
-      __half2 b = __floats2half2_rn(v[k].z * inv * g[k].z, v[k].w * inv * g[k].w);
-      o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+      o2[i] = pack_half4(v[k].x * inv * g[k].x, v[k].y * inv * g[k].y, v[k].z * inv * g[k].z, v[k].w * inv * g[k].w);
     }
   }
 }
@@ -135,9 +134,7 @@ __global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* x, const
   for (int i = lane; i < nv; i += 32) {
     const float4 v = ld_dep_f32x4(xr + i);
     const float4 g = g4[i];
-    __half2 a = __floats2half2_rn(v.x * inv * g.x, v.y * inv * g.y);
-    __half2 b = __floats2half2_rn(v.z * inv * g.z, v.w * inv * g.w);
-    o2[i] = make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+    o2[i] = pack_half4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
   }
 }
 void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s) {
@@ -171,10 +168,7 @@ __device__ __forceinline__ void bf16x8_to_float(const uint4& v, float (&f)[8]) {
 __device__ __forceinline__ uint4 float8_to_f16x8(const float (&f)[8]) {
   uint32_t o[4];
 #pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    __half2 h = __floats2half2_rn(f[2 * i], f[2 * i + 1]);
-    o[i] = *reinterpret_cast<uint32_t*>(&h);
-  }
+  for (int i = 0; i < 4; ++i) o[i] = pack_half2(f[2 * i], f[2 * i + 1]);   // saturating: bf16 reaches far beyond fp16
   return make_uint4(o[0], o[1], o[2], o[3]);
 }
 

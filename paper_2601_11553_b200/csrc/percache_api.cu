@@ -87,6 +87,8 @@ struct percache {
   uint64_t next_serial = 0;
 
   Plan plan;
+  float* capture_host = nullptr;   // debugging aid: layer inputs of the next calls are copied here (see header)
+  int64_t capture_capacity = 0;    // floats
   int32_t decode_reserve = 0;     // context slots kept free behind every prompt for percache_decode
   percache_stats_t stats{};
   std::vector<cudaEvent_t> events;
@@ -188,10 +190,13 @@ void refresh_page_stats(percache* h) {
 // Pages in use by stored chunks.
 int64_t pages_in_use(const percache* h) { return h->cfg.pool_pages - static_cast<int64_t>(h->free_pages.size()); }
 
-// Make `need` more pages fit under the limit.  Without the LFU flag this only checks.  With it, chunks are
-// evicted least-frequently-used first (ties: oldest first), never one whose id is in `keep`.  Nothing is
-// evicted unless the whole request can be met.  Returns the number of chunks evicted, or a negative code.
-int make_room(percache* h, int64_t need, const std::unordered_map<uint64_t, int64_t>& keep) {
+// Which chunks would have to go so that `need` more pages fit under the limit.  Nothing changes here.  Without the
+// LFU flag this only checks.  With it, victims are taken least-frequently-used first (ties: oldest first), never a
+// chunk whose id is in `keep`, and none unless the whole request can be met.  Returns the number of victims, or a
+// negative code.
+int pick_victims(const percache* h, int64_t need, const std::unordered_map<uint64_t, int64_t>& keep,
+                 std::vector<uint64_t>* victims) {
+  victims->clear();
   int64_t over = pages_in_use(h) + need - h->store_limit;
   if (over <= 0) return 0;
   if (!(h->flags & PERCACHE_FLAG_EVICT_LFU)) return PERCACHE_E_NOSPACE;
@@ -201,15 +206,64 @@ int make_room(percache* h, int64_t need, const std::unordered_map<uint64_t, int6
   std::sort(order.begin(), order.end());
   size_t n_evict = 0;
   for (; n_evict < order.size() && over > 0; ++n_evict)
-    over -= static_cast<int64_t>(h->table[order[n_evict].second].pages.size());
+    over -= static_cast<int64_t>(h->table.find(order[n_evict].second)->second.pages.size());
   if (over > 0) return PERCACHE_E_NOSPACE;
-  for (size_t i = 0; i < n_evict; ++i) {
-    auto it = h->table.find(order[i].second);
-    release_pages(h, it->second.pages);
-    h->table.erase(it);
-  }
+  for (size_t i = 0; i < n_evict; ++i) victims->push_back(order[i].second);
   return static_cast<int>(n_evict);
 }
+
+// Pages of a call that stores chunks, taken so that the call can still be undone.  New pages come from the free
+// list first and then from the pages of the chosen victims, which stay in the table until apply(): a call that
+// fails on the host before that gives its free-list pages back (undo_host) and the store is exactly as it was.
+// apply() is called right before the first kernel that writes pages; from then on the victims are gone and a
+// failure only returns the new pages (undo_device).
+struct PageTxn {
+  percache* h;
+  std::vector<uint64_t> victims;
+  std::vector<int32_t> victim_pages, from_free, from_victims;
+  bool applied = false;
+  explicit PageTxn(percache* hh) : h(hh) {}
+  void set_victims(const std::vector<uint64_t>& v) {
+    victims = v;
+    for (uint64_t id : v) {
+      const ChunkEntry& e = h->table.find(id)->second;
+      victim_pages.insert(victim_pages.end(), e.pages.begin(), e.pages.end());
+    }
+  }
+  int take(int n, std::vector<int32_t>* out) {
+    for (int i = 0; i < n; ++i) {
+      if (!h->free_pages.empty()) {
+        from_free.push_back(h->free_pages.back());
+        out->push_back(h->free_pages.back());
+        h->free_pages.pop_back();
+      } else if (from_victims.size() < victim_pages.size()) {
+        const int32_t pg = victim_pages[from_victims.size()];
+        from_victims.push_back(pg);
+        out->push_back(pg);
+      } else {
+        return PERCACHE_E_NOSPACE;
+      }
+    }
+    return PERCACHE_OK;
+  }
+  void undo_host() {          // before apply(): the free list gets its pages back in the order they left
+    for (auto p = from_free.rbegin(); p != from_free.rend(); ++p) h->free_pages.push_back(*p);
+    from_free.clear();
+    from_victims.clear();
+  }
+  void apply() {
+    for (uint64_t id : victims) h->table.erase(id);
+    for (size_t i = from_victims.size(); i < victim_pages.size(); ++i) h->free_pages.push_back(victim_pages[i]);
+    applied = true;
+  }
+  void undo_device() {        // after apply(): the new pages return to the free list, the victims stay evicted
+    for (auto p = from_victims.rbegin(); p != from_victims.rend(); ++p) h->free_pages.push_back(*p);
+    for (auto p = from_free.rbegin(); p != from_free.rend(); ++p) h->free_pages.push_back(*p);
+    from_free.clear();
+    from_victims.clear();
+  }
+  void undo() { if (applied) undo_device(); else undo_host(); }
+};
 
 // upload a page list through the pinned index block and run `fn` with the device pointer
 template <typename Fn>
@@ -266,8 +320,15 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   const bool small_rows = !use_ref && !(h->flags & PERCACHE_FLAG_NO_SMALL_ROW_KERNELS) && Mi <= SMALL_GEMM_MAX_ROWS &&
                           d % 256 == 0 && D.q_dim % 256 == 0 && D.d_ffn % 256 == 0;
   bool ok = true;
+  // debugging aid: the residual stream as it enters layer l goes to capture_host[l] (stream order does the rest)
+  auto capture = [&](int l) {
+    if (h->capture_host && static_cast<int64_t>(l + 1) * Mi * d <= h->capture_capacity)
+      ok = ok && cudaMemcpyAsync(h->capture_host + static_cast<size_t>(l) * Mi * d, h->resid,
+                                 static_cast<size_t>(Mi) * d * sizeof(float), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  };
   for (int l = 0; l < D.n_layers && ok && Mi > 0; ++l) {
     LayerWeights& W = h->layers[l];
+    capture(l);
     if (!small_rows) {
       timer.begin(PERCACHE_PH_NORM);
       launch_rmsnorm(h->resid, W.g_attn, h->xn, Mi, d, D.rms_eps, s);
@@ -376,6 +437,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     }
     timer.end();
   }
+  if (Mi > 0) capture(D.n_layers);
   return ok;
 }
 
@@ -436,7 +498,7 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   h->m_cap = cfg->max_batch_new_rows;
   h->ctx_cap = cfg->max_batch_ctx_tokens;
   cudaDeviceGetAttribute(&h->n_sms, cudaDevAttrMultiProcessorCount, cfg->device);
-  h->gu_blk = umma_gemm_block_n(EPI_SWIGLU) / 2;
+  h->gu_blk = UMMA_GEMM_MIN_BLOCK_N / 2;
 
   const int L = D.n_layers, d = D.d_model, F = D.d_ffn;
   bool ok = true;
@@ -542,7 +604,7 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
     launch_bf16_to_f32(p, W.g_attn, d, s);
     p = stage_bf16(S.ffn_norm, d, weights_on_device, tmp0, s, &cuda_ok);
     launch_bf16_to_f32(p, W.g_ffn, d, s);
-    const int bn = umma_gemm_block_n(EPI_QKV);
+    const int bn = UMMA_GEMM_MIN_BLOCK_N;
     cuda_ok = cuda_ok && make_operand_map(&W.m_wqkv, W.wqkv, D.qkv_dim, d, bn) == 0 &&
               make_operand_map(&W.m_wo, W.wo, d, D.q_dim, bn) == 0 &&
               make_operand_map(&W.m_wgu, W.wgu, 2 * F, d, bn) == 0 && make_operand_map(&W.m_wd, W.wd, d, F, bn) == 0;
@@ -576,8 +638,14 @@ int percache_set_store_limit(percache_t* h, int64_t pages) {
   if (!h || pages < 1 || pages > h->cfg.pool_pages) return PERCACHE_E_INVAL;
   const int64_t old = h->store_limit;
   h->store_limit = pages;
-  const int rc = make_room(h, 0, {});
+  std::vector<uint64_t> victims;
+  const int rc = pick_victims(h, 0, {}, &victims);
   if (rc < 0) { h->store_limit = old; return rc; }
+  for (uint64_t id : victims) {
+    auto it = h->table.find(id);
+    release_pages(h, it->second.pages);
+    h->table.erase(it);
+  }
   h->stats.evictions = rc;
   refresh_page_stats(h);
   return PERCACHE_OK;
@@ -635,20 +703,18 @@ int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, co
   const int n_pages = (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
   ChunkEntry ent;
   ent.n_tokens = n_tokens;
-  ent.serial = h->next_serial++;
-  int rc = make_room(h, n_pages, {});
+  std::vector<uint64_t> victims;
+  int rc = pick_victims(h, n_pages, {}, &victims);
   if (rc < 0) return rc;
-  h->stats.evictions = rc;
-  rc = alloc_pages(h, n_pages, &ent.pages);
-  if (rc != PERCACHE_OK) return rc;
+  const int evicted = rc;
+  rc = PERCACHE_OK;
   const size_t elems = static_cast<size_t>(h->dims.n_layers) * n_tokens * h->dims.kv_dim;
   __nv_bfloat16 *dk = nullptr, *dv = nullptr;
-  if (!ptr_is_device) {
+  if (!ptr_is_device) {      // staging copies first: an allocation failure must leave the store untouched
     if (cudaMalloc(reinterpret_cast<void**>(&dk), elems * 2) != cudaSuccess ||
         cudaMalloc(reinterpret_cast<void**>(&dv), elems * 2) != cudaSuccess) {
       cudaGetLastError();
       if (dk) cudaFree(dk);
-      release_pages(h, ent.pages);
       return PERCACHE_E_NOMEM;
     }
     if (cudaMemcpyAsync(dk, k, elems * 2, cudaMemcpyHostToDevice, h->stream) != cudaSuccess ||
@@ -658,15 +724,28 @@ int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, co
     dk = static_cast<__nv_bfloat16*>(const_cast<void*>(k));
     dv = static_cast<__nv_bfloat16*>(const_cast<void*>(v));
   }
-  if (rc == PERCACHE_OK)
+  PageTxn txn(h);
+  if (rc == PERCACHE_OK) {
+    txn.set_victims(victims);
+    rc = txn.take(n_pages, &ent.pages);
+  }
+  if (rc == PERCACHE_OK) {
+    txn.apply();
+    ent.serial = h->next_serial++;
     rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
       launch_chunk_pages_copy(dk, h->kpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 1,
                               h->stream);
       launch_chunk_pages_copy(dv, h->vpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim, 1,
                               h->stream);
     });
-  if (!ptr_is_device) { cudaFree(dk); cudaFree(dv); }
-  if (rc != PERCACHE_OK) { release_pages(h, ent.pages); return rc; }
+  }
+  if (!ptr_is_device) {
+    cudaStreamSynchronize(h->stream);
+    cudaFree(dk);
+    cudaFree(dv);
+  }
+  if (rc != PERCACHE_OK) { txn.undo(); refresh_page_stats(h); return rc; }
+  h->stats.evictions = evicted;
   h->table.emplace(chunk_id, std::move(ent));
   refresh_page_stats(h);
   return PERCACHE_OK;
@@ -678,17 +757,23 @@ int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tok
   if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
   ChunkEntry ent;
   ent.n_tokens = n_tokens;
-  ent.serial = h->next_serial++;
-  int rc = make_room(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, {});
+  const int n_pages = (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
+  std::vector<uint64_t> victims;
+  int rc = pick_victims(h, n_pages, {}, &victims);
   if (rc < 0) return rc;
-  h->stats.evictions = rc;
-  rc = alloc_pages(h, (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
-  if (rc != PERCACHE_OK) return rc;
+  const int evicted = rc;
+  PageTxn txn(h);
+  txn.set_victims(victims);
+  rc = txn.take(n_pages, &ent.pages);
+  if (rc != PERCACHE_OK) { txn.undo(); return rc; }
+  txn.apply();
+  ent.serial = h->next_serial++;
   rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
     launch_fill_synthetic(h->kpool, h->vpool, d_pages, n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.kv_dim,
                           seed, chunk_id, h->stream);
   });
-  if (rc != PERCACHE_OK) { release_pages(h, ent.pages); return rc; }
+  if (rc != PERCACHE_OK) { txn.undo(); refresh_page_stats(h); return rc; }
+  h->stats.evictions = evicted;
   h->table.emplace(chunk_id, std::move(ent));
   refresh_page_stats(h);
   return PERCACHE_OK;
@@ -799,13 +884,19 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     plan.cu_ctx.push_back(static_cast<int32_t>(ctx_total));
     plan.cu_new.push_back(static_cast<int32_t>(new_total));
   }
-  // every host-side check has passed: make the new pages fit (may evict, never a chunk this batch hits)
-  const int evicted = make_room(h, pages_needed, hit_uses);
-  if (evicted < 0) return evicted;
+  // every argument check has passed: choose what would have to be evicted so that the new pages fit (never a chunk
+  // this batch hits).  The store itself changes only when the device work is about to start (PageTxn::apply).
+  PageTxn txn(h);
+  {
+    std::vector<uint64_t> victims;
+    const int rc = pick_victims(h, pages_needed, hit_uses, &victims);
+    if (rc < 0) return rc;
+    txn.set_victims(victims);
+  }
+  const int evicted = static_cast<int>(txn.victims.size());
 
   // ---------------------------------------------------------------- pages for the chunks that will be stored
   std::vector<std::pair<uint64_t, ChunkEntry>> pending;
-  std::vector<int32_t> all_new_pages;
   std::unordered_map<uint64_t, size_t> pending_of;
   for (int b = 0; b < n_prompts; ++b)
     for (int i = 0; i < prompts[b].n_chunks; ++i) {
@@ -816,13 +907,20 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       ChunkEntry ent;
       ent.n_tokens = prompts[b].chunk_len[i];
       ent.serial = h->next_serial++;
-      alloc_pages(h, (ent.n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages);
-      all_new_pages.insert(all_new_pages.end(), ent.pages.begin(), ent.pages.end());
+      if (txn.take((ent.n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS, &ent.pages) != PERCACHE_OK) {
+        txn.undo();
+        return PERCACHE_E_NOSPACE;
+      }
       pending_of.emplace(id, pending.size());
       pending.emplace_back(id, std::move(ent));
     }
+  // A failure before the device work leaves the store exactly as it was.  Once kernels have written pages and the
+  // assembled context, the evicted chunks stay evicted, the new pages are released and the last call's context is
+  // forgotten (percache_decode then refuses to continue it).
   auto fail = [&](int code) {
-    release_pages(h, all_new_pages);
+    if (txn.applied) h->plan = Plan();
+    txn.undo();
+    refresh_page_stats(h);
     return code;
   };
 
@@ -941,6 +1039,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     const size_t wide = static_cast<size_t>(std::max(std::max(D.qkv_dim, 2 * D.d_ffn), d));
     if (!dev_alloc(h, &h->cref, static_cast<size_t>(h->m_cap) * wide)) return fail(PERCACHE_E_NOMEM);
   }
+  if (h->capture_host && static_cast<int64_t>(D.n_layers + 1) * M * d > h->capture_capacity) return fail(PERCACHE_E_CAPACITY);
+  txn.apply();      // from here on kernels write pages and the context
 
   timer.begin(PERCACHE_PH_IO);
   for (const Seg& sg : segs)
@@ -1007,6 +1107,13 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
   st.device_us = 1000.0 * ms;
   timer.collect();
+  return PERCACHE_OK;
+}
+
+int percache_debug_capture_layers(percache_t* h, float* host_buf, int64_t capacity_floats) {
+  if (!h || (host_buf && capacity_floats <= 0)) return PERCACHE_E_INVAL;
+  h->capture_host = host_buf;
+  h->capture_capacity = host_buf ? capacity_floats : 0;
   return PERCACHE_OK;
 }
 

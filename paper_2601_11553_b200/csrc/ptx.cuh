@@ -15,7 +15,7 @@ enum : int {
   DEV_ERR_NONE = 0,
   DEV_ERR_GEMM_PRODUCER = 101, DEV_ERR_GEMM_MMA = 102, DEV_ERR_GEMM_EPILOGUE = 103,
   DEV_ERR_ATTN_PRODUCER = 201, DEV_ERR_ATTN_MMA = 202, DEV_ERR_ATTN_SOFTMAX = 203, DEV_ERR_ATTN_CORR = 204,
-  DEV_ERR_BAD_INDEX = 301,
+  DEV_ERR_WAIT_PROBE = 901,        // the test kernel whose wait is meant to run out
 };
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;      // 2 s per wait

@@ -32,7 +32,7 @@ PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
            "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
            "percache_get_stats", "percache_set_flags", "percache_decode", "percache_set_decode_reserve", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx", "percache_debug_attn_plan",
-           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_path_key", "percache_qa_top1", "percache_strerror")
+           "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_debug_capture_layers", "percache_debug_wait_probe", "percache_path_key", "percache_qa_top1", "percache_strerror")
 
 
 class PerCacheError(RuntimeError):
@@ -105,6 +105,8 @@ def load_library() -> C.CDLL:
     lib.percache_debug_attn_plan.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
     lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
+    lib.percache_debug_capture_layers.argtypes = [vp, vp, i64]
+    lib.percache_debug_wait_probe.argtypes = [i32, C.c_uint32, C.POINTER(i32), C.POINTER(u64)]
     lib.percache_qa_top1.argtypes = [i32, vp, vp, i32, i32, vp, i32, C.c_float, vp, vp, vp, C.POINTER(C.c_float)]
     lib.percache_path_key.argtypes = [C.POINTER(u64), i32]
     lib.percache_path_key.restype = u64
@@ -340,6 +342,16 @@ class PerCache:
             res[name] = buf[:n].copy()
         return res
 
+    def capture_layers(self, buf: Optional[np.ndarray]) -> None:
+        """percache_debug_capture_layers: float32 host array [n_layers + 1, rows, d_model] (flat capacity counts), or
+        None to switch the capture off.  The array must stay alive until then."""
+        if buf is None:
+            _check(self._lib.percache_debug_capture_layers(self._h, None, 0), "percache_debug_capture_layers")
+            return
+        if buf.dtype != np.float32 or not buf.flags["C_CONTIGUOUS"]:
+            raise ValueError("capture buffer must be C-contiguous float32")
+        _check(self._lib.percache_debug_capture_layers(self._h, _ptr(buf), int(buf.size)), "percache_debug_capture_layers")
+
     def read_ctx(self, prompt: int, layer: int, n_total: int):
         """Assembled (rotated K, V) of one prompt and layer: two float16 arrays [n_total, kv_dim]."""
         k = np.empty((n_total, self.kv_dim), dtype=np.float16)
@@ -378,6 +390,14 @@ def debug_gemm(a_f16: np.ndarray, b_f16: np.ndarray, use_reference: bool = False
     _check(lib.percache_debug_gemm(device, m, n, k, _ptr(np.ascontiguousarray(a_f16)), _ptr(np.ascontiguousarray(b_f16)),
                                    _ptr(c), 2 if pair else (1 if use_reference else 0)), "percache_debug_gemm")
     return c
+
+
+def debug_wait_probe(limit_us: int = 1000, device: int = 0):
+    """percache_debug_wait_probe: returns (return code, recorded device code, [ns waited by the two waiters])."""
+    code = C.c_int32(0)
+    waited = (C.c_uint64 * 2)()
+    rc = load_library().percache_debug_wait_probe(device, int(limit_us), C.byref(code), waited)
+    return int(rc), int(code.value), [int(waited[0]), int(waited[1])]
 
 
 NOALLOC_SCRATCH_BYTES = 16 << 20

@@ -84,21 +84,27 @@ def weight_shapes(shape: ModelShape) -> Dict[str, tuple]:
     }
 
 
-def make_layer_weights(shape: ModelShape, seed: int, layer: int, std: float = 0.02) -> Dict[str, np.ndarray]:
-    """bf16 bit patterns of one layer's weights: projections ~ N(0, std), norm gains = 1."""
+def make_layer_weights(shape: ModelShape, seed: int, layer: int, std: float = 0.02,
+                       random_gains: bool = False) -> Dict[str, np.ndarray]:
+    """bf16 bit patterns of one layer's weights: projections ~ N(0, std); norm gains = 1 as the workload
+    descriptions say, or, with random_gains, 1 + 0.3 N(0, 1) per element and norm (for checks that must notice a
+    gain that is dropped, swapped between the two norms, or read at the wrong index)."""
     out: Dict[str, np.ndarray] = {}
     for i, (name, shp) in enumerate(weight_shapes(shape).items()):
         rng = np.random.default_rng([seed, 7001, layer, i])
         w = rng.standard_normal(shp, dtype=np.float32) * np.float32(std)
         out[name] = f32_to_bf16_bits(w)
-    ones = f32_to_bf16_bits(np.ones(shape.d_model, dtype=np.float32))
-    out["attn_norm"] = ones.copy()
-    out["ffn_norm"] = ones.copy()
+    for j, name in enumerate(("attn_norm", "ffn_norm")):
+        g = np.ones(shape.d_model, dtype=np.float32)
+        if random_gains:
+            g = g + np.float32(0.3) * np.random.default_rng([seed, 7006, layer, j]).standard_normal(
+                shape.d_model, dtype=np.float32)
+        out[name] = f32_to_bf16_bits(g)
     return out
 
 
-def make_weights(shape: ModelShape, seed: int, std: float = 0.02) -> List[Dict[str, np.ndarray]]:
-    return [make_layer_weights(shape, seed, l, std) for l in range(shape.n_layers)]
+def make_weights(shape: ModelShape, seed: int, std: float = 0.02, random_gains: bool = False) -> List[Dict[str, np.ndarray]]:
+    return [make_layer_weights(shape, seed, l, std, random_gains) for l in range(shape.n_layers)]
 
 
 def make_hidden(seed: int, tag: Sequence[int], n_tokens: int, d_model: int) -> np.ndarray:

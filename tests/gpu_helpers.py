@@ -102,3 +102,94 @@ def check_ctx(handle: pcb.PerCache, results: Sequence[orc.PromptResult], layers:
             worst = max(worst, float(err.max()) if err.size else 0.0)
             assert err.size == 0 or err.max() <= 1.0 + 1e-6, f"rotated K off by {err.max()} ulp (prompt {b}, layer {l})"
     return {"k_rot_max_ulp": worst}
+
+
+# --------------------------------------------------------------------------- teacher-forced, sampled-row checks
+def layout_only_store(ids_lens: Dict[int, int], cached: Sequence[int], shape: wl.ModelShape) -> orc.Store:
+    """A store that knows which chunks are cached and how long they are, without holding any tensor (the arrays
+    are zero-strided views): enough for the oracle's layout step at sizes where the tensors would not fit."""
+    st = orc.Store()
+    for c in cached:
+        z = np.broadcast_to(np.float64(0.0), (shape.n_layers, ids_lens[c], shape.n_kv_heads, shape.head_dim))
+        st.kv[c] = (z, z)
+    return st
+
+
+def sample_rows(layout: orc.Layout, n_random: int, rng: np.random.Generator) -> np.ndarray:
+    """Row indices (into the prompt's new rows): the first and last row of every run of consecutive new slots,
+    plus n_random others."""
+    new = layout.new_slots
+    m = new.shape[0]
+    if m == 0:
+        return np.zeros(0, dtype=np.int64)
+    brk = np.nonzero(np.diff(new) != 1)[0]
+    picks = set([0, m - 1] + [int(i) for i in brk] + [int(i) + 1 for i in brk])
+    rest = np.setdiff1d(np.arange(m), np.fromiter(picks, dtype=np.int64))
+    if n_random > 0 and rest.size:
+        picks.update(int(i) for i in rng.choice(rest, size=min(n_random, rest.size), replace=False))
+    return np.array(sorted(picks), dtype=np.int64)
+
+
+def teacher_forced_check(w: wl.Workload, layers: Sequence[int], n_random_per_prompt: int, flags: int = 0,
+                         random_gains: bool = False) -> Dict[str, float]:
+    """Full-size, full-depth parity where a whole oracle run is out of reach.
+
+    The library runs the workload once, handing out the residual stream as it enters every block.  For each
+    checked block the oracle gets the library's own input of that block (all new rows: the block's K and V depend
+    on every one of them), forms the block's output for sampled rows, and that is compared with the library's
+    input of the next block.  Blocks are then independent, so any subset can be checked; what an error in block l
+    does to later blocks is outside this check (end-to-end runs at full depth cover that on the smaller workloads).
+    Cached chunks hold the seeded integer pool values on both sides.
+    """
+    shape = w.shape
+    weights = wl.make_weights(shape, w.seed, random_gains=random_gains)
+    model = H.oracle_model(shape, weights)
+    ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
+    cached = set(w.cached_ids)
+    lstore = layout_only_store(ids_lens, w.cached_ids, shape)
+    oprompts = [H.oracle_prompt(p, [i for i, c in enumerate(p.chunk_ids) if c in cached]) for p in w.prompts]
+    layouts = [orc.assemble_layout(lstore, op) for op in oprompts]
+    m_total = sum(len(l.new_slots) for l in layouts)
+    cap = np.empty((shape.n_layers + 1, m_total, shape.d_model), dtype=np.float32)
+    with make_handle(shape, weights, w.prompts, flags=flags) as h:
+        for c in w.cached_ids:
+            h.put_chunk_synthetic(c, ids_lens[c], w.seed)
+        h.capture_layers(cap)
+        got = h.prefill(specs_for(w.prompts, w.cached_ids))
+        h.capture_layers(None)
+        check_plan(h.read_plan(), layouts)
+        stats = h.stats()
+    cu = np.cumsum([0] + [len(l.new_slots) for l in layouts])
+    for b, g in enumerate(got):        # the last capture is the call's output
+        assert np.array_equal(g.out_hidden, cap[shape.n_layers, cu[b]:cu[b + 1]])
+    rng = np.random.default_rng([w.seed, 7010])
+    rows_of = [sample_rows(l, n_random_per_prompt, rng) for l in layouts]
+    hkv, hd = shape.n_kv_heads, shape.head_dim
+    worst = {"max_abs": 0.0, "mean_abs": 0.0, "rows_per_layer": int(sum(r.size for r in rows_of)),
+             "layers": list(layers), "device_us": stats["device_us"]}
+    for l in layers:
+        pool: Dict[int, tuple] = {}
+
+        def seg(c):       # this layer's stored K, V of chunk c (the integer pool values), generated once per layer
+            if c not in pool:
+                n = ids_lens[c]
+                pool[c] = tuple(orc.bf16_bits_to_f64(wl.pool_kv_values(w.seed, c, which, l, n, hkv * hd)).reshape(n, hkv, hd)
+                                for which in (0, 1))
+            return pool[c]
+        errs = []
+        for b, (p, lay) in enumerate(zip(w.prompts, layouts)):
+            if rows_of[b].size == 0:
+                continue
+            segs, start = [], 0
+            for i, (c, n) in enumerate(zip(p.chunk_ids, p.chunk_len)):
+                if lay.hit_mask[i]:
+                    segs.append((start,) + seg(c))
+                start += n
+            x = cap[l, cu[b]:cu[b + 1]].astype(np.float64)
+            want, _, _ = orc.block_rows(model, l, x, lay.new_slots, lay.n_total, segs, rows_of[b])
+            errs.append(np.abs(cap[l + 1, cu[b] + rows_of[b]].astype(np.float64) - want))
+        e = np.concatenate(errs)
+        worst["max_abs"] = max(worst["max_abs"], float(e.max()))
+        worst["mean_abs"] = max(worst["mean_abs"], float(e.mean()))
+        assert e.max() <= TOL_MAX_ABS and e.mean() <= TOL_MEAN_ABS, (w.name, l, float(e.max()), float(e.mean()))
+    return worst

@@ -12,7 +12,8 @@ pytestmark = pytest.mark.gpu
 
 
 def run_case(w: wl.Workload, flags: int, check_store: bool = True):
-    weights = wl.make_weights(w.shape, w.seed)
+    # RMSNorm gains drawn away from 1: a gain that is dropped, swapped between the two norms or mis-indexed must fail
+    weights = wl.make_weights(w.shape, w.seed, random_gains=True)
     model = H.oracle_model(w.shape, weights)
     ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
     store = G.oracle_store_alone(model, w.seed, [(c, ids_lens[c]) for c in w.cached_ids])
@@ -66,6 +67,12 @@ def test_small_model_parity(case, flags):
     run_case(wl.small_workload(**case), flags)
 
 
+def test_wide_model_uses_the_two_pass_norm():
+    """d_model above 2048 takes the RMSNorm kernel that walks the row twice; gains are random here as well."""
+    w = wl.small_workload(seed=49, n_layers=2, chunk_lens=[96, 40], n_query=33, hit_idx=[0], d_model=2304)
+    run_case(w, 0)
+
+
 def test_all_hits_no_query_rows_is_rejected_or_empty():
     """A prompt whose every chunk hits and that has no query has no new rows: the call succeeds with n_new = 0."""
     w = wl.small_workload(seed=45, n_layers=1, chunk_lens=[48, 20], n_query=0, hit_idx=[0, 1])
@@ -81,7 +88,7 @@ def test_all_hits_no_query_rows_is_rejected_or_empty():
 
 def test_batch_of_ragged_prompts_and_first_miss_wins():
     shape = wl.small_workload(seed=46, n_layers=2, chunk_lens=[8], n_query=1, hit_idx=[]).shape
-    weights = wl.make_weights(shape, 46)
+    weights = wl.make_weights(shape, 46, random_gains=True)
     model = H.oracle_model(shape, weights)
     mk = lambda cid, n: wl.chunk_hidden_for(46, cid, n, shape.d_model)
     prompts = [

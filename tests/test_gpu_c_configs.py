@@ -12,8 +12,8 @@ from tests import helpers as H
 pytestmark = pytest.mark.gpu
 
 
-def run_workload(w: wl.Workload, ctx_layers=None):
-    weights = wl.make_weights(w.shape, w.seed)
+def run_workload(w: wl.Workload, ctx_layers=None, random_gains=False):
+    weights = wl.make_weights(w.shape, w.seed, random_gains=random_gains)
     model = H.oracle_model(w.shape, weights)
     ids_lens = {c: l for p in w.prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
     if w.cache_source == "integer_pool":
@@ -62,7 +62,7 @@ def test_config1_28_layers_bernoulli_hits():
 def test_config2_shape_two_layers():
     w = wl.config2()
     w.shape = wl.ModelShape(n_layers=2, **wl.SHAPE_B)
-    run_workload(w)
+    run_workload(w, random_gains=True)
 
 
 def test_config3_shape_batched_ragged_zipf_pool():
@@ -73,4 +73,4 @@ def test_config3_shape_batched_ragged_zipf_pool():
 def test_config4_shape_long_context_90pct_hits():
     w = wl.config4(0.9)
     w.shape = wl.ModelShape(n_layers=2, **wl.SHAPE_A)
-    run_workload(w)
+    run_workload(w, random_gains=True)

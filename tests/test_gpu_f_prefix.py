@@ -15,7 +15,7 @@ pytestmark = pytest.mark.gpu
 
 def test_prefix_tree_sequence():
     shape = wl.small_workload(seed=71, n_layers=3, chunk_lens=[16], n_query=1, hit_idx=[]).shape
-    weights = wl.make_weights(shape, 71)
+    weights = wl.make_weights(shape, 71, random_gains=True)
     model = H.oracle_model(shape, weights)
     lens = {1: 130, 5: 100, 7: 37, 9: 152, 12: 64}
     hid = {c: wl.chunk_hidden_for(71, c, n, shape.d_model) for c, n in lens.items()}

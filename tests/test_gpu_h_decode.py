@@ -18,7 +18,7 @@ def _decode_case(seed, n_layers, prompts_spec, n_steps, reserve, flags=0, **mode
                             **model_kw)
           for b, (cl, nq, hi) in enumerate(prompts_spec)]
     shape = ws[0].shape
-    weights = wl.make_weights(shape, seed)
+    weights = wl.make_weights(shape, seed, random_gains=True)     # the small-row projections fold the norm in
     model = H.oracle_model(shape, weights)
     prompts = [w.prompts[0] for w in ws]
     cached = [c for w in ws for c in w.cached_ids]

@@ -50,3 +50,21 @@ def test_reference_arm_under_a_two_process_launch_prints_one_line():
     d = json.loads(lines[0])
     assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["cpu_baseline"]["kind"] == "oracle"
     assert d["e2e"]["h2d_bytes_per_step"] == 0 and d["value"] > 0
+
+
+def test_self_launch_command_starts_one_rank_per_gpu():
+    """`bench.py --gpus N` without a launcher around it starts N ranks itself; the command it builds is checked here
+    with the CPU arm in place of the GPU arm (two gloo-free ranks, rank 0 prints the single line)."""
+    import argparse
+    sys.path.insert(0, ROOT)
+    import bench
+    args = argparse.Namespace(gpus=2, forward=["--gpus", "2", "--steps", "1", "--warmup", "0", "--workload", "cfg0",
+                                               "--impl", "reference"])
+    cmd = bench.replica_launch_command(args, 29519)
+    assert cmd[1:3] == ["-m", "torch.distributed.run"] and "--nproc-per-node" in cmd and cmd[cmd.index("--nproc-per-node") + 1] == "2"
+    assert cmd[cmd.index("--master-addr") + 1] == "127.0.0.1" and cmd[cmd.index("--master-port") + 1] == "29519"
+    assert os.path.basename(cmd[cmd.index("--master-port") + 2]) == "bench.py"
+    r = subprocess.run(cmd, capture_output=True, text=True, timeout=600, cwd=ROOT)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1 and json.loads(lines[0])["n_gpus"] == 2

@@ -447,3 +447,74 @@ def test_prefix_tree_reuse_equals_full_prefill_over_a_sequence_of_queries():
         full, _, _ = orc.dense_prefill(model, np.concatenate([hs[c] for c in ids] + [qh]))
         assert np.allclose(res.out_hidden, full[res.layout.new_slots], atol=1e-9), qi
     assert (1, 5, 9, 12) in store.kv and (5, 1) in store.kv and (1,) in store.kv and 1 not in store.kv
+
+
+# --------------------------------------------------------------------------- #
+# the block-by-block form used for teacher-forced checks at full size
+# --------------------------------------------------------------------------- #
+def _hit_segments(store, prompt, layout, layer):
+    segs, start = [], 0
+    for i, (cid, n) in enumerate(zip(prompt.chunk_ids, prompt.chunk_len)):
+        if layout.hit_mask[i]:
+            segs.append((start, store.kv[cid][0][layer], store.kv[cid][1][layer]))
+        start += n
+    return segs
+
+
+@pytest.mark.parametrize("mask", [(1, 0, 1), (0, 0, 0), (0, 1, 1)])
+def test_block_rows_chained_over_layers_is_reuse_prefill(mask):
+    """block_rows fed its own outputs, all rows chosen, walks the same path as reuse_prefill (itself pinned to an
+    independent decoder); with a subset of rows it returns exactly those rows; and with prefix hits the chain ends
+    at plain full prefill."""
+    shape, weights, model = tiny_model(seed=35, n_layers=3)
+    lens, nq = [7, 16, 5], 6
+    hs, qh = _chunks(shape, 35, lens, nq)
+    ids = [100, 101, 102]
+    store = orc.Store()
+    for i in range(3):            # cached content computed in some other context: each chunk alone
+        if mask[i]:
+            orc.reuse_prefill(model, store, [orc.Prompt([ids[i]], [lens[i]], [hs[i]], np.zeros((0, shape.d_model)))])
+    pr = orc.Prompt(ids, lens, [None if mask[i] else hs[i] for i in range(3)], qh)
+    want = orc.reuse_prefill(model, store, [pr], commit=False, keep_ctx=True)[0]
+    lay = want.layout
+    m = lay.new_slots.shape[0]
+    x = np.concatenate([hs[i] for i in range(3) if not mask[i]] + [qh])
+    some = np.array([0, m // 2, m - 1])
+    for l in range(3):
+        out_all, k_new, v_new = orc.block_rows(model, l, x, lay.new_slots, lay.n_total,
+                                               _hit_segments(store, pr, lay, l), np.arange(m))
+        out_some, _, _ = orc.block_rows(model, l, x, lay.new_slots, lay.n_total, _hit_segments(store, pr, lay, l), some)
+        assert np.allclose(out_some, out_all[some], atol=1e-12)
+        # the new rows' V is what reuse_prefill put into the assembled context at those slots
+        assert np.array_equal(v_new, want.v_ctx[l][lay.new_slots])
+        assert np.allclose(orc.rope(k_new, lay.new_slots, model.rope_theta), want.k_ctx[l][lay.new_slots], atol=1e-12)
+        x = out_all
+    assert np.allclose(x, want.out_hidden, atol=1e-10)
+
+
+def test_block_rows_with_prefix_hits_ends_at_full_prefill():
+    shape, weights, model = tiny_model(seed=36, n_layers=2)
+    lens, nq = [9, 12], 4
+    hs, qh = _chunks(shape, 36, lens, nq)
+    full, k_all, v_all = orc.dense_prefill(model, np.concatenate(hs + [qh]))
+    new = np.arange(lens[0], sum(lens) + nq)
+    x = np.concatenate([hs[1], qh])
+    for l in range(2):
+        x, _, _ = orc.block_rows(model, l, x, new, sum(lens) + nq, [(0, k_all[l][:lens[0]], v_all[l][:lens[0]])],
+                                 np.arange(new.shape[0]))
+    assert np.allclose(x, full[new], atol=1e-9)
+
+
+def test_block_rows_hit_segment_placement_matters():
+    """A segment placed one slot off, or K and V swapped, must change the result (the check is not vacuous)."""
+    shape, weights, model = tiny_model(seed=37, n_layers=1)
+    hs, qh = _chunks(shape, 37, [8, 8], 3)
+    _, kc, vc = orc.dense_prefill(model, hs[0])
+    new = np.arange(8, 19)
+    x = np.concatenate([hs[1], qh])
+    rows = np.arange(11)
+    good, _, _ = orc.block_rows(model, 0, x, new, 19, [(0, kc[0], vc[0])], rows)
+    swapped, _, _ = orc.block_rows(model, 0, x, new, 19, [(0, vc[0], kc[0])], rows)
+    assert np.max(np.abs(good - swapped)) > 1e-3
+    rolled, _, _ = orc.block_rows(model, 0, x, new, 19, [(0, np.roll(kc[0], 1, axis=0), np.roll(vc[0], 1, axis=0))], rows)
+    assert np.max(np.abs(good - rolled)) > 1e-4
