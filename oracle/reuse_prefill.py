@@ -163,6 +163,9 @@ class Prompt:
     chunk_len: Sequence[int]
     chunk_hidden: Sequence[Optional[np.ndarray]]      # float64 [len, d] or None (expected hit)
     query_hidden: np.ndarray                          # float64 [n_query, d]
+    # Prefix matching only (Appendix B, "Tokenization Inconsistency", second measure): the tensors of the last
+    # `tail_drop` tokens of the final matched node are discarded and those tokens are computed from their inputs.
+    tail_drop: int = 0
 
 
 @dataclass
@@ -238,10 +241,23 @@ def assemble_layout(store: Store, prompt: Prompt, match_prefix: bool = False) ->
             walking = False
             if prompt.chunk_hidden is None or i >= len(prompt.chunk_hidden) or prompt.chunk_hidden[i] is None:
                 raise MissNoInput(f"chunk {cid} missed and no hidden states were given")
+    # the final matched node keeps only its first chunk_len - tail_drop tokens (prefix matching only)
+    drop = int(getattr(prompt, "tail_drop", 0) or 0)
+    last_hit = int(np.nonzero(hit)[0][-1]) if hit.any() else -1
+    if drop:
+        if not match_prefix or drop < 0:
+            raise ValueError("tail_drop needs prefix matching and a non-negative count")
+        if last_hit >= 0:
+            if drop > prompt.chunk_len[last_hit]:
+                raise ValueError("tail_drop exceeds the length of the final matched chunk")
+            if prompt.chunk_hidden is None or last_hit >= len(prompt.chunk_hidden) or prompt.chunk_hidden[last_hit] is None:
+                raise MissNoInput("tail_drop needs the hidden states of the final matched chunk")
+    for i, n in enumerate(prompt.chunk_len):
+        reuse_len = n - drop if (i == last_hit and drop) else n
         for o in range(n):
             slot_chunk.append(i)
             slot_off.append(o)
-            is_new.append(0 if hit[i] else 1)
+            is_new.append(0 if (hit[i] and o < reuse_len) else 1)
     nq = 0 if prompt.query_hidden is None else prompt.query_hidden.shape[0]
     for o in range(nq):
         slot_chunk.append(n_chunks)
@@ -307,8 +323,9 @@ def reuse_prefill(model: Model, store: Store, prompts: Sequence[Prompt], commit:
             for i, (cid, n) in enumerate(zip(store_keys(prompt, match_prefix), prompt.chunk_len)):
                 if lay.hit_mask[i]:                                 # load and place in order
                     ck, cv = store.kv[cid]
-                    k_pre[start:start + n] = ck[l]
-                    v_all[start:start + n] = cv[l]
+                    reused = lay.slot_is_new[start:start + n] == 0      # all of the chunk unless its tail is dropped
+                    k_pre[start:start + n][reused] = ck[l][reused]
+                    v_all[start:start + n][reused] = cv[l][reused]
                 start += n
             k_rot = rope(k_pre, pos_all, model.rope_theta)          # every slot at its own position
             q_rot = rope(q, new, model.rope_theta)

@@ -518,3 +518,41 @@ def test_block_rows_hit_segment_placement_matters():
     assert np.max(np.abs(good - swapped)) > 1e-3
     rolled, _, _ = orc.block_rows(model, 0, x, new, 19, [(0, np.roll(kc[0], 1, axis=0), np.roll(vc[0], 1, axis=0))], rows)
     assert np.max(np.abs(good - rolled)) > 1e-4
+
+
+@pytest.mark.parametrize("drop", [0, 1, 5, 17])
+def test_prefix_reuse_with_the_tail_of_the_last_matched_chunk_recomputed(drop):
+    """Appendix B, tokenisation paragraph, second measure: the last few tokens of the final matched node are computed
+    from their inputs instead of being loaded.  Layout by hand; and since the recomputed rows see the same prefix,
+    the result still is plain full prefill."""
+    shape, weights, model = tiny_model(seed=38, n_layers=2)
+    lens, nq = [6, 17, 4], 5
+    hs, qh = _chunks(shape, 38, lens, nq)
+    full, _, _ = orc.dense_prefill(model, np.concatenate(hs + [qh]))
+    store = orc.Store()
+    orc.reuse_prefill(model, store, [orc.Prompt([100, 101], lens[:2], hs[:2], np.zeros((0, shape.d_model)))],
+                      match_prefix=True)
+    pr = orc.Prompt([100, 101, 102], lens, [None, hs[1], hs[2]], qh, tail_drop=drop)
+    res = orc.reuse_prefill(model, store, [pr], match_prefix=True, commit=False)[0]
+    lay = res.layout
+    assert lay.hit_mask.tolist() == [1, 1, 0]
+    l_pre = 6 + 17 - drop                                   # L_pre of Appendix B.1
+    assert lay.slot_is_new.tolist() == [0] * l_pre + [1] * (32 - l_pre)
+    assert lay.new_slots.tolist() == list(range(l_pre, 32))
+    assert lay.slot_chunk.tolist() == [0] * 6 + [1] * 17 + [2] * 4 + [3] * 5
+    assert np.allclose(res.out_hidden, full[l_pre:], atol=1e-9)
+
+
+def test_tail_drop_is_refused_outside_prefix_matching_and_without_inputs():
+    shape, weights, model = tiny_model(seed=39, n_layers=1)
+    hs, qh = _chunks(shape, 39, [8, 8], 2)
+    store = orc.Store()
+    orc.reuse_prefill(model, store, [orc.Prompt([1, 2], [8, 8], hs, np.zeros((0, shape.d_model)))], match_prefix=True)
+    with pytest.raises(orc.MissNoInput):
+        orc.reuse_prefill(model, store, [orc.Prompt([1, 2], [8, 8], [None, None], qh, tail_drop=3)], match_prefix=True)
+    with pytest.raises(ValueError):
+        orc.reuse_prefill(model, store, [orc.Prompt([1, 2], [8, 8], hs, qh, tail_drop=9)], match_prefix=True)
+    st2 = orc.Store()
+    orc.reuse_prefill(model, st2, [orc.Prompt([1, 2], [8, 8], hs, np.zeros((0, shape.d_model)))])
+    with pytest.raises(ValueError):
+        orc.reuse_prefill(model, st2, [orc.Prompt([1, 2], [8, 8], hs, qh, tail_drop=3)])
