@@ -80,6 +80,9 @@ extern "C" {
 #define PERCACHE_FLAG_EVICT_LFU          8u  /* when the store is full, evict least-frequently-used chunks instead
                                                 of failing with PERCACHE_E_NOSPACE (see percache_set_store_limit)  */
 
+#define PERCACHE_FLAG_PAPER_MODE         64u  /* creation only: the handle works exactly as the paper states the scheme
+                                                (see "Paper-faithful mode" below)                                 */
+
 typedef struct percache percache_t;   /* opaque */
 
 typedef struct {
@@ -147,6 +150,11 @@ typedef struct {
   const void* query_hidden;             /* bf16 [n_query][d_model]                                          */
   int32_t hidden_on_device;             /* 1: chunk_hidden[i] and query_hidden point to device memory       */
   int32_t match_mode;                   /* PERCACHE_MATCH_*                                                 */
+  int32_t reuse_tail_drop;              /* PERCACHE_MATCH_PREFIX_PATH only, else must be 0 (paper Appendix B,
+                                           tokenisation paragraph): the tensors of the last reuse_tail_drop tokens
+                                           of the final matched chunk are not reused; those tokens are computed
+                                           from chunk_hidden (which must then be given for that chunk) and are not
+                                           stored again.  0 <= drop <= that chunk's length                      */
 } percache_prompt_t;
 
 typedef struct {
@@ -166,6 +174,25 @@ typedef struct {
  * Synchronous: returns after the stream has drained. */
 PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
+
+/* Paper-faithful mode (a handle created with PERCACHE_FLAG_PAPER_MODE).  percache_prefill then computes what the
+ * paper describes, without the three departures listed at the top of this file:
+ *  - matching is the prefix-tree walk (every prompt must use PERCACHE_MATCH_PREFIX_PATH, Section 3.2.2);
+ *  - a node holds the chunk's Q, K and V of every block (Sections 3.2.1 and 5.3: all three projections are skipped
+ *    for cached rows), bf16, Q and K after position encoding at the positions the node has on its path;
+ *  - all L_total rows of the prompt run through every block; the L_pre rows of the matched chain skip only the
+ *    projections and the position encoding, for the others the position counter starts at L_pre (Appendix B.1);
+ *    reuse_tail_drop shortens L_pre by the tail of the chain's last node (Appendix B, tokenisation paragraph);
+ *  - out_hidden receives ALL n_total rows (out_capacity_rows >= n_total); n_new still counts the computed rows.
+ * Q, K (both rotated) and V of every row are rounded to bf16 before the attention uses them, loaded or computed
+ * alike, because that is what the store holds.  The attention reads Q, K and V of all rows straight from the pages
+ * through a per-prompt page table (nothing is gathered or rotated at query time).  Restrictions of this mode: hidden
+ * states must be given for every chunk (the whole prompt is embedded); chunk lengths and reuse_tail_drop must be
+ * multiples of 16 (pages are copied whole; the query may have any length); max_batch_new_rows bounds the rows of a
+ * batch, i.e. the sum of n_total; percache_put_chunk_kv, _put_chunk_synthetic and percache_decode return
+ * PERCACHE_E_INVAL; the debugging flags that select the plain kernels are refused.  percache_get_chunk_kv returns the
+ * node's K (rotated) and V, percache_get_chunk_q its Q: bf16 [n_layers][n_tokens][n_q_heads][head_dim], host. */
+PERCACHE_API int percache_get_chunk_q(percache_t* h, uint64_t chunk_id, void* q_host);
 
 /* Decode step after a prefill (paper Section 2.1: inference is a prefill over the prompt followed by a decode
  * stage that produces one token at a time, attending to the keys and values of everything before it).

@@ -216,7 +216,7 @@ decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* par
       L = fmaf(wgt, lv[u], L);
     }
   }
-  out[(static_cast<size_t>(mg.row) * n_q_heads + mg.kv_head * GROUP + h) * HEAD_DIM + d] = __float2half_rn(acc / L);
+  out[(static_cast<size_t>(mg.row) * n_q_heads + mg.kv_head * GROUP + h) * HEAD_DIM + d] = to_half_sat(acc / L);
 }
 
 }  // namespace

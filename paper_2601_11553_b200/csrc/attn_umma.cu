@@ -38,6 +38,7 @@ struct AttnArgs {
   const AttnItem* items;
   const int32_t* cta_first;
   const int32_t* row_pos;
+  const int32_t* page_table;      // PAGED: one page id per 16 context slots; an item's ctx0 indexes its prompt's first entry
   __half* out;
   float* partial_o;
   float* partial_ml;
@@ -59,6 +60,12 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return y;
 }
 
+// PAGED = false: Q from the query buffer, K and V from the assembled context, all fp16.
+// PAGED = true (paper-faithful mode): Q, K and V are read straight from the bf16 pages of the store through the
+// prompt's page table, one 16-row page per bulk copy (nothing is gathered into a contiguous context first, and K
+// needs no rotation because that mode caches it after position encoding); the MMAs then run on bf16 operands and
+// P is written to TMEM as bf16.  Everything else is the same kernel.
+template <bool PAGED>
 __global__ void __launch_bounds__(ATT_THREADS, 1)
 umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, AttnArgs args) {
@@ -117,7 +124,51 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   // An item's `unit` = g * pairs + pair covers query heads (g * group + 2 * pair, +1) and KV head g.
   const int pairs = group / 2;
 
-  if (warp == 8) {
+  if (warp == 8 && PAGED) {
+    // ---------------------------------------------------------------- TMA producer, paged: the whole warp works.
+    // A 128-row tile is eight pages; lane l copies page (l & 7) of 64-column half ((l >> 3) & 1) (and, for Q, of
+    // head (l >> 4)): 32 copies for a Q tile pair, 16 each for a K and a V block, all counted by one barrier.
+    uint32_t unit_it = 0, kvit = 0;
+    bool ok = true;
+    const int pg = lane & 7, hf = (lane >> 3) & 1;
+    for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
+      const AttnItem t = w == w_begin ? first_item : args.items[w];
+      const int gp = t.unit;
+      const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
+      const int nb = t.blk_end - t.blk_begin;
+      const int32_t* pt = args.page_table + t.ctx0;
+      // the tile's first row sits at a position that is a multiple of 128 (tiles start at a prompt's first row)
+      const int q_page = __ldg(pt + (__ldg(args.row_pos + t.row0) >> 4) + pg);
+      ok = mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { cta_failed = 1; break; }
+      if (lane == 0) mbar_arrive_expect_tx(&q_full, 2 * TILE_BYTES);
+      __syncwarp();
+      tma_load_2d(q_smem + (lane >> 4) * TILE_BYTES + hf * HALF_TILE_BYTES + pg * (PAGE_TOKENS * 128), &tmQ, &q_full,
+                  (h0 + (lane >> 4)) * HEAD_DIM + hf * 64, q_page * PAGE_TOKENS);
+      for (int j = 0; j < nb; ++j, ++kvit) {
+        const int st = kvit & 1;
+        const uint32_t ph = (kvit >> 1) & 1u;
+        const int kv_page = __ldg(pt + (t.blk_begin + j) * (BLK / PAGE_TOKENS) + pg);
+        ok = mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { cta_failed = 1; break; }
+        if (lane == 0) mbar_arrive_expect_tx(&k_full[st], TILE_BYTES);
+        __syncwarp();
+        if (lane < 16)
+          tma_load_2d(k_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES + pg * (PAGE_TOKENS * 128), &tmK, &k_full[st],
+                      g * HEAD_DIM + hf * 64, kv_page * PAGE_TOKENS);
+        ok = mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { cta_failed = 1; break; }
+        if (lane == 0) mbar_arrive_expect_tx(&v_full[st], TILE_BYTES);
+        __syncwarp();
+        if (lane < 16)
+          tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES + pg * (PAGE_TOKENS * 128), &tmV, &v_full[st],
+                      g * HEAD_DIM + hf * 64, kv_page * PAGE_TOKENS);
+      }
+    }
+  } else if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
       uint32_t unit_it = 0, kvit = 0;
@@ -153,8 +204,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   } else if (warp == 9) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, 0, 0, 0);        // A, B K-major
-      constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, 0, 0, 1);   // B (V) MN-major
+      constexpr int AB = PAGED ? 1 : 0;                                       // operand type: 0 fp16, 1 bf16
+      constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, AB, 0, 0);       // A, B K-major
+      constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, AB, 0, 1);  // B (V) MN-major
       uint32_t unit_it = 0, kvit = 0;
       bool ok = true;
       // S_i(kvidx) = Q_i K(kvidx)^T
@@ -294,8 +346,13 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), args.scale_log2, neg_m));
           sum0 += p0;
           sum1 += p1;
-          __half2 hh = __floats2half2_rn(p0, p1);
-          p[c] = *reinterpret_cast<uint32_t*>(&hh);
+          if constexpr (PAGED) {            // P in the operand type of V
+            __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
+            p[c] = *reinterpret_cast<uint32_t*>(&bb);
+          } else {
+            __half2 hh = __floats2half2_rn(p0, p1);
+            p[c] = *reinterpret_cast<uint32_t*>(&hh);
+          }
         }
         const float sum = sum0 + sum1;
         l += sum;
@@ -325,11 +382,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             for (int e = 0; e < 4; ++e) {
               uint32_t pk[4];
 #pragma unroll
-              for (int q = 0; q < 4; ++q) {
-                __half2 hh = __floats2half2_rn(__uint_as_float(o[8 * e + 2 * q]) * inv_l,
-                                               __uint_as_float(o[8 * e + 2 * q + 1]) * inv_l);
-                pk[q] = *reinterpret_cast<uint32_t*>(&hh);
-              }
+              for (int q = 0; q < 4; ++q)     // saturating: P is rounded but the row sum is not, so a quotient of
+                                              // values at the fp16 limit can land just beyond it
+                pk[q] = pack_half2(__uint_as_float(o[8 * e + 2 * q]) * inv_l, __uint_as_float(o[8 * e + 2 * q + 1]) * inv_l);
               *reinterpret_cast<uint4*>(dst + c * 32 + e * 8) = make_uint4(pk[0], pk[1], pk[2], pk[3]);
             }
           }
@@ -453,10 +508,8 @@ attention_merge_kernel(const AttnMerge* __restrict__ merges, const float* partia
 #pragma unroll
   for (int k = 0; k < MERGE_ROWS; ++k) {
     if (r0 + k >= mg.n_rows) break;
-    __half2 a = __floats2half2_rn(acc[k].x * inv[k], acc[k].y * inv[k]);
-    __half2 b = __floats2half2_rn(acc[k].z * inv[k], acc[k].w * inv[k]);
     *reinterpret_cast<uint2*>(out + (static_cast<size_t>(mg.row0 + r0 + k) * n_q_heads + head) * HEAD_DIM + lane * 4) =
-        make_uint2(*reinterpret_cast<uint32_t*>(&a), *reinterpret_cast<uint32_t*>(&b));
+        make_uint2(pack_half2(acc[k].x * inv[k], acc[k].y * inv[k]), pack_half2(acc[k].z * inv[k], acc[k].w * inv[k]));
   }
 }
 }  // namespace
@@ -469,28 +522,48 @@ void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* 
              n_kv_heads);
 }
 
+int make_paged_attn_maps(AttnMaps* out, const __nv_bfloat16* qpool_layer, const __nv_bfloat16* kpool_layer,
+                         const __nv_bfloat16* vpool_layer, int64_t pool_pages, int q_dim, int kv_dim) {
+  // one page (16 rows) of a 64-column half per copy; the element type only matters for out-of-range fill, which
+  // never happens here (page ids and columns are always inside the pool)
+  const uint32_t box[2] = {64u, static_cast<uint32_t>(PAGE_TOKENS)};
+  const uint64_t rows = static_cast<uint64_t>(pool_pages) * PAGE_TOKENS;
+  const uint64_t qd[2] = {static_cast<uint64_t>(q_dim), rows}, qs[1] = {static_cast<uint64_t>(q_dim) * 2};
+  const uint64_t kd[2] = {static_cast<uint64_t>(kv_dim), rows}, ks[1] = {static_cast<uint64_t>(kv_dim) * 2};
+  if (encode_f16_map(&out->q, qpool_layer, 2, qd, qs, box) != 0) return -1;
+  if (encode_f16_map(&out->k, kpool_layer, 2, kd, ks, box) != 0) return -1;
+  if (encode_f16_map(&out->v, vpool_layer, 2, kd, ks, box) != 0) return -1;
+  return 0;
+}
+
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
-                          int n_kv_heads, int* err_word, cudaStream_t s) {
+                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table) {
   if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0) return -1;
-  static bool smem_set[MAX_DEVICES] = {};      // once per device: the call costs host time on every launch otherwise
+  const bool paged = page_table != nullptr;
+  static bool smem_set[2][MAX_DEVICES] = {};   // once per device: the call costs host time on every launch otherwise
   const int dev = current_device_slot();
-  if (!smem_set[dev]) {
-    if (cudaFuncSetAttribute(umma_attention_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES) !=
-        cudaSuccess)
-      return -1;
-    smem_set[dev] = true;
+  if (!smem_set[paged][dev]) {
+    const cudaError_t e = paged ? cudaFuncSetAttribute(umma_attention_kernel<true>,
+                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
+                                : cudaFuncSetAttribute(umma_attention_kernel<false>,
+                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
+    if (e != cudaSuccess) return -1;
+    smem_set[paged][dev] = true;
   }
   AttnArgs a{};
-  a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out;
+  a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out; a.page_table = page_table;
   a.partial_o = partial_o; a.partial_ml = partial_ml;
   a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
   a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
   a.err_word = err_word;
-  return launch_pdl(umma_attention_kernel, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v,
-                    a) == cudaSuccess ? 0 : -1;
+  if (paged)
+    return launch_pdl(umma_attention_kernel<true>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k,
+                      maps.v, a) == cudaSuccess ? 0 : -1;
+  return launch_pdl(umma_attention_kernel<false>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k,
+                    maps.v, a) == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace pc

@@ -3,6 +3,7 @@
 // (called from a separate kernel on an fp32 matrix), so both produce identical bytes from identical sums.
 #pragma once
 #include "kernels.h"
+#include "ptx.cuh"
 
 namespace pc {
 
@@ -10,19 +11,6 @@ namespace pc {
 // rounded to fp16 right after, and the division was a third of the SwiGLU epilogue's time
 __device__ __forceinline__ float silu_f(float x) { return __fdividef(x, 1.0f + __expf(-x)); }
 
-// Two floats to packed fp16 (a in the low half), round to nearest even, SATURATING: a magnitude beyond the
-// largest finite fp16 value (65504) becomes +-65504 instead of infinity (NaN stays NaN).  Every fp16 operand the
-// library forms goes through this conversion, so an out-of-range activation or cached bf16 value clips instead
-// of turning into inf and, one masked product later, NaN.
-__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
-  uint32_t r;
-  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));   // first source -> upper half
-  return r;
-}
-__device__ __forceinline__ __half to_half_sat(float a) {
-  const uint32_t r = pack_half2(a, 0.f);
-  return __ushort_as_half(static_cast<unsigned short>(r & 0xffffu));
-}
 __device__ __forceinline__ uint32_t pack_bf162(__nv_bfloat16 a, __nv_bfloat16 b) {
   __nv_bfloat162 h(a, b);
   return *reinterpret_cast<uint32_t*>(&h);
@@ -67,6 +55,24 @@ __device__ __forceinline__ void qkv_store4_cs(const QkvEpilogue& e, int row, con
   const bool is_q = hb < e.n_q_heads;
   const bool is_k = !is_q && hb < e.n_q_heads + e.n_kv_heads;
   const float4 t0 = cs.t0, t1 = cs.t1;
+  if (e.paged) {
+    // Paper-faithful mode (Section 3.2.1: the Q, K and V tensors of the attention module are what is collected;
+    // Appendix B.1: position encoding with the counter offset by the cached length): rotate Q and K to the row's
+    // position, round everything to bf16 and write it to the row's page slot.  The identity table entries make the
+    // same arithmetic a plain copy for V.
+    const int q_dim = e.n_q_heads * HEAD_DIM, kv_dim2 = e.n_kv_heads * HEAD_DIM;
+    __nv_bfloat16* dst = is_q ? e.qpool + static_cast<size_t>(rw.pool_tok) * q_dim + hb * HEAD_DIM + c
+                              : (is_k ? e.kpool + static_cast<size_t>(rw.pool_tok) * kv_dim2 + (hb - e.n_q_heads) * HEAD_DIM + c
+                                      : e.vpool + static_cast<size_t>(rw.pool_tok) * kv_dim2 +
+                                            (hb - e.n_q_heads - e.n_kv_heads) * HEAD_DIM + c);
+    *reinterpret_cast<uint2*>(dst) =
+        make_uint2(pack_bf162(__float2bfloat16_rn(lo.x * t0.x - hi.x * t0.y), __float2bfloat16_rn(lo.y * t0.z - hi.y * t0.w)),
+                   pack_bf162(__float2bfloat16_rn(lo.z * t1.x - hi.z * t1.y), __float2bfloat16_rn(lo.w * t1.z - hi.w * t1.w)));
+    *reinterpret_cast<uint2*>(dst + ROPE_HALF) =
+        make_uint2(pack_bf162(__float2bfloat16_rn(hi.x * t0.x + lo.x * t0.y), __float2bfloat16_rn(hi.y * t0.z + lo.y * t0.w)),
+                   pack_bf162(__float2bfloat16_rn(hi.z * t1.x + lo.z * t1.y), __float2bfloat16_rn(hi.w * t1.z + lo.w * t1.w)));
+    return;
+  }
   if (is_q) {
     __half* dst = e.q_out + static_cast<size_t>(row) * (e.n_q_heads * HEAD_DIM) + hb * HEAD_DIM + c;
     *reinterpret_cast<uint2*>(dst) = pack_half4(lo.x * t0.x - hi.x * t0.y, lo.y * t0.z - hi.y * t0.w,

@@ -94,7 +94,9 @@ void launch_bf16_to_f16(const __nv_bfloat16* src, __half* dst, int64_t n, cudaSt
 void launch_interleave_rows_bf16_to_f16(const __nv_bfloat16* gate, const __nv_bfloat16* up, __half* dst, int rows,
                                         int cols, int blk, cudaStream_t s);
 void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStream_t s);
-void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s);
+// out row r = norm of x row (row_index ? row_index[r] : r); row_index is host-written before the call's first kernel
+void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s,
+                    const int32_t* row_index = nullptr);
 void launch_gather_rerope(const GatherItem* items, int n_items, int n_layers, const __nv_bfloat16* kpool,
                           const __nv_bfloat16* vpool, int64_t pool_pages, __half* kctx, __half* vctx,
                           int64_t ctx_cap, int kv_dim, const float2* rope, cudaStream_t s);
@@ -115,6 +117,10 @@ struct QkvEpilogue {
   __half* kctx;               // layer base: [ctx_cap][kv_dim]
   __half* vctx;
   int32_t n_q_heads, n_kv_heads;
+  // Paper-faithful mode: every row owns a page slot (rows.pool_tok >= 0) and Q, K, V all go to pages as bf16, Q and K
+  // after rotation (what the attention uses and what the cache then holds); q_out, kctx, vctx are unused.
+  __nv_bfloat16* qpool;       // layer base: [pool_pages*16][q_dim], or nullptr outside that mode
+  int32_t paged;
 };
 struct ResidualEpilogue { float* resid; int32_t ld; };          // resid[row][col] += acc
 struct SwigluEpilogue { __half* act; int32_t ld; };             // act[row][j] = silu(gate) * up
@@ -165,7 +171,12 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
 // CTA c (of n_ctas) runs items [cta_first[c], cta_first[c + 1]).
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
-                          int n_kv_heads, int* err_word, cudaStream_t s);
+                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table = nullptr);
+// Maps for the paged form of the attention (paper-faithful mode): Q, K and V are read straight from the bf16 pages
+// of one layer, 16 rows (one page) per bulk copy; an item's ctx0 then is the index of its prompt's first entry in
+// page_table (one page id per 16 context slots, padded to whole 128-slot blocks).
+int make_paged_attn_maps(AttnMaps* out, const __nv_bfloat16* qpool_layer, const __nv_bfloat16* kpool_layer,
+                         const __nv_bfloat16* vpool_layer, int64_t pool_pages, int q_dim, int kv_dim);
 void launch_attention_merge(const AttnMerge* merges, int n_merges, const float* partial_o, const float* partial_ml,
                             __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
 

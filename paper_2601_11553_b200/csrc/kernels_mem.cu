@@ -75,7 +75,8 @@ void launch_bf16_to_f32(const __nv_bfloat16* src, float* dst, int64_t n, cudaStr
 // are issued before the first is used.
 template <int VPL>
 __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* x, const float* __restrict__ gain,
-                                                      __half* __restrict__ out, int M, int d, float eps) {
+                                                      __half* __restrict__ out, int M, int d, float eps,
+                                                      const int32_t* __restrict__ row_index) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
   const int nv = d >> 2;
@@ -87,9 +88,11 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* x, const floa
     const int i = lane + 32 * k;
     g[k] = i < nv ? __ldg(reinterpret_cast<const float4*>(gain) + i) : make_float4(0.f, 0.f, 0.f, 0.f);
   }
+  // which row of x this output row normalises (a host-written list, or the same row)
+  const int src_row = (row_index != nullptr && row < M) ? __ldg(row_index + row) : row;
   pdl_wait();
   if (row >= M) return;
-  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(src_row) * d);
   float4 v[VPL];
 #pragma unroll
   for (int k = 0; k < VPL; ++k) {
@@ -113,13 +116,15 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(const float* x, const floa
 }
 // Rows of any length: two passes over global memory.
 __global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* x, const float* __restrict__ gain,
-                                                           __half* __restrict__ out, int M, int d, float eps) {
+                                                           __half* __restrict__ out, int M, int d, float eps,
+                                                           const int32_t* __restrict__ row_index) {
   const int row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   pdl_launch_dependents();
   pdl_wait();
   if (row >= M) return;
   const int lane = threadIdx.x & 31;
-  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(row) * d);
+  const int src_row = row_index != nullptr ? __ldg(row_index + row) : row;
+  const float4* xr = reinterpret_cast<const float4*>(x + static_cast<size_t>(src_row) * d);
   const int nv = d >> 2;
   float ss = 0.f;
   for (int i = lane; i < nv; i += 32) {
@@ -137,12 +142,13 @@ __global__ void __launch_bounds__(256) rmsnorm_long_kernel(const float* x, const
     o2[i] = pack_half4(v.x * inv * g.x, v.y * inv * g.y, v.z * inv * g.z, v.w * inv * g.w);
   }
 }
-void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s) {
+void launch_rmsnorm(const float* x, const float* gain, __half* out, int M, int d, float eps, cudaStream_t s,
+                    const int32_t* row_index) {
   if (M <= 0) return;
   const dim3 grid((M + 7) / 8), block(256);
-  if (d <= 1024) launch_pdl(rmsnorm_kernel<8>, grid, block, 0, s, x, gain, out, M, d, eps);
-  else if (d <= 2048) launch_pdl(rmsnorm_kernel<16>, grid, block, 0, s, x, gain, out, M, d, eps);
-  else launch_pdl(rmsnorm_long_kernel, grid, block, 0, s, x, gain, out, M, d, eps);
+  if (d <= 1024) launch_pdl(rmsnorm_kernel<8>, grid, block, 0, s, x, gain, out, M, d, eps, row_index);
+  else if (d <= 2048) launch_pdl(rmsnorm_kernel<16>, grid, block, 0, s, x, gain, out, M, d, eps, row_index);
+  else launch_pdl(rmsnorm_long_kernel, grid, block, 0, s, x, gain, out, M, d, eps, row_index);
 }
 
 // ------------------------------------------------------------------------------------------------

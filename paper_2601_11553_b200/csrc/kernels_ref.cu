@@ -159,7 +159,7 @@ ref_attention_kernel(const __half* __restrict__ q, const __half* __restrict__ kc
     m_run = m_new;
     __syncthreads();
   }
-  out[(static_cast<size_t>(row) * n_q_heads + h) * HEAD_DIM + tid] = __float2half_rn(acc / l_run);
+  out[(static_cast<size_t>(row) * n_q_heads + h) * HEAD_DIM + tid] = to_half_sat(acc / l_run);
 }
 void launch_ref_attention(const __half* q, const __half* kctx, const __half* vctx, __half* out, const int32_t* row_pos,
                           const int32_t* row_ctx0, int M, int n_q_heads, int n_kv_heads, cudaStream_t s) {

@@ -29,6 +29,7 @@ struct LayerWeights {
   GemmOperand m_wqkv, m_wo, m_wgu, m_wd;                  // B maps with 128-row boxes
   GemmOperand m_wqkv256, m_wo256, m_wgu256, m_wd256;      // and with 256-row boxes
   AttnMaps attn_maps;
+  AttnMaps paged_maps;                                    // paper-faithful mode: Q, K, V pages of this layer
 };
 
 struct Plan {   // integer description of the last successful call (host)
@@ -63,6 +64,8 @@ struct percache {
   std::vector<LayerWeights> layers;
   float2* rope = nullptr;
   __nv_bfloat16 *kpool = nullptr, *vpool = nullptr;    // [L][pool_pages][16][kv_dim]
+  __nv_bfloat16* qpool = nullptr;                       // paper-faithful mode only: [L][pool_pages][16][q_dim]
+  bool paper_mode = false;
   __half *kctx = nullptr, *vctx = nullptr;              // [L][ctx_cap][kv_dim]
   float* resid = nullptr;                               // [m_cap][d]
   __nv_bfloat16* xin = nullptr;                         // [m_cap][d]
@@ -335,7 +338,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
       timer.end();
     }
 
-    QkvEpilogue qe;
+    QkvEpilogue qe{};
     qe.rows = RowIndex{d_row_slot, d_row_pos, d_row_pool};
     qe.rope = h->rope;
     qe.q_out = h->qbuf;
@@ -441,6 +444,324 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   return ok;
 }
 
+
+// ---------------------------------------------------------------------------------------------------------------
+// Paper-faithful mode (PERCACHE_FLAG_PAPER_MODE): the scheme as the paper states it.  The chunk list is matched as a
+// path of the cache tree (Section 3.2.2); a node holds the chunk's Q, K and V of every block, Q and K after position
+// encoding (Sections 3.2.1, 5.3); all L_total rows of the prompt go through every block and only the rows of the
+// matched chain (L_pre of them, less the dropped tail of its last node) skip the three projections and the position
+// encoding (Appendix B.1).  Every row of the prompt owns a page slot (rows that are not chunk content, i.e. query
+// tokens and a recomputed tail, get scratch pages for the duration of the call), the QKV epilogue writes pages only,
+// and the attention reads Q, K and V through the prompt's page table: nothing is gathered or rotated.
+// ---------------------------------------------------------------------------------------------------------------
+int prefill_paper(percache* h, const percache_prompt_t* prompts, int32_t n_prompts, percache_result_t* results) {
+  const auto t_host0 = std::chrono::steady_clock::now();
+  const ModelDims& D = h->dims;
+  const int d = D.d_model;
+  if (h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION)) return PERCACHE_E_INVAL;
+
+  // ---------------------------------------------------------------- match the chains, sizes
+  std::vector<std::vector<uint64_t>> keys(n_prompts);
+  std::vector<std::vector<uint8_t>> hit(n_prompts);
+  std::vector<int> n_match(n_prompts, 0), l_pre(n_prompts, 0);
+  std::unordered_map<uint64_t, std::pair<int, int>> first_miss;
+  std::unordered_map<uint64_t, int64_t> hit_uses;
+  Plan plan;
+  plan.cu_ctx.assign(1, 0);
+  plan.cu_new.assign(1, 0);
+  int64_t rows_total = 0, new_total = 0, hit_tokens = 0, pages_needed = 0, pt_entries = 0, visible_pairs = 0;
+  int chunks_hit = 0, chunks_missed = 0;
+  for (int b = 0; b < n_prompts; ++b) {
+    const percache_prompt_t& P = prompts[b];
+    if (P.n_chunks < 0 || P.n_query < 0 || (P.n_chunks > 0 && (!P.chunk_ids || !P.chunk_len)) ||
+        (P.n_query > 0 && !P.query_hidden) || P.match_mode != PERCACHE_MATCH_PREFIX_PATH || P.reuse_tail_drop < 0 ||
+        P.reuse_tail_drop % PAGE_TOKENS != 0)
+      return PERCACHE_E_INVAL;
+    keys[b].resize(static_cast<size_t>(P.n_chunks));
+    hit[b].assign(static_cast<size_t>(P.n_chunks), 0);
+    uint64_t path = PATH_KEY_SEED;
+    bool walking = true;
+    int64_t T = 0;
+    for (int i = 0; i < P.n_chunks; ++i) {
+      const int len = P.chunk_len[i];
+      if (len <= 0 || len % PAGE_TOKENS != 0) return PERCACHE_E_INVAL;     // pages are copied whole in this mode
+      if (!P.chunk_hidden || !P.chunk_hidden[i]) return PERCACHE_E_MISS_NO_INPUT;   // the whole prompt is embedded
+      path = path_key_step(path, P.chunk_ids[i]);
+      keys[b][i] = path;
+      auto it = h->table.find(path);
+      const bool stored = it != h->table.end();
+      if (stored && it->second.n_tokens != len) return PERCACHE_E_LEN_MISMATCH;
+      if (stored && walking) {
+        hit[b][i] = 1;
+        n_match[b] = i + 1;
+        l_pre[b] += len;
+        ++chunks_hit;
+        ++hit_uses[path];
+      } else {
+        walking = false;
+        ++chunks_missed;
+        // the first prompt that computes a node keeps it; any other computation of it lives in scratch pages
+        if (!stored && !first_miss.count(path)) first_miss.emplace(path, std::make_pair(b, i));
+        pages_needed += len / PAGE_TOKENS;
+      }
+      T += len;
+    }
+    if (n_match[b] > 0) {
+      if (P.reuse_tail_drop > P.chunk_len[n_match[b] - 1]) return PERCACHE_E_INVAL;
+      l_pre[b] -= P.reuse_tail_drop;
+      pages_needed += P.reuse_tail_drop / PAGE_TOKENS;
+    }
+    pages_needed += (P.n_query + PAGE_TOKENS - 1) / PAGE_TOKENS;
+    T += P.n_query;
+    if (T <= 0) return PERCACHE_E_INVAL;
+    if (T > h->cfg.max_prompt_tokens) return PERCACHE_E_CAPACITY;
+    if (results[b].out_capacity_rows < T || !results[b].out_hidden) return PERCACHE_E_CAPACITY;   // all rows come back
+    hit_tokens += l_pre[b];
+    rows_total += T;
+    new_total += T - l_pre[b];
+    pt_entries += (T + 127) / 128 * (128 / PAGE_TOKENS);
+    if (rows_total > h->m_cap || rows_total > h->ctx_cap) return PERCACHE_E_CAPACITY;
+    plan.cu_ctx.push_back(static_cast<int32_t>(rows_total));
+    plan.cu_new.push_back(static_cast<int32_t>(new_total));
+  }
+  if (static_cast<size_t>(pt_entries) > 4 * static_cast<size_t>(h->ctx_cap)) return PERCACHE_E_CAPACITY;
+
+  PageTxn txn(h);
+  {
+    std::vector<uint64_t> victims;
+    const int rc = pick_victims(h, pages_needed, hit_uses, &victims);
+    if (rc < 0) return rc;
+    txn.set_victims(victims);
+  }
+  const int evicted = static_cast<int>(txn.victims.size());
+  std::vector<std::pair<uint64_t, ChunkEntry>> pending;
+  std::vector<int32_t> scratch;                   // pages that only live for this call
+  auto fail = [&](int code) {
+    if (txn.applied) h->plan = Plan();
+    txn.undo();
+    refresh_page_stats(h);
+    return code;
+  };
+
+  // ---------------------------------------------------------------- index assembly
+  const int64_t M = rows_total, M_new = new_total;
+  int32_t* row_src = h->h_index;                  // new row -> row of the residual stream (its global row)
+  int32_t* row_pos = row_src + h->m_cap;          // new row -> position
+  int32_t* row_pool = row_pos + h->m_cap;         // new row -> page * 16 + offset
+  int32_t* pos_all = row_pool + h->m_cap;         // global row -> position
+  int32_t* page_table = pos_all + h->m_cap;       // in place of the gather items
+  AttnItem* attn_items = reinterpret_cast<AttnItem*>(page_table + 4 * h->ctx_cap);
+  int32_t* cta_first = reinterpret_cast<int32_t*>(attn_items) + 8 * h->max_attn_items;
+  AttnMerge* merges = reinterpret_cast<AttnMerge*>(cta_first + h->n_sms + 1);
+  struct Seg { const void* src; int on_device; int row0; int n; };
+  std::vector<Seg> segs;
+  std::vector<AttnBaseTile> base_tiles;
+  plan.slot_chunk.resize(static_cast<size_t>(M));
+  plan.slot_offset.resize(static_cast<size_t>(M));
+  plan.slot_is_new.resize(static_cast<size_t>(M));
+  plan.row_slot.resize(static_cast<size_t>(M_new));
+  int64_t r = 0;
+  int32_t pt_next = 0;
+  for (int b = 0; b < n_prompts; ++b) {
+    const percache_prompt_t& P = prompts[b];
+    const int32_t g0 = plan.cu_ctx[b];
+    const int32_t T = plan.cu_ctx[b + 1] - g0;
+    const int32_t pt0 = pt_next;
+    plan.ctx0.push_back(g0);
+    plan.dec_len.push_back(0);
+    int32_t t = 0;
+    for (int i = 0; i <= P.n_chunks; ++i) {
+      const bool is_query = (i == P.n_chunks);
+      const int len = is_query ? P.n_query : P.chunk_len[i];
+      if (len == 0) continue;
+      const bool is_hit = !is_query && hit[b][i];
+      const int reuse_len = !is_hit ? 0 : len - (i == n_match[b] - 1 ? P.reuse_tail_drop : 0);
+      // pages of this stretch of slots: the stored node's, new ones that will become a node, or scratch
+      std::vector<int32_t> fresh;
+      const std::vector<int32_t>* stored_pages = nullptr;
+      bool keep = false;
+      if (is_hit) stored_pages = &h->table.find(keys[b][i])->second.pages;
+      if (!is_query && !is_hit) {
+        auto fm = first_miss.find(keys[b][i]);
+        keep = fm != first_miss.end() && fm->second.first == b && fm->second.second == i;
+      }
+      const int n_fresh = (len - reuse_len + PAGE_TOKENS - 1) / PAGE_TOKENS;
+      if (n_fresh > 0 && txn.take(n_fresh, &fresh) != PERCACHE_OK) return fail(PERCACHE_E_NOSPACE);
+      if (keep) {
+        ChunkEntry ent;
+        ent.n_tokens = len;
+        ent.serial = h->next_serial++;
+        ent.pages = fresh;
+        pending.emplace_back(keys[b][i], std::move(ent));
+      } else {
+        scratch.insert(scratch.end(), fresh.begin(), fresh.end());
+      }
+      for (int o = 0; o < len; o += PAGE_TOKENS)
+        page_table[pt_next++] = o < reuse_len ? (*stored_pages)[o / PAGE_TOKENS] : fresh[(o - reuse_len) / PAGE_TOKENS];
+      segs.push_back(Seg{is_query ? P.query_hidden : P.chunk_hidden[i], P.hidden_on_device, g0 + t, len});
+      for (int o = 0; o < len; ++o) {
+        plan.slot_chunk[g0 + t + o] = i;
+        plan.slot_offset[g0 + t + o] = o;
+        plan.slot_is_new[g0 + t + o] = o < reuse_len ? 0 : 1;
+        pos_all[g0 + t + o] = t + o;
+        visible_pairs += t + o + 1;
+        if (o >= reuse_len) {
+          row_src[r] = g0 + t + o;
+          row_pos[r] = t + o;
+          row_pool[r] = fresh[(o - reuse_len) / PAGE_TOKENS] * PAGE_TOKENS + ((o - reuse_len) % PAGE_TOKENS);
+          plan.row_slot[r] = t + o;
+          ++r;
+        }
+      }
+      t += len;
+    }
+    // pad the prompt's table to whole 128-slot blocks with its last page (those slots are never visible)
+    const int32_t last_page = page_table[pt_next - 1];
+    while ((pt_next - pt0) % (128 / PAGE_TOKENS) != 0) page_table[pt_next++] = last_page;
+    for (int32_t r0 = 0; r0 < T; r0 += 128) {
+      AttnBaseTile a{};
+      a.row0 = g0 + r0;
+      a.n_rows = std::min(128, T - r0);
+      a.ctx0 = pt0;                                   // the paged attention reads ctx0 as the table offset
+      a.n_blocks = (r0 + a.n_rows + 127) / 128;
+      base_tiles.push_back(a);
+    }
+  }
+  int n_attn_ctas = 0, n_merges = 0;
+  {
+    std::vector<AttnItem> v_items;
+    std::vector<int32_t> v_first;
+    std::vector<AttnMerge> v_merges;
+    plan_attention(base_tiles, D.n_kv_heads * (D.n_q_heads / D.n_kv_heads / 2), h->n_sms, h->partial_slots, &v_items,
+                   &v_first, &v_merges);
+    if (v_items.size() > h->max_attn_items || v_merges.size() > h->max_attn_merges ||
+        v_first.size() > static_cast<size_t>(h->n_sms) + 1)
+      return fail(PERCACHE_E_CAPACITY);
+    std::copy(v_items.begin(), v_items.end(), attn_items);
+    std::fill(cta_first, cta_first + h->n_sms + 1, static_cast<int32_t>(v_items.size()));
+    std::copy(v_first.begin(), v_first.end(), cta_first);
+    std::copy(v_merges.begin(), v_merges.end(), merges);
+    n_attn_ctas = static_cast<int>(v_first.size()) - 1;
+    n_merges = static_cast<int>(v_merges.size());
+  }
+  const double plan_us =
+      std::chrono::duration<double, std::micro>(std::chrono::steady_clock::now() - t_host0).count();
+
+  // ---------------------------------------------------------------- device work
+  cudaStream_t s = h->stream;
+  percache_stats_t& st = h->stats;
+  std::memset(st.phase_us, 0, sizeof(st.phase_us));
+  std::memset(st.phase_launches, 0, sizeof(st.phase_launches));
+  PhaseTimer timer(h);
+  bool ok = true;
+  txn.apply();
+  const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(merges + n_merges) - h->h_index);
+  ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
+  const DevIndex ix = dev_index(h);
+  const int32_t* d_page_table = reinterpret_cast<const int32_t*>(ix.items);
+  timer.begin(PERCACHE_PH_IO);
+  for (const Seg& sg : segs)
+    ok = ok && cudaMemcpyAsync(h->xin + static_cast<size_t>(sg.row0) * d, sg.src, static_cast<size_t>(sg.n) * d * 2,
+                               sg.on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s) == cudaSuccess;
+  cudaEventRecord(h->ev_begin, s);
+  launch_bf16_to_f32(h->xin, h->resid, M * d, s);
+  timer.end();
+
+  const int Mi = static_cast<int>(M), Mn = static_cast<int>(M_new);
+  const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS;
+  const bool may_pair = !(h->flags & PERCACHE_FLAG_SINGLE_CTA_GEMM);
+  auto gemm = [&](const GemmOperand& A, const GemmOperand& B128, const GemmOperand& B256, int rows, int N, int K,
+                  GemmEpilogueKind kind, const void* epi, bool residual) {
+    int bn, ks, pr;
+    umma_gemm_pick_shape(rows, N, K, h->n_sms, residual, may_pair, &bn, &ks, &pr);
+    return launch_umma_gemm(A, (bn == 256 && !pr) ? B256 : B128, rows, N, K, bn, kind, epi, nullptr, h->d_err, h->n_sms, s,
+                            ks, pr) == 0;
+  };
+  for (int l = 0; l < D.n_layers && ok; ++l) {
+    LayerWeights& W = h->layers[l];
+    if (Mn > 0) {       // projections and position encoding on the rows the loaded tensors do not cover
+      timer.begin(PERCACHE_PH_NORM);
+      launch_rmsnorm(h->resid, W.g_attn, h->xn, Mn, d, D.rms_eps, s, ix.row_slot);
+      timer.end();
+      QkvEpilogue qe{};
+      qe.rows = RowIndex{ix.row_slot, ix.row_pos, ix.row_pool};
+      qe.rope = h->rope;
+      qe.qpool = h->qpool + l * pool_layer * D.q_dim;
+      qe.kpool = h->kpool + l * pool_layer * D.kv_dim;
+      qe.vpool = h->vpool + l * pool_layer * D.kv_dim;
+      qe.n_q_heads = D.n_q_heads;
+      qe.n_kv_heads = D.n_kv_heads;
+      qe.paged = 1;
+      timer.begin(PERCACHE_PH_QKV);
+      ok = ok && gemm(h->m_xn, W.m_wqkv, W.m_wqkv256, Mn, D.qkv_dim, d, EPI_QKV, &qe, false);
+      timer.end();
+    }
+    // loaded and computed tensors side by side in the pages: the sequence is L_total rows long again
+    timer.begin(PERCACHE_PH_ATTN);
+    ok = ok && launch_umma_attention(W.paged_maps, ix.attn_items, ix.cta_first, n_attn_ctas, ix.row_ctx0, h->attn_out,
+                                     h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s,
+                                     d_page_table) == 0;
+    launch_attention_merge(ix.merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
+    timer.end();
+    ResidualEpilogue re{h->resid, d};
+    timer.begin(PERCACHE_PH_OPROJ);
+    ok = ok && gemm(h->m_attn, W.m_wo, W.m_wo256, Mi, d, D.q_dim, EPI_RESIDUAL, &re, true);
+    timer.end();
+    timer.begin(PERCACHE_PH_NORM);
+    launch_rmsnorm(h->resid, W.g_ffn, h->xn, Mi, d, D.rms_eps, s);
+    timer.end();
+    SwigluEpilogue se{h->act, D.d_ffn};
+    timer.begin(PERCACHE_PH_GATEUP);
+    ok = ok && gemm(h->m_xn, W.m_wgu, W.m_wgu256, Mi, 2 * D.d_ffn, d, EPI_SWIGLU, &se, false);
+    timer.end();
+    timer.begin(PERCACHE_PH_DOWN);
+    ok = ok && gemm(h->m_act, W.m_wd, W.m_wd256, Mi, d, D.d_ffn, EPI_RESIDUAL, &re, true);
+    timer.end();
+  }
+  cudaEventRecord(h->ev_end, s);
+  timer.begin(PERCACHE_PH_IO);
+  for (int b = 0; b < n_prompts && ok; ++b) {
+    const int T = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+    ok = ok && cudaMemcpyAsync(results[b].out_hidden, h->resid + static_cast<size_t>(plan.cu_ctx[b]) * d,
+                               static_cast<size_t>(T) * d * sizeof(float),
+                               results[b].out_on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  }
+  ok = ok && cudaMemcpyAsync(h->h_err, h->d_err, sizeof(int), cudaMemcpyDeviceToHost, s) == cudaSuccess;
+  timer.end();
+  const cudaError_t sync_rc = cudaStreamSynchronize(s);
+  if (!ok || sync_rc != cudaSuccess || cudaGetLastError() != cudaSuccess) return fail(PERCACHE_E_CUDA);
+  if (*h->h_err != 0) return fail(PERCACHE_E_DEVICE_TIMEOUT);
+
+  // ---------------------------------------------------------------- commit
+  for (auto& pe : pending) h->table.emplace(pe.first, std::move(pe.second));
+  for (const auto& hu : hit_uses) h->table[hu.first].retrievals += hu.second;
+  release_pages(h, scratch);
+  st.evictions = evicted;
+  for (int b = 0; b < n_prompts; ++b) {
+    results[b].n_total = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+    results[b].n_new = plan.cu_new[b + 1] - plan.cu_new[b];
+    if (results[b].hit_mask && prompts[b].n_chunks > 0)
+      std::memcpy(results[b].hit_mask, hit[b].data(), static_cast<size_t>(prompts[b].n_chunks));
+  }
+  h->plan = std::move(plan);
+  st.n_prompts = n_prompts;
+  st.chunks_hit = chunks_hit;
+  st.chunks_missed = chunks_missed;
+  st.ctx_tokens = rows_total;
+  st.hit_tokens = hit_tokens;
+  st.new_rows = new_total;
+  refresh_page_stats(h);
+  st.host_plan_us = plan_us;
+  st.attn_visible_pairs = visible_pairs;
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
+  st.device_us = 1000.0 * ms;
+  timer.collect();
+  return PERCACHE_OK;
+}
+
+
 }  // namespace
 
 extern "C" {
@@ -505,6 +826,9 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   const size_t pool_elems = static_cast<size_t>(L) * cfg->pool_pages * PAGE_TOKENS * D.kv_dim;
   const size_t ctx_elems = static_cast<size_t>(L) * h->ctx_cap * D.kv_dim;
   ok = ok && dev_alloc(h, &h->kpool, pool_elems) && dev_alloc(h, &h->vpool, pool_elems);
+  h->paper_mode = (cfg->flags & PERCACHE_FLAG_PAPER_MODE) != 0;
+  const size_t qpool_elems = static_cast<size_t>(L) * cfg->pool_pages * PAGE_TOKENS * D.q_dim;
+  if (h->paper_mode) ok = ok && dev_alloc(h, &h->qpool, qpool_elems);
   ok = ok && dev_alloc(h, &h->kctx, ctx_elems) && dev_alloc(h, &h->vctx, ctx_elems);
   ok = ok && dev_alloc(h, &h->rope, static_cast<size_t>(cfg->max_prompt_tokens) * ROPE_HALF);
   ok = ok && dev_alloc(h, &h->resid, static_cast<size_t>(h->m_cap) * d);
@@ -565,6 +889,11 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   cudaMemsetAsync(h->attn_out, 0, static_cast<size_t>(h->m_cap) * D.q_dim * 2, h->stream);
   cudaMemsetAsync(h->xn, 0, static_cast<size_t>(h->m_cap) * d * 2, h->stream);
   cudaMemsetAsync(h->act, 0, static_cast<size_t>(h->m_cap) * F * 2, h->stream);
+  if (h->paper_mode) {      // there the attention copies whole pages, also ones a prompt only partly fills
+    cudaMemsetAsync(h->qpool, 0, qpool_elems * 2, h->stream);
+    cudaMemsetAsync(h->kpool, 0, pool_elems * 2, h->stream);
+    cudaMemsetAsync(h->vpool, 0, pool_elems * 2, h->stream);
+  }
 
   // ---- weights: bf16 -> fp16 copies in the layouts the GEMMs read.  Every bf16 value of magnitude
   // >= 2^-17 is exactly representable in fp16; smaller ones round with absolute error <= 2^-25.
@@ -613,6 +942,11 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
               make_operand_map(&W.m_wgu256, W.wgu, 2 * F, d, 256) == 0 && make_operand_map(&W.m_wd256, W.wd, d, F, 256) == 0;
     cuda_ok = cuda_ok && make_attn_maps(&W.attn_maps, h->qbuf, h->m_cap, D.q_dim, h->kctx + l * ctx_layer,
                                         h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim) == 0;
+    if (h->paper_mode) {
+      const size_t pl = static_cast<size_t>(cfg->pool_pages) * PAGE_TOKENS;
+      cuda_ok = cuda_ok && make_paged_attn_maps(&W.paged_maps, h->qpool + l * pl * D.q_dim, h->kpool + l * pl * D.kv_dim,
+                                                h->vpool + l * pl * D.kv_dim, cfg->pool_pages, D.q_dim, D.kv_dim) == 0;
+    }
   }
   launch_build_rope_table(h->rope, cfg->max_prompt_tokens, static_cast<double>(cfg->rope_theta), s);
   cuda_ok = cuda_ok && make_operand_map(&h->m_xn, h->xn, h->m_cap, d, 128) == 0 &&
@@ -673,7 +1007,7 @@ int percache_destroy(percache_t* h) {
 
 int percache_set_flags(percache_t* h, uint32_t flags) {
   if (!h) return PERCACHE_E_INVAL;
-  h->flags = flags;
+  h->flags = (flags & ~PERCACHE_FLAG_PAPER_MODE) | (h->flags & PERCACHE_FLAG_PAPER_MODE);   // the mode is fixed at creation
   return PERCACHE_OK;
 }
 
@@ -697,7 +1031,7 @@ int percache_drop_chunk(percache_t* h, uint64_t chunk_id) {
 
 int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, const void* k, const void* v,
                           int32_t ptr_is_device) {
-  if (!h || !k || !v || n_tokens <= 0) return PERCACHE_E_INVAL;
+  if (!h || !k || !v || n_tokens <= 0 || h->paper_mode) return PERCACHE_E_INVAL;   // that mode's entries hold Q as well
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
   const int n_pages = (n_tokens + PAGE_TOKENS - 1) / PAGE_TOKENS;
@@ -752,7 +1086,7 @@ int percache_put_chunk_kv(percache_t* h, uint64_t chunk_id, int32_t n_tokens, co
 }
 
 int percache_put_chunk_synthetic(percache_t* h, uint64_t chunk_id, int32_t n_tokens, uint64_t seed) {
-  if (!h || n_tokens <= 0) return PERCACHE_E_INVAL;
+  if (!h || n_tokens <= 0 || h->paper_mode) return PERCACHE_E_INVAL;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   if (h->table.count(chunk_id)) return PERCACHE_E_EXISTS;
   ChunkEntry ent;
@@ -807,10 +1141,29 @@ int percache_get_chunk_kv(percache_t* h, uint64_t chunk_id, void* k_host, void* 
   return rc;
 }
 
+int percache_get_chunk_q(percache_t* h, uint64_t chunk_id, void* q_host) {
+  if (!h || !q_host || !h->paper_mode) return PERCACHE_E_INVAL;
+  if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  auto it = h->table.find(chunk_id);
+  if (it == h->table.end()) return PERCACHE_E_NOTFOUND;
+  const ChunkEntry& ent = it->second;
+  const size_t elems = static_cast<size_t>(h->dims.n_layers) * ent.n_tokens * h->dims.q_dim;
+  __nv_bfloat16* dq = nullptr;
+  if (cudaMalloc(reinterpret_cast<void**>(&dq), elems * 2) != cudaSuccess) { cudaGetLastError(); return PERCACHE_E_NOMEM; }
+  int rc = with_chunk_pages(h, ent.pages, [&](const int32_t* d_pages) {
+    launch_chunk_pages_copy(dq, h->qpool, d_pages, ent.n_tokens, h->dims.n_layers, h->cfg.pool_pages, h->dims.q_dim, 0,
+                            h->stream);
+  });
+  if (rc == PERCACHE_OK && cudaMemcpy(q_host, dq, elems * 2, cudaMemcpyDeviceToHost) != cudaSuccess) rc = PERCACHE_E_CUDA;
+  cudaFree(dq);
+  return rc;
+}
+
 int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts, percache_result_t* results) {
   if (!h || !prompts || !results || n_prompts <= 0) return PERCACHE_E_INVAL;
   if (n_prompts > h->cfg.max_batch_prompts) return PERCACHE_E_CAPACITY;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  if (h->paper_mode) return prefill_paper(h, prompts, n_prompts, results);
   const auto t_host0 = std::chrono::steady_clock::now();
   const ModelDims& D = h->dims;
   const int d = D.d_model;
@@ -819,6 +1172,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   struct Seg { const void* src; int on_device; int row0; int n; };   // input rows to stage
   std::vector<Seg> segs;
   std::vector<std::vector<uint8_t>> hit(n_prompts);
+  std::vector<int> last_hit(n_prompts, -1);                          // index of the final matched chunk, or -1
   std::unordered_map<uint64_t, std::pair<int, int>> first_miss;      // id -> (prompt, chunk) that will store it
   std::unordered_map<uint64_t, int64_t> hit_uses;                    // id -> prompt occurrences that hit it
   // Store key of every chunk: its id, or in prefix mode the key of the path of ids up to and including it.
@@ -871,6 +1225,20 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
         }
       }
       T += len;
+    }
+    // Prefix matching only: the final matched chunk gives up its last reuse_tail_drop tokens, which are computed
+    // from their inputs like any new row (and not stored again: the chunk is in the store already).
+    last_hit[b] = -1;
+    for (int i = P.n_chunks - 1; i >= 0 && last_hit[b] < 0; --i)
+      if (hit[b][i]) last_hit[b] = i;
+    if (P.reuse_tail_drop != 0) {
+      if (P.reuse_tail_drop < 0 || P.match_mode != PERCACHE_MATCH_PREFIX_PATH) return PERCACHE_E_INVAL;
+      if (last_hit[b] >= 0) {
+        if (P.reuse_tail_drop > P.chunk_len[last_hit[b]]) return PERCACHE_E_INVAL;
+        if (!P.chunk_hidden || !P.chunk_hidden[last_hit[b]]) return PERCACHE_E_MISS_NO_INPUT;
+        n_new += P.reuse_tail_drop;
+        hit_tokens -= P.reuse_tail_drop;
+      }
     }
     T += P.n_query;
     n_new += P.n_query;
@@ -953,29 +1321,35 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       const int len = is_query ? P.n_query : P.chunk_len[i];
       if (len == 0) continue;
       const bool is_hit = !is_query && hit[b][i];
+      // tokens [0, reuse_len) of the chunk come from the store, the rest (all of a missed chunk or of the query,
+      // the dropped tail of the final matched chunk) are new rows
+      const int reuse_len = !is_hit ? 0 : len - (i == last_hit[b] ? P.reuse_tail_drop : 0);
       for (int o = 0; o < len; ++o) {
         plan.slot_chunk[pbase + t + o] = i;
         plan.slot_offset[pbase + t + o] = o;
-        plan.slot_is_new[pbase + t + o] = is_hit ? 0 : 1;
+        plan.slot_is_new[pbase + t + o] = o < reuse_len ? 0 : 1;
       }
-      if (is_hit) {
+      if (reuse_len > 0) {
         const ChunkEntry& ent = h->table.find(keys[b][i])->second;
-        for (int o = 0; o < len; o += PAGE_TOKENS) {
+        for (int o = 0; o < reuse_len; o += PAGE_TOKENS) {
           GatherItem& g = items[n_items++];
           g.dst_slot = ctx0 + t + o;
           g.src_page = ent.pages[o / PAGE_TOKENS];
-          g.n_tok = std::min(PAGE_TOKENS, len - o);
+          g.n_tok = std::min(PAGE_TOKENS, reuse_len - o);
           g.pos = t + o;
         }
-      } else {
+      }
+      if (reuse_len < len) {
         const ChunkEntry* ent = nullptr;
-        if (!is_query) {
+        if (!is_query && !is_hit) {
           auto fm = first_miss.find(keys[b][i]);
           if (fm != first_miss.end() && fm->second.first == b && fm->second.second == i)
             ent = &pending[pending_of[keys[b][i]]].second;
         }
-        segs.push_back(Seg{is_query ? P.query_hidden : P.chunk_hidden[i], P.hidden_on_device, static_cast<int>(r), len});
-        for (int o = 0; o < len; ++o, ++r) {
+        const char* src = static_cast<const char*>(is_query ? P.query_hidden : P.chunk_hidden[i]);
+        segs.push_back(Seg{src + static_cast<size_t>(reuse_len) * d * 2, P.hidden_on_device, static_cast<int>(r),
+                           len - reuse_len});
+        for (int o = reuse_len; o < len; ++o, ++r) {
           row_slot[r] = ctx0 + t + o;
           row_pos[r] = t + o;
           row_pool[r] = ent ? ent->pages[o / PAGE_TOKENS] * PAGE_TOKENS + (o % PAGE_TOKENS) : -1;
@@ -1125,7 +1499,7 @@ int percache_set_decode_reserve(percache_t* h, int32_t tokens_per_prompt) {
 
 int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_t hidden_on_device, float* out_hidden,
                     int32_t out_on_device) {
-  if (!h || !hidden || !out_hidden || n_prompts <= 0) return PERCACHE_E_INVAL;
+  if (!h || !hidden || !out_hidden || n_prompts <= 0 || h->paper_mode) return PERCACHE_E_INVAL;
   Plan& plan = h->plan;
   if (static_cast<size_t>(n_prompts) + 1 != plan.cu_ctx.size()) return PERCACHE_E_INVAL;   // not the last call's batch
   if (n_prompts > h->m_cap) return PERCACHE_E_CAPACITY;

@@ -30,6 +30,21 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
   return t;
 }
 
+// ---------------------------------------------------------------- fp16 conversion
+// Two floats to packed fp16 (a in the low half), round to nearest even, SATURATING: a magnitude beyond the
+// largest finite fp16 value (65504) becomes +-65504 instead of infinity (NaN stays NaN).  Every fp16 operand the
+// library forms goes through this conversion, so an out-of-range activation or cached bf16 value clips instead
+// of turning into inf and, one masked product later, NaN.
+__device__ __forceinline__ uint32_t pack_half2(float a, float b) {
+  uint32_t r;
+  asm("cvt.rn.satfinite.f16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(b), "f"(a));   // first source -> upper half
+  return r;
+}
+__device__ __forceinline__ __half to_half_sat(float a) {
+  const uint32_t r = pack_half2(a, 0.f);
+  return __ushort_as_half(static_cast<unsigned short>(r & 0xffffu));
+}
+
 // ---------------------------------------------------------------- programmatic dependent launch
 // Every kernel of a prefill call is launched with programmatic stream serialisation: the next kernel's
 // CTAs may start (barrier init, TMEM allocation, descriptor prefetch) while this one is still running.

@@ -27,10 +27,11 @@ E_MISS_NO_INPUT, E_CAPACITY, E_DEVICE_TIMEOUT, E_CUDA, E_NOTFOUND = -6, -7, -8, 
 FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION, FLAG_EVICT_LFU = 1, 2, 4, 8
 FLAG_SINGLE_CTA_GEMM = 16
 FLAG_NO_SMALL_ROW_KERNELS = 32
+FLAG_PAPER_MODE = 64
 PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
-           "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_put_chunk_synthetic",
+           "percache_has_chunk", "percache_drop_chunk", "percache_get_chunk_kv", "percache_get_chunk_q", "percache_put_chunk_synthetic",
            "percache_get_stats", "percache_set_flags", "percache_decode", "percache_set_decode_reserve", "percache_set_store_limit", "percache_chunk_info", "percache_debug_read_plan", "percache_debug_read_ctx", "percache_debug_attn_plan",
            "percache_debug_gemm", "percache_debug_gemm_noalloc", "percache_debug_capture_layers", "percache_debug_wait_probe", "percache_path_key", "percache_qa_top1", "percache_strerror")
 
@@ -57,7 +58,7 @@ class LayerWeights(C.Structure):
 class PromptStruct(C.Structure):
     _fields_ = [("n_chunks", C.c_int32), ("chunk_ids", C.POINTER(C.c_uint64)), ("chunk_len", C.POINTER(C.c_int32)),
                 ("chunk_hidden", C.POINTER(C.c_void_p)), ("n_query", C.c_int32), ("query_hidden", C.c_void_p),
-                ("hidden_on_device", C.c_int32), ("match_mode", C.c_int32)]
+                ("hidden_on_device", C.c_int32), ("match_mode", C.c_int32), ("reuse_tail_drop", C.c_int32)]
 
 
 class ResultStruct(C.Structure):
@@ -94,6 +95,7 @@ def load_library() -> C.CDLL:
     lib.percache_has_chunk.argtypes = [vp, u64, C.POINTER(i32)]
     lib.percache_drop_chunk.argtypes = [vp, u64]
     lib.percache_get_chunk_kv.argtypes = [vp, u64, vp, vp]
+    lib.percache_get_chunk_q.argtypes = [vp, u64, vp]
     lib.percache_put_chunk_synthetic.argtypes = [vp, u64, i32, u64]
     lib.percache_get_stats.argtypes = [vp, C.POINTER(StatsStruct)]
     lib.percache_set_flags.argtypes = [vp, C.c_uint32]
@@ -158,6 +160,7 @@ class PromptSpec:
     query_hidden: Any                            # [n_query, d]
     n_query: Optional[int] = None
     match_prefix: bool = False                   # True: PERCACHE_MATCH_PREFIX_PATH (the paper's prefix-tree walk)
+    tail_drop: int = 0                           # reuse_tail_drop (prefix matching only)
 
 
 @dataclass
@@ -181,6 +184,8 @@ class PerCache:
         self.d_model = d_model
         self.n_layers = n_layers
         self.kv_dim = n_kv_heads * head_dim
+        self.q_dim = n_q_heads * head_dim
+        self.paper_mode = bool(flags & FLAG_PAPER_MODE)
         if max_batch_ctx_tokens is None:
             max_batch_ctx_tokens = max_prompt_tokens * max_batch_prompts
         if max_batch_new_rows is None:
@@ -259,6 +264,15 @@ class PerCache:
         _check(self._lib.percache_get_chunk_kv(self._h, chunk_id, _ptr(k), _ptr(v)), "percache_get_chunk_kv")
         return k, v
 
+    def get_chunk_q(self, chunk_id: int) -> np.ndarray:
+        """Paper-faithful mode: the node's cached Q, bf16 bits [n_layers, n_tokens, n_q_heads*head_dim]."""
+        n = self.has_chunk(chunk_id)
+        if n is None:
+            raise PerCacheError(E_NOTFOUND, "percache_get_chunk_q")
+        q = np.empty((self.n_layers, n, self.q_dim), dtype=np.uint16)
+        _check(self._lib.percache_get_chunk_q(self._h, chunk_id, _ptr(q)), "percache_get_chunk_q")
+        return q
+
     # ------------------------------------------------------------------ prefill
     def prefill(self, prompts: Sequence[PromptSpec], out: Optional[Sequence[Any]] = None) -> List[PromptResult]:
         """percache_prefill.  `out[b]`: optional caller buffer float32 [rows >= n_new, d] (numpy or device tensor)."""
@@ -285,7 +299,7 @@ class PerCache:
                         hid[i] = _ptr(hcur)
             nq = int(p.n_query if p.n_query is not None else (0 if p.query_hidden is None else p.query_hidden.shape[0]))
             ps[b] = PromptStruct(nc, ids, lens, hid, nq, _ptr(p.query_hidden) if nq > 0 else None, 1 if on_dev else 0,
-                                 1 if p.match_prefix else 0)
+                                 1 if p.match_prefix else 0, int(p.tail_drop))
             keep += [ids, lens, hid]
             if out is not None and out[b] is not None:
                 ob = out[b]
@@ -297,7 +311,9 @@ class PerCache:
             outs.append(ob)
             masks.append(mask)
         _check(self._lib.percache_prefill(self._h, ps, n, rs), "percache_prefill")
-        return [PromptResult(outs[b][: rs[b].n_new], masks[b][: len(prompts[b].chunk_ids)], int(rs[b].n_new),
+        # rows that come back: the new rows, or every row of the prompt in the paper-faithful mode
+        n_out = [int(rs[b].n_total if self.paper_mode else rs[b].n_new) for b in range(n)]
+        return [PromptResult(outs[b][: n_out[b]], masks[b][: len(prompts[b].chunk_ids)], int(rs[b].n_new),
                              int(rs[b].n_total)) for b in range(n)]
 
     # ------------------------------------------------------------------ introspection

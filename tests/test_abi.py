@@ -42,7 +42,7 @@ def test_struct_sizes_match_header():
     # natural alignment of the declarations in percache.h
     assert C.sizeof(pcb.Config) == 96
     assert C.sizeof(pcb.LayerWeights) == 72
-    assert C.sizeof(pcb.PromptStruct) == 56
+    assert C.sizeof(pcb.PromptStruct) == 64
     assert C.sizeof(pcb.ResultStruct) == 40
     assert C.sizeof(pcb.StatsStruct) == 184
 

@@ -54,3 +54,48 @@ def test_prefix_tree_sequence():
                                         match_prefix=True)])[0]
         assert got.hit_mask.tolist() == [1, 0, 0]
         assert h.has_chunk(pcb.path_key([1, 5])) == lens[5]
+
+
+@pytest.mark.parametrize("drop", [1, 16, 37, 100])
+def test_tail_of_the_final_matched_chunk_is_recomputed(drop):
+    """reuse_tail_drop (paper Appendix B, tokenisation paragraph): the last tokens of the final matched chunk are new
+    rows computed from their inputs; layout bit-exact, hidden states within tolerance of the oracle and of plain
+    full prefill, nothing stored twice.  Cases: one token, one whole page, a ragged count, the whole chunk."""
+    shape = wl.small_workload(seed=72, n_layers=2, chunk_lens=[16], n_query=1, hit_idx=[]).shape
+    weights = wl.make_weights(shape, 72, random_gains=True)
+    model = H.oracle_model(shape, weights)
+    lens = {1: 130, 5: 100, 9: 48}
+    hid = {c: wl.chunk_hidden_for(72, c, n, shape.d_model) for c, n in lens.items()}
+    qh = wl.make_hidden(72, (2, 0), 19, shape.d_model)
+    f64 = orc.bf16_bits_to_f64
+    store = orc.Store()
+    h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
+                     n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
+                     pool_pages=64, max_prompt_tokens=400, max_batch_prompts=1)
+    with h:
+        warm = [1, 5]
+        orc.reuse_prefill(model, store, [orc.Prompt(warm, [lens[c] for c in warm], [f64(hid[c]) for c in warm],
+                                                    np.zeros((0, shape.d_model)))], match_prefix=True)
+        h.prefill([pcb.PromptSpec(warm, [lens[c] for c in warm], [hid[c] for c in warm], None, 0, match_prefix=True)])
+        pages_before = h.stats()["pages_used"]
+        ids = [1, 5, 9]
+        want = orc.reuse_prefill(model, store, [orc.Prompt(ids, [lens[c] for c in ids], [None, f64(hid[5]), f64(hid[9])],
+                                                           f64(qh), tail_drop=drop)], match_prefix=True,
+                                 keep_ctx=True, commit=False)[0]
+        got = h.prefill([pcb.PromptSpec(ids, [lens[c] for c in ids], [None, hid[5], hid[9]], qh, match_prefix=True,
+                                        tail_drop=drop)])[0]
+        assert got.hit_mask.tolist() == [1, 1, 0] == want.layout.hit_mask.tolist()
+        assert got.n_new == drop + lens[9] + 19 and got.n_total == 297
+        G.check_plan(h.read_plan(), [want.layout])
+        G.check_ctx(h, [want], range(shape.n_layers))
+        c = G.compare_hidden(got.out_hidden, want.out_hidden)
+        assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
+        full, _, _ = orc.dense_prefill(model, np.concatenate([f64(hid[c]) for c in ids] + [f64(qh)]))
+        c = G.compare_hidden(got.out_hidden, full[want.layout.new_slots])
+        assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
+        # only chunk 9's node was added
+        assert h.stats()["pages_used"] == pages_before + 3 and h.has_chunk(pcb.path_key(ids)) == 48
+        # outside prefix matching the field must be zero
+        with pytest.raises(pcb.PerCacheError) as e:
+            h.prefill([pcb.PromptSpec([77], [16], [hid[9][:16]], qh, tail_drop=1)])
+        assert e.value.code == pcb.E_INVAL
