@@ -76,7 +76,12 @@ def test_tail_of_the_final_matched_chunk_is_recomputed(drop):
         warm = [1, 5]
         orc.reuse_prefill(model, store, [orc.Prompt(warm, [lens[c] for c in warm], [f64(hid[c]) for c in warm],
                                                     np.zeros((0, shape.d_model)))], match_prefix=True)
-        h.prefill([pcb.PromptSpec(warm, [lens[c] for c in warm], [hid[c] for c in warm], None, 0, match_prefix=True)])
+        # the library gets exactly the oracle's nodes (same bf16 bits), under their path keys, so that gathered
+        # bytes can be compared bit for bit
+        for path, (ck, cv) in store.kv.items():
+            L, n = ck.shape[0], ck.shape[1]
+            h.put_chunk_kv(pcb.path_key(list(path)), np.ascontiguousarray(orc.f64_to_bf16_bits(ck).reshape(L, n, -1)),
+                           np.ascontiguousarray(orc.f64_to_bf16_bits(cv).reshape(L, n, -1)))
         pages_before = h.stats()["pages_used"]
         ids = [1, 5, 9]
         want = orc.reuse_prefill(model, store, [orc.Prompt(ids, [lens[c] for c in ids], [None, f64(hid[5]), f64(hid[9])],

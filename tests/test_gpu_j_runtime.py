@@ -82,8 +82,9 @@ def test_bounded_wait_runs_out_and_the_device_stays_usable():
     assert 1.0e6 <= waited[0] < 50.0e6            # the first waiter gave up after its own limit (1 ms)...
     assert waited[1] < 100.0e6                    # ...and the second long before its own (1 s): it saw the error word
     a = (np.random.default_rng(5).standard_normal((200, 256)) * 0.5).astype(np.float16)
-    c = pcb.debug_gemm(a, a)
-    assert np.max(np.abs(c - a.astype(np.float64) @ a.astype(np.float64).T)) < 1e-2
+    b = (np.random.default_rng(6).standard_normal((256, 256)) * 0.5).astype(np.float16)
+    c = pcb.debug_gemm(a, b)
+    assert np.max(np.abs(c - a.astype(np.float64) @ b.astype(np.float64).T)) < 1e-2
     rc2, code2, _ = pcb.debug_wait_probe(limit_us=200)
     assert rc2 == pcb.E_DEVICE_TIMEOUT and code2 == 901
 

@@ -70,7 +70,8 @@ def test_sequence_of_queries_against_the_paper_mode_oracle():
         a = h.prefill([pcb.PromptSpec(ids, [lens[c] for c in ids], [hid[c] for c in ids], qh, match_prefix=True)])[0]
         b = h.prefill([pcb.PromptSpec(ids, [lens[c] for c in ids], [hid[c] for c in ids], qh, match_prefix=True)])[0]
         assert h.stats()["pages_free"] == pages_before and a.hit_mask.tolist() == [1, 1, 1, 1]
-        assert np.array_equal(a.out_hidden[-40:], b.out_hidden[-40:])          # same pages, same arithmetic
+        # same pages, same arithmetic (up to the order of the atomic additions of a K-split residual GEMM)
+        assert np.max(np.abs(a.out_hidden - b.out_hidden)) < 1e-4
 
 
 def test_batch_and_refusals():
