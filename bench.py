@@ -36,7 +36,7 @@ from paper_2601_11553_b200 import workloads as wl
 METRIC = "reuse_prefill_tokens_per_s"
 UNIT = "tokens/s"
 DEFAULT_WORKLOAD = "cfg4_50"      # the largest single-GPU workload that uses both halves of the method
-TABLE_WORKLOADS = ("cfg0", "cfg1", "cfg2", "cfg3", "cfg4_100", "cfg4_90", "cfg4_50", "cfg4_0")
+TABLE_WORKLOADS = ("cfg0", "cfg1", "cfg2", "cfg3", "cfg4_100", "cfg4_90", "cfg4_50", "cfg4_0", "prefix_cfg1", "paper_cfg1")
 
 
 def load_peaks():
@@ -118,7 +118,9 @@ def flops_per_step(w: wl.Workload, new_rows: int, visible_pairs: int):
     s = w.shape
     per_row = {"qkv": 2 * s.d_model * (s.q_dim + 2 * s.kv_dim), "oproj": 2 * s.q_dim * s.d_model,
                "gateup": 2 * s.d_model * 2 * s.d_ffn, "down": 2 * s.d_ffn * s.d_model}
-    out = {k: v * new_rows * s.n_layers for k, v in per_row.items()}
+    # paper-faithful mode: only the projections skip the cached rows, the rest of every block runs on all rows
+    rows = {k: (w.total_tokens if (w.paper_mode and k != "qkv") else new_rows) for k in per_row}
+    out = {k: v * rows[k] * s.n_layers for k, v in per_row.items()}
     out["attn"] = 4 * s.n_q_heads * s.head_dim * visible_pairs * s.n_layers
     return out
 
@@ -233,6 +235,27 @@ class OracleBlockSample:
 def cpu_baseline_for(w: wl.Workload):
     """Oracle tokens/s on the host for workload w: a whole run where it takes seconds, else the bounded block sample."""
     tokens = w.total_tokens
+    if w.paper_mode:                                       # the paper-faithful oracle, a few layers of the real call
+        from oracle import paper_mode as pm
+        from oracle import reuse_prefill as orc
+        n_sample = max(1, min(w.shape.n_layers, 2))
+        shape = wl.ModelShape(n_layers=n_sample, **{k: getattr(w.shape, k) for k in
+                                                    ("d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn")})
+        model = _oracle_model(shape, wl.make_weights(shape, w.seed))
+        store = pm.PaperStore()
+        p = w.prompts[0]
+        f64 = orc.bf16_bits_to_f64
+        n_c = len(w.cached_ids)
+        pm.paper_prefill(model, store, [pm.PaperPrompt(list(p.chunk_ids[:n_c]), list(p.chunk_len[:n_c]),
+                                                       [f64(h) for h in p.chunk_hidden[:n_c]], np.zeros((0, shape.d_model)))])
+        t0 = time.perf_counter()
+        pm.paper_prefill(model, store, [pm.PaperPrompt(list(p.chunk_ids), list(p.chunk_len), [f64(h) for h in p.chunk_hidden],
+                                                       f64(p.query_hidden))], commit=False)
+        t = time.perf_counter() - t0
+        scale = w.shape.n_layers / n_sample
+        return {"value": tokens / (t * scale), "unit": UNIT, "cores": _oracle_cores(), "kind": "oracle",
+                "sample": f"first {n_sample} of {w.shape.n_layers} layers of {w.name} through oracle.paper_mode, all rows, "
+                          f"one call ({t:.1f} s), time x {scale:g}", "extrapolated": True}
     if w.new_rows() * w.shape.n_layers <= 3000:            # cfg0-sized: the whole call
         step, cores = oracle_sample(w, w.shape.n_layers)
         t = step()
@@ -324,6 +347,7 @@ class Bench:
 
     def __init__(self, shape, seed, workloads, local, torch, pcb):
         self.torch, self.pcb = torch, pcb
+        self.paper_mode = workloads[0].paper_mode
         self.dev = torch.device("cuda", local)
         self.local = local
         self.shape = shape
@@ -338,11 +362,11 @@ class Bench:
         max_tokens = max(w.total_tokens for w in workloads)
         self.h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
                               n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
-                              pool_pages=sum((l + 15) // 16 for l in ids_lens.values()) + 64,
+                              pool_pages=2 * sum((l + 15) // 16 for l in ids_lens.values()) + 256,
                               max_prompt_tokens=max(p.n_total for w in workloads for p in w.prompts),
                               max_batch_prompts=max(len(w.prompts) for w in workloads),
                               max_batch_ctx_tokens=max_tokens, max_batch_new_rows=max_tokens, device=local,
-                              stream=self.stream.cuda_stream)
+                              stream=self.stream.cuda_stream, flags=pcb.FLAG_PAPER_MODE if self.paper_mode else 0)
 
     def close(self):
         self.h.close()
@@ -352,6 +376,13 @@ class Bench:
         alone through the library itself, or the seeded integer pool), others of the workload are dropped."""
         h, pcb = self.h, self.pcb
         cached = set(w.cached_ids)
+        if w.match_prefix:       # the cached chain: one prefill of exactly that prefix, stored under its path keys
+            p = w.prompts[0]
+            n = len(w.cached_ids)
+            if n and h.has_chunk(pcb.path_key(list(p.chunk_ids[:n]))) is None:
+                h.prefill([pcb.PromptSpec(list(p.chunk_ids[:n]), list(p.chunk_len[:n]), list(p.chunk_hidden[:n]), None, 0,
+                                          match_prefix=True)])
+            return
         for c in w.cached_ids:
             if h.has_chunk(c) is not None:
                 continue
@@ -371,6 +402,9 @@ class Bench:
         self.set_cache_state(w)
         cached = set(w.cached_ids)
         missed = sorted({c for p in w.prompts for c in p.chunk_ids if c not in cached})
+        if w.match_prefix:       # nodes are stored under the key of their path
+            missed = [pcb.path_key(list(p.chunk_ids[: i + 1])) for p in w.prompts
+                      for i, c in enumerate(p.chunk_ids) if c not in cached]
 
         def to_dev(a):
             return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
@@ -381,12 +415,15 @@ class Bench:
         def specs(conv):
             out = []
             for p in w.prompts:
-                hid = [None if c in cached else conv(hh) for c, hh in zip(p.chunk_ids, p.chunk_hidden)] \
-                    if p.chunk_hidden else None
-                out.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, conv(p.query_hidden), p.n_query))
+                hid = [None if (c in cached and not w.paper_mode) else conv(hh)
+                       for c, hh in zip(p.chunk_ids, p.chunk_hidden)] if p.chunk_hidden else None
+                out.append(pcb.PromptSpec(list(p.chunk_ids), list(p.chunk_len), hid, conv(p.query_hidden), p.n_query,
+                                          match_prefix=w.match_prefix))
             return out
 
         n_new = [p.n_query + sum(l for c, l in zip(p.chunk_ids, p.chunk_len) if c not in cached) for p in w.prompts]
+        if w.paper_mode:         # every row of the prompt comes back
+            n_new = [p.n_total for p in w.prompts]
         specs_dev = specs(to_dev)
         out_dev = [torch.empty((n, shape.d_model), dtype=torch.float32, device=dev) for n in n_new]
 
@@ -514,15 +551,20 @@ def run_gpu(args):
         torch.cuda.synchronize(dev)
 
     main_w = wl.by_name(args.workload)
+    if args.layers > 0:
+        main_w.shape = wl.ModelShape(n_layers=args.layers, **{k: getattr(main_w.shape, k) for k in
+                                                              ("d_model", "n_q_heads", "n_kv_heads", "head_dim", "d_ffn")})
+        main_w.name += f"@{args.layers}layers"
+        args.no_table = True
     # Workloads that share the main one's model run on the same handle (the long-context sweep: one model, four hit
     # rates with nested hit sets, run from the fullest cache to the emptiest); the others get a handle each.
     table_names = [] if (args.no_table or world > 1) else [n for n in TABLE_WORKLOADS if n != main_w.name]
     groups = {}
     for name in [main_w.name] + table_names:
         w = main_w if name == main_w.name else wl.by_name(name)
-        groups.setdefault((w.seed, w.shape), []).append(w)
+        groups.setdefault((w.seed, w.shape, w.paper_mode), []).append(w)
     rows, main = [], None
-    for (seed, shape), ws in groups.items():
+    for (seed, shape, _paper), ws in groups.items():
         ws.sort(key=lambda w: -len(w.cached_ids))
         b = Bench(shape, seed, ws, local, torch, pcb)
         for w in ws:
@@ -579,8 +621,8 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": r["total_ms"] / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
-        "config": {"workload": w.name, "description": w.description, "tokens_per_step": tokens,
-                   "new_rows_per_step": new_rows, "hit_tokens_per_step": int(st["hit_tokens"]),
+        "config": {"workload": w.name, "reduced_depth": args.layers > 0, "description": w.description,
+                   "tokens_per_step": tokens, "new_rows_per_step": new_rows, "hit_tokens_per_step": int(st["hit_tokens"]),
                    "prompts_per_step": len(w.prompts), "ms_per_prompt": r["total_ms"] / args.steps / len(w.prompts),
                    "computed_rows_per_s": world * new_rows * args.steps / (r["total_ms"] / 1000.0),
                    "l2": f"inputs exceed L2: {shape.params_per_layer * shape.n_layers * 2 / 1e6:.0f} MB of weights are "
@@ -589,8 +631,10 @@ def run_gpu(args):
                    "device_ms_per_step_kernels_only": r["dev_us"] / args.steps / 1000.0,
                    "host_plan_us": st["host_plan_us"], "phase_pass_ms_per_step": float(sum(r["ms_ph"])) / r["ph_steps"]},
         "clocks": r["clocks"],
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": new_rows * shape.d_model * 2,
-                "d2h_bytes_per_step": new_rows * shape.d_model * 4, "ms_per_step": r["e2e_ms"] / args.steps},
+        "e2e": {"value": e2e_value, "unit": UNIT,
+                "h2d_bytes_per_step": (tokens if w.paper_mode else new_rows) * shape.d_model * 2,
+                "d2h_bytes_per_step": (tokens if w.paper_mode else new_rows) * shape.d_model * 4,
+                "ms_per_step": r["e2e_ms"] / args.steps},
         "gpu_launches": kernels_per_step * args.steps,
         "roofline": roof, "kernels": per_phase, "cpu_baseline": cpu,
         "step_tflops": main_row["step_tflops"], "step_frac_of_tensor_peak": main_row["step_frac_of_tensor_peak"],
@@ -746,6 +790,9 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-table", action="store_true", help="time the named workload only, not the per-workload table")
     ap.add_argument("--flags", type=int, default=0, help="PERCACHE_FLAG_* bits kept set during the timed passes")
+    ap.add_argument("--layers", type=int, default=0,
+                    help="profiling aid: run the workload on a model cut to this many layers (every launch keeps its shape, "
+                         "a profiler capture stays small); the line then says reduced_depth and is not a result")
     args = ap.parse_args()
     args.forward = sys.argv[1:]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl != "reference":

@@ -145,6 +145,11 @@ class Workload:
     #   "same_inputs_l1" : single layer; K/V from the same chunk hidden states (any method agrees)
     #   "integer_pool"   : counter-based integer generator (pool_kv_values)
     cache_source: str = "prefill_alone"
+    # True: chunks are matched as a path of the cache tree (the paper's rule); cached_ids then is a prefix of the list
+    # and the cached content comes from a prefill of exactly that prefix ("prefill_prefix")
+    match_prefix: bool = False
+    # True: the paper-faithful mode of the library (cached Q as well, every row of the prompt continues)
+    paper_mode: bool = False
 
     @property
     def total_tokens(self) -> int:
@@ -256,7 +261,23 @@ def config4(hit_rate: float, with_hidden: bool = True) -> Workload:
                     description=f"28 layers, 64x512+256=33024 tokens, {n_hits}/64 chunks hit")
 
 
+def prefix_config1(paper_mode: bool, with_hidden: bool = True) -> Workload:
+    """The 28-layer workload's prompt (8 x 256 + 64 tokens) with the first four chunks cached as a chain of the cache
+    tree: the case the paper itself reuses.  Run in the library's default reading (only the 1088 new rows continue)
+    or in the paper-faithful mode (all 2112 rows continue, the cached ones skip the projections)."""
+    shape = ModelShape(n_layers=28, **SHAPE_A)
+    p = _single_prompt(shape, 1, 8, 256, 64, with_hidden=with_hidden)
+    return Workload("paper_cfg1" if paper_mode else "prefix_cfg1", shape, 1, [p], cached_ids=list(p.chunk_ids[:4]),
+                    cache_source="prefill_prefix", match_prefix=True, paper_mode=paper_mode,
+                    description="28 layers, 8x256+64=2112 tokens, first 4 chunks cached as a prefix chain"
+                                + (", paper-faithful mode (all rows continue)" if paper_mode else ", new rows only"))
+
+
 def by_name(name: str, with_hidden: bool = True) -> Workload:
+    if name == "prefix_cfg1":
+        return prefix_config1(False, with_hidden)
+    if name == "paper_cfg1":
+        return prefix_config1(True, with_hidden)
     if name == "cfg0":
         return config0(with_hidden)
     if name == "cfg1":
