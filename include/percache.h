@@ -80,6 +80,9 @@ extern "C" {
 #define PERCACHE_FLAG_EVICT_LFU          8u  /* when the store is full, evict least-frequently-used chunks instead
                                                 of failing with PERCACHE_E_NOSPACE (see percache_set_store_limit)  */
 
+#define PERCACHE_FLAG_GATHER_FREE       128u  /* take the gather-free form of percache_prefill whenever it is possible
+                                                (see percache_prefill), not only when the cached part dominates   */
+#define PERCACHE_FLAG_ALWAYS_GATHER     256u  /* never take it: always assemble the contiguous context              */
 #define PERCACHE_FLAG_PAPER_MODE         64u  /* creation only: the handle works exactly as the paper states the scheme
                                                 (see "Paper-faithful mode" below)                                 */
 
@@ -171,7 +174,16 @@ typedef struct {
  * with the same length (different length -> PERCACHE_E_LEN_MISMATCH).  On success every missed chunk is
  * stored (its K/V as computed inside its prompt; if two prompts of the batch miss the same id, the
  * first prompt's is kept) and query tokens are not.  Too few free pages -> PERCACHE_E_NOSPACE.
- * Synchronous: returns after the stream has drained. */
+ * Synchronous: returns after the stream has drained.
+ * Two forms compute the same result.  The default one copies every cached token's K and V into a contiguous context
+ * (K rotated to its position there) and lets the attention read that.  The gather-free one leaves them in their
+ * pages: the attention walks the prompt's page table, rotates K as it loads it and reads V where it is, so the fetch
+ * and its traffic disappear; there P and V enter the second attention product as bf16 (the store's format) instead
+ * of fp16.  It is taken when the batch has at least 8 cached tokens per new row (or PERCACHE_FLAG_GATHER_FREE is
+ * set), every chunk length and reuse_tail_drop is a multiple of 16, no decode reserve is set and
+ * PERCACHE_FLAG_ALWAYS_GATHER is not; rows that are not stored (query tokens) then occupy pages of the store for the
+ * duration of the call (they count against the store limit).  After a gather-free call there is no assembled
+ * context: percache_decode and percache_debug_read_ctx return PERCACHE_E_INVAL. */
 PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
 
@@ -266,6 +278,8 @@ typedef struct {
   int32_t phase_launches[PERCACHE_PH_COUNT];   /* kernels launched per class (always filled)      */
   int64_t attn_visible_pairs;                  /* sum over new rows of (position + 1)             */
   int64_t evictions;                           /* chunks evicted by the last prefill / put call   */
+  int32_t gather_free;                         /* 1: the last prefill took the gather-free form   */
+  int32_t reserved0;
 } percache_stats_t;
 
 PERCACHE_API int percache_get_stats(percache_t* h, percache_stats_t* out);

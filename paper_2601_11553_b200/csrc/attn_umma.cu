@@ -26,6 +26,7 @@ namespace pc {
 namespace {
 
 constexpr int ATT_THREADS = 320;
+constexpr int ATT_THREADS_ROT = 384;          // + two warps that rotate K on its way from the pages (MODE 2)
 constexpr int BLK = 128;                       // rows per tile and context slots per block
 constexpr int HALF_TILE_BYTES = BLK * 64 * 2;  // 16 KB: 128 rows x 64 fp16 (one swizzled half)
 constexpr int TILE_BYTES = 2 * HALF_TILE_BYTES;
@@ -38,7 +39,10 @@ struct AttnArgs {
   const AttnItem* items;
   const int32_t* cta_first;
   const int32_t* row_pos;
-  const int32_t* page_table;      // PAGED: one page id per 16 context slots; an item's ctx0 indexes its prompt's first entry
+  const int32_t* page_table;      // paged forms: one page id per 16 context slots; an item's ctx0 indexes its prompt's first entry
+  const __nv_bfloat16* kpool;     // MODE 2: this layer's K pages [pool_pages * 16][kv_dim], unrotated bf16
+  const float2* rope;             // MODE 2: (cos, sin)[position][64]
+  int32_t rope_rows;              // MODE 2: positions the table covers
   __half* out;
   float* partial_o;
   float* partial_ml;
@@ -60,15 +64,24 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
   return y;
 }
 
-// PAGED = false: Q from the query buffer, K and V from the assembled context, all fp16.
-// PAGED = true (paper-faithful mode): Q, K and V are read straight from the bf16 pages of the store through the
-// prompt's page table, one 16-row page per bulk copy (nothing is gathered into a contiguous context first, and K
-// needs no rotation because that mode caches it after position encoding); the MMAs then run on bf16 operands and
-// P is written to TMEM as bf16.  Everything else is the same kernel.
-template <bool PAGED>
-__global__ void __launch_bounds__(ATT_THREADS, 1)
+// MODE 0: Q from the query buffer, K and V from the assembled context, all fp16.
+// MODE 1 (paper-faithful mode): Q, K and V are read straight from the bf16 pages of the store through the prompt's
+// page table, one 16-row page per bulk copy (nothing is gathered into a contiguous context first, and K needs no
+// rotation because that mode caches it after position encoding); both MMAs run on bf16 operands and P is written to
+// TMEM as bf16.
+// MODE 2 (gather-free form of the default mode, where the store holds K before rotation): Q from the fp16 query
+// buffer; V straight from its pages by bulk copies (the PV MMA then runs on bf16 operands, P as bf16); K is loaded
+// from its pages by two extra warps with 16-byte vector loads, rotated to the slot's position in this prompt in fp32
+// (paper Appendix B.1: position encodings must be those of the positions in the full sequence) and written as fp16
+// straight into the swizzled shared-memory tile the S MMA reads.  Hit tokens are then never copied to a contiguous
+// context: the page gather and its write + re-read of every cached K and V byte disappear.
+// Everything else is the same kernel.
+template <int MODE>
+__global__ void __launch_bounds__(MODE == 2 ? ATT_THREADS_ROT : ATT_THREADS, 1)
 umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, AttnArgs args) {
+  constexpr bool PAGED = MODE == 1;                  // Q, K, V all by page copies
+  constexpr bool PV_BF16 = MODE != 0;                // V comes from the bf16 pages
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t q_full, q_empty;
   __shared__ __align__(8) uint64_t k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
@@ -99,7 +112,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     mbar_init(&q_full, 1);
     mbar_init(&q_empty, 1);
     for (int s = 0; s < KV_STAGES; ++s) {
-      mbar_init(&k_full[s], 1); mbar_init(&k_empty[s], 1);
+      mbar_init(&k_full[s], MODE == 2 ? 2 : 1); mbar_init(&k_empty[s], 1);      // MODE 2: one arrival per rotating warp
       mbar_init(&v_full[s], 1); mbar_init(&v_empty[s], 1);
     }
     for (int i = 0; i < 2; ++i) {
@@ -168,6 +181,96 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                       g * HEAD_DIM + hf * 64, kv_page * PAGE_TOKENS);
       }
     }
+  } else if (warp == 8 && MODE == 2) {
+    // ---------------------------------------------------------------- TMA producer, MODE 2: Q tiles from the query
+    // buffer (lanes 0-3, one 128-row box each), V blocks from the pages (lanes 0-15, one page each)
+    uint32_t unit_it = 0, kvit = 0;
+    bool ok = true;
+    const int pg = lane & 7, hf = (lane >> 3) & 1;
+    for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
+      const AttnItem t = w == w_begin ? first_item : args.items[w];
+      const int gp = t.unit;
+      const int g = gp / pairs, h0 = g * group + 2 * (gp % pairs);
+      const int nb = t.blk_end - t.blk_begin;
+      const int32_t* pt = args.page_table + t.ctx0;
+      ok = mbar_wait(&q_empty, (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+      ok = __all_sync(0xffffffffu, ok);
+      if (!ok) { cta_failed = 1; break; }
+      if (lane == 0) mbar_arrive_expect_tx(&q_full, 2 * TILE_BYTES);
+      __syncwarp();
+      if (lane < 4)
+        tma_load_2d(q_smem + (lane >> 1) * TILE_BYTES + (lane & 1) * HALF_TILE_BYTES, &tmQ, &q_full,
+                    (h0 + (lane >> 1)) * HEAD_DIM + (lane & 1) * 64, t.row0);
+      for (int j = 0; j < nb; ++j, ++kvit) {
+        const int st = kvit & 1;
+        const uint32_t ph = (kvit >> 1) & 1u;
+        const int v_page = __ldg(pt + (t.blk_begin + j) * (BLK / PAGE_TOKENS) + pg);
+        ok = mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { cta_failed = 1; break; }
+        if (lane == 0) mbar_arrive_expect_tx(&v_full[st], TILE_BYTES);
+        __syncwarp();
+        if (lane < 16)
+          tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES + pg * (PAGE_TOKENS * 128), &tmV, &v_full[st],
+                      g * HEAD_DIM + hf * 64, v_page * PAGE_TOKENS);
+      }
+    }
+  } else if (warp >= 10) {
+    // ---------------------------------------------------------------- K from the pages, rotated on load (MODE 2 only:
+    // the other forms are launched without these warps).  64 threads: thread (r0 = tid / 8, j = tid % 8) takes rows
+    // r0, r0 + 8, ... of the block and, in each, the 16-byte vector j of the head's low half and the one of its high
+    // half (elements 8j..8j+7 and 64 + 8j..): together they are eight rotation pairs.  The results go to the place
+    // the 128-byte swizzle gives vector j of that row (j ^ (row & 7)), in both 64-column halves of the tile.
+    if constexpr (MODE == 2) {
+      const int tid = (warp - 10) * 32 + lane;
+      const int j = tid & 7, r0 = tid >> 3;
+      const int kv_dim = args.n_kv_heads * HEAD_DIM;
+      uint32_t kvit = 0;
+      bool ok = true;
+      for (int w = w_begin; w < w_end && ok; ++w) {
+        const AttnItem t = w == w_begin ? first_item : args.items[w];
+        const int g = t.unit / pairs;
+        const int nb = t.blk_end - t.blk_begin;
+        const int32_t* pt = args.page_table + t.ctx0;
+        for (int jb = 0; jb < nb; ++jb, ++kvit) {
+          const int st = kvit & 1;
+          const uint32_t ph = (kvit >> 1) & 1u;
+          const int blk = t.blk_begin + jb;
+          ok = mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) { cta_failed = 1; break; }
+          uint8_t* tile = k_smem + st * TILE_BYTES;
+#pragma unroll 4
+          for (int rr = 0; rr < BLK / 8; ++rr) {
+            const int row = r0 + 8 * rr;
+            const int page = __ldg(pt + blk * (BLK / PAGE_TOKENS) + (row >> 4));
+            const int pos = min(blk * BLK + row, args.rope_rows - 1);     // slots past the prompt are masked anyway
+            const __nv_bfloat16* src = args.kpool + (static_cast<size_t>(page) * PAGE_TOKENS + (row & 15)) * kv_dim +
+                                       g * HEAD_DIM + j * 8;
+            const uint4 vlo = ld_dep_v4(src), vhi = ld_dep_v4(src + ROPE_HALF);
+            const float4* csp = reinterpret_cast<const float4*>(args.rope + static_cast<size_t>(pos) * ROPE_HALF + j * 8);
+            const float4 c0 = __ldg(csp), c1 = __ldg(csp + 1), c2 = __ldg(csp + 2), c3 = __ldg(csp + 3);
+            const float cs[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
+            const uint32_t wl[4] = {vlo.x, vlo.y, vlo.z, vlo.w}, wh[4] = {vhi.x, vhi.y, vhi.z, vhi.w};
+            uint32_t ol[4], oh[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {          // two bf16 elements per 32-bit word
+              const float l0 = __uint_as_float(wl[q] << 16), l1 = __uint_as_float(wl[q] & 0xffff0000u);
+              const float h0 = __uint_as_float(wh[q] << 16), h1 = __uint_as_float(wh[q] & 0xffff0000u);
+              const float ca = cs[4 * q], sa = cs[4 * q + 1], cb = cs[4 * q + 2], sb = cs[4 * q + 3];
+              ol[q] = pack_half2(l0 * ca - h0 * sa, l1 * cb - h1 * sb);
+              oh[q] = pack_half2(h0 * ca + l0 * sa, h1 * cb + l1 * sb);
+            }
+            uint8_t* dst = tile + row * 128 + ((j ^ (row & 7)) << 4);
+            *reinterpret_cast<uint4*>(dst) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+            *reinterpret_cast<uint4*>(dst + HALF_TILE_BYTES) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+          }
+          fence_proxy_async_smem();            // the MMA reads the tile through the async proxy
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&k_full[st]);
+        }
+      }
+    }
   } else if (warp == 8) {
     // ---------------------------------------------------------------- TMA producer
     if (lane == 0) {
@@ -204,9 +307,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   } else if (warp == 9) {
     // ---------------------------------------------------------------- MMA issuer
     if (lane == 0) {
-      constexpr int AB = PAGED ? 1 : 0;                                       // operand type: 0 fp16, 1 bf16
-      constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, AB, 0, 0);       // A, B K-major
-      constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, AB, 0, 1);  // B (V) MN-major
+      // operand type of each MMA: 0 fp16, 1 bf16 (both operands of one MMA always have the same type)
+      constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, PAGED ? 1 : 0, 0, 0);          // A, B K-major
+      constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, PV_BF16 ? 1 : 0, 0, 1);   // B (V) MN-major
       uint32_t unit_it = 0, kvit = 0;
       bool ok = true;
       // S_i(kvidx) = Q_i K(kvidx)^T
@@ -346,7 +449,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), args.scale_log2, neg_m));
           sum0 += p0;
           sum1 += p1;
-          if constexpr (PAGED) {            // P in the operand type of V
+          if constexpr (PV_BF16) {          // P in the operand type of V
             __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
             p[c] = *reinterpret_cast<uint32_t*>(&bb);
           } else {
@@ -538,32 +641,38 @@ int make_paged_attn_maps(AttnMaps* out, const __nv_bfloat16* qpool_layer, const 
 
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
-                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table) {
+                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table, int mode,
+                          const __nv_bfloat16* kpool_layer, const float2* rope, int rope_rows) {
   if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
-  if (group < 2 || group % 2 != 0) return -1;
-  const bool paged = page_table != nullptr;
-  static bool smem_set[2][MAX_DEVICES] = {};   // once per device: the call costs host time on every launch otherwise
+  if (group < 2 || group % 2 != 0 || mode < 0 || mode > 2) return -1;
+  if (mode != 0 && page_table == nullptr) return -1;
+  if (mode == 2 && (kpool_layer == nullptr || rope == nullptr || rope_rows <= 0)) return -1;
+  static bool smem_set[3][MAX_DEVICES] = {};   // once per device: the call costs host time on every launch otherwise
   const int dev = current_device_slot();
-  if (!smem_set[paged][dev]) {
-    const cudaError_t e = paged ? cudaFuncSetAttribute(umma_attention_kernel<true>,
-                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
-                                : cudaFuncSetAttribute(umma_attention_kernel<false>,
-                                                       cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
+  if (!smem_set[mode][dev]) {
+    const cudaError_t e =
+        mode == 0 ? cudaFuncSetAttribute(umma_attention_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
+        : mode == 1 ? cudaFuncSetAttribute(umma_attention_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
+                    : cudaFuncSetAttribute(umma_attention_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
     if (e != cudaSuccess) return -1;
-    smem_set[paged][dev] = true;
+    smem_set[mode][dev] = true;
   }
   AttnArgs a{};
   a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out; a.page_table = page_table;
+  a.kpool = kpool_layer; a.rope = rope; a.rope_rows = rope_rows;
   a.partial_o = partial_o; a.partial_ml = partial_ml;
   a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
   a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
   a.err_word = err_word;
-  if (paged)
-    return launch_pdl(umma_attention_kernel<true>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k,
-                      maps.v, a) == cudaSuccess ? 0 : -1;
-  return launch_pdl(umma_attention_kernel<false>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k,
-                    maps.v, a) == cudaSuccess ? 0 : -1;
+  cudaError_t rc;
+  if (mode == 1)
+    rc = launch_pdl(umma_attention_kernel<1>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
+  else if (mode == 2)
+    rc = launch_pdl(umma_attention_kernel<2>, dim3(n_ctas), dim3(ATT_THREADS_ROT), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
+  else
+    rc = launch_pdl(umma_attention_kernel<0>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
+  return rc == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace pc

@@ -96,6 +96,7 @@ __device__ __forceinline__ void qkv_store4_cs(const QkvEpilogue& e, int row, con
               l3 = __bfloat162float(bl3);
   const float h0 = __bfloat162float(bh0), h1 = __bfloat162float(bh1), h2 = __bfloat162float(bh2),
               h3 = __bfloat162float(bh3);
+  if (e.skip_ctx) return;
   __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(rw.slot) * kv_dim + kvh * HEAD_DIM + c;
   if (is_k) {
     *reinterpret_cast<uint2*>(dst) = pack_half4(l0 * t0.x - h0 * t0.y, l1 * t0.z - h1 * t0.w, l2 * t1.x - h2 * t1.y,

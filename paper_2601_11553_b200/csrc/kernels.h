@@ -121,6 +121,9 @@ struct QkvEpilogue {
   // after rotation (what the attention uses and what the cache then holds); q_out, kctx, vctx are unused.
   __nv_bfloat16* qpool;       // layer base: [pool_pages*16][q_dim], or nullptr outside that mode
   int32_t paged;
+  // Gather-free form of the default mode: the attention reads K and V from the pages, so nothing is written to the
+  // assembled context (every row then has a page slot).
+  int32_t skip_ctx;
 };
 struct ResidualEpilogue { float* resid; int32_t ld; };          // resid[row][col] += acc
 struct SwigluEpilogue { __half* act; int32_t ld; };             // act[row][j] = silu(gate) * up
@@ -169,9 +172,16 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
                    const __half* vctx_layer, int64_t ctx_cap, int kv_dim);
 // partial_o: fp32 [slots][2 heads][128 rows][128]; partial_ml: fp32 [slots][2][128][2] (reference max, sum).
 // CTA c (of n_ctas) runs items [cta_first[c], cta_first[c + 1]).
+// mode 0: Q from the query buffer, K/V from the assembled context (maps over those buffers).
+// mode 1: Q, K, V from the pages (maps from make_paged_attn_maps; paper-faithful mode).
+// mode 2: Q from the query buffer (maps.q), V from the pages (maps.v), K loaded from kpool_layer through the page
+//         table and rotated on load with the (cos, sin) table `rope` of rope_rows positions; maps.k is unused.
+// In modes 1 and 2 an item's ctx0 is the index of its prompt's first entry in page_table.
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
-                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table = nullptr);
+                          int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table = nullptr,
+                          int mode = 0, const __nv_bfloat16* kpool_layer = nullptr, const float2* rope = nullptr,
+                          int rope_rows = 0);
 // Maps for the paged form of the attention (paper-faithful mode): Q, K and V are read straight from the bf16 pages
 // of one layer, 16 rows (one page) per bulk copy; an item's ctx0 then is the index of its prompt's first entry in
 // page_table (one page id per 16 context slots, padded to whole 128-slot blocks).

@@ -30,16 +30,19 @@ struct LayerWeights {
   GemmOperand m_wqkv256, m_wo256, m_wgu256, m_wd256;      // and with 256-row boxes
   AttnMaps attn_maps;
   AttnMaps paged_maps;                                    // paper-faithful mode: Q, K, V pages of this layer
+  AttnMaps gf_maps;                                       // gather-free default mode: query buffer + V pages
 };
 
 struct Plan {   // integer description of the last successful call (host)
   std::vector<int32_t> cu_ctx, cu_new, slot_chunk, slot_offset, slot_is_new, row_slot;
   std::vector<int32_t> ctx0;      // device context slot of every prompt's slot 0 (prompts are decode_reserve apart)
   std::vector<int32_t> dec_len;   // tokens appended to every prompt by percache_decode since the prefill
+  bool ctx_assembled = true;      // false after a gather-free call: there is no contiguous context to read or extend
 };
 
 constexpr int MAX_EVENTS = 1024;
 constexpr int64_t GATHER_OVERLAP_MIN_BYTES = 512ll << 20;   // below this the per-layer waits cost more than they hide
+constexpr int64_t GATHER_FREE_MIN_RATIO = 8;                // cached tokens per new row from which the fetch is skipped
 
 // Key of a path of chunk ids (prefix mode): fold the ids with a 64-bit mixer (the SplitMix64 output function).
 constexpr uint64_t PATH_KEY_SEED = 0x70657263616368ull;
@@ -307,7 +310,8 @@ DevIndex dev_index(const percache* h) {
 // projection, RMSNorm, SwiGLU FFN.  Layer l's attention first waits for ev_gather[l] when the fetch runs beside.
 // n_decode_items > 0: the attention work is a decode step's list of DecodeAttnItem / DecodeAttnMerge records.
 bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_merges, bool overlap_gather,
-                bool use_ref, PhaseTimer& timer, cudaStream_t s, int n_decode_items = 0) {
+                bool use_ref, PhaseTimer& timer, cudaStream_t s, int n_decode_items = 0,
+                const int32_t* gather_free_page_table = nullptr) {
   const ModelDims& D = h->dims;
   const int d = D.d_model;
   const size_t pool_layer = static_cast<size_t>(h->cfg.pool_pages) * PAGE_TOKENS * D.kv_dim;
@@ -321,6 +325,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   // A handful of rows (decode) is a matter of reading the weights once: CUDA-core kernels bound by HBM, with the
   // RMSNorm folded into the QKV and gate/up projections
   const bool small_rows = !use_ref && !(h->flags & PERCACHE_FLAG_NO_SMALL_ROW_KERNELS) && Mi <= SMALL_GEMM_MAX_ROWS &&
+                          gather_free_page_table == nullptr &&
                           d % 256 == 0 && D.q_dim % 256 == 0 && D.d_ffn % 256 == 0;
   bool ok = true;
   // debugging aid: the residual stream as it enters layer l goes to capture_host[l] (stream order does the rest)
@@ -348,6 +353,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
     qe.vctx = h->vctx + l * ctx_layer;
     qe.n_q_heads = D.n_q_heads;
     qe.n_kv_heads = D.n_kv_heads;
+    qe.skip_ctx = gather_free_page_table != nullptr ? 1 : 0;
     timer.begin(PERCACHE_PH_QKV);
     if (small_rows) {
       ok = ok && launch_small_gemm(EPI_QKV, &qe, Mi, D.qkv_dim, d, h->resid, W.g_attn, D.rms_eps, nullptr, W.wqkv, 0,
@@ -374,6 +380,12 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
                                          reinterpret_cast<const DecodeAttnMerge*>(d_merges), n_merges, h->qbuf, qe.kctx,
                                          qe.vctx, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads,
                                          s) == 0;
+    } else if (gather_free_page_table != nullptr) {
+      // K and V straight from the pages (K rotated on load): no assembled context
+      ok = ok && launch_umma_attention(W.gf_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
+                                       h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s,
+                                       gather_free_page_table, 2, qe.kpool, h->rope, h->cfg.max_prompt_tokens) == 0;
+      launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
     } else {
       ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
                                        h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s) == 0;
@@ -701,7 +713,7 @@ int prefill_paper(percache* h, const percache_prompt_t* prompts, int32_t n_promp
     timer.begin(PERCACHE_PH_ATTN);
     ok = ok && launch_umma_attention(W.paged_maps, ix.attn_items, ix.cta_first, n_attn_ctas, ix.row_ctx0, h->attn_out,
                                      h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s,
-                                     d_page_table) == 0;
+                                     d_page_table, 1) == 0;
     launch_attention_merge(ix.merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
     timer.end();
     ResidualEpilogue re{h->resid, d};
@@ -754,6 +766,7 @@ int prefill_paper(percache* h, const percache_prompt_t* prompts, int32_t n_promp
   refresh_page_stats(h);
   st.host_plan_us = plan_us;
   st.attn_visible_pairs = visible_pairs;
+  st.gather_free = 1;            // this mode never gathers
   float ms = 0.f;
   cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
   st.device_us = 1000.0 * ms;
@@ -889,11 +902,10 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
   cudaMemsetAsync(h->attn_out, 0, static_cast<size_t>(h->m_cap) * D.q_dim * 2, h->stream);
   cudaMemsetAsync(h->xn, 0, static_cast<size_t>(h->m_cap) * d * 2, h->stream);
   cudaMemsetAsync(h->act, 0, static_cast<size_t>(h->m_cap) * F * 2, h->stream);
-  if (h->paper_mode) {      // there the attention copies whole pages, also ones a prompt only partly fills
-    cudaMemsetAsync(h->qpool, 0, qpool_elems * 2, h->stream);
-    cudaMemsetAsync(h->kpool, 0, pool_elems * 2, h->stream);
-    cudaMemsetAsync(h->vpool, 0, pool_elems * 2, h->stream);
-  }
+  // the paged forms of the attention copy whole pages, also ones a prompt only partly fills
+  if (h->paper_mode) cudaMemsetAsync(h->qpool, 0, qpool_elems * 2, h->stream);
+  cudaMemsetAsync(h->kpool, 0, pool_elems * 2, h->stream);
+  cudaMemsetAsync(h->vpool, 0, pool_elems * 2, h->stream);
 
   // ---- weights: bf16 -> fp16 copies in the layouts the GEMMs read.  Every bf16 value of magnitude
   // >= 2^-17 is exactly representable in fp16; smaller ones round with absolute error <= 2^-25.
@@ -942,6 +954,15 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
               make_operand_map(&W.m_wgu256, W.wgu, 2 * F, d, 256) == 0 && make_operand_map(&W.m_wd256, W.wd, d, F, 256) == 0;
     cuda_ok = cuda_ok && make_attn_maps(&W.attn_maps, h->qbuf, h->m_cap, D.q_dim, h->kctx + l * ctx_layer,
                                         h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim) == 0;
+    {
+      // gather-free form of the default mode: Q as above, V one page (16 rows) of a 64-column half per copy
+      const size_t pl = static_cast<size_t>(cfg->pool_pages) * PAGE_TOKENS;
+      W.gf_maps = W.attn_maps;
+      const uint32_t box[2] = {64u, static_cast<uint32_t>(PAGE_TOKENS)};
+      const uint64_t vd[2] = {static_cast<uint64_t>(D.kv_dim), static_cast<uint64_t>(pl)};
+      const uint64_t vs[1] = {static_cast<uint64_t>(D.kv_dim) * 2};
+      cuda_ok = cuda_ok && encode_f16_map(&W.gf_maps.v, h->vpool + l * pl * D.kv_dim, 2, vd, vs, box) == 0;
+    }
     if (h->paper_mode) {
       const size_t pl = static_cast<size_t>(cfg->pool_pages) * PAGE_TOKENS;
       cuda_ok = cuda_ok && make_paged_attn_maps(&W.paged_maps, h->qpool + l * pl * D.q_dim, h->kpool + l * pl * D.kv_dim,
@@ -1194,6 +1215,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   plan.cu_new.assign(1, 0);
   int64_t ctx_total = 0, new_total = 0, hit_tokens = 0, pages_needed = 0, visible_pairs = 0;
   int chunks_hit = 0, chunks_missed = 0;
+  // for the gather-free form: whether every stretch of slots starts on a page boundary, how many pages the rows that
+  // are not chunk content to be stored would need for the duration of the call, and the size of the page tables
+  bool page_aligned = true;
+  int64_t scratch_pages = 0, pt_entries = 0;
   for (int b = 0; b < n_prompts; ++b) {
     const percache_prompt_t& P = prompts[b];
     if (P.n_query < 0 || (P.n_chunks > 0 && !P.chunk_len) || (P.n_query > 0 && !P.query_hidden))
@@ -1204,6 +1229,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     for (int i = 0; i < P.n_chunks; ++i) {
       const int len = P.chunk_len[i];
       if (len <= 0) return PERCACHE_E_INVAL;
+      if (len % PAGE_TOKENS != 0) page_aligned = false;
       const uint64_t key = keys[b][i];
       auto it = h->table.find(key);
       const bool stored = it != h->table.end();
@@ -1222,6 +1248,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
         if (!stored && !first_miss.count(key)) {
           first_miss.emplace(key, std::make_pair(b, i));
           pages_needed += (len + PAGE_TOKENS - 1) / PAGE_TOKENS;
+        } else {
+          scratch_pages += (len + PAGE_TOKENS - 1) / PAGE_TOKENS;     // computed but not kept
         }
       }
       T += len;
@@ -1238,10 +1266,14 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
         if (!P.chunk_hidden || !P.chunk_hidden[last_hit[b]]) return PERCACHE_E_MISS_NO_INPUT;
         n_new += P.reuse_tail_drop;
         hit_tokens -= P.reuse_tail_drop;
+        if (P.reuse_tail_drop % PAGE_TOKENS != 0) page_aligned = false;
+        scratch_pages += P.reuse_tail_drop / PAGE_TOKENS;
       }
     }
+    scratch_pages += (P.n_query + PAGE_TOKENS - 1) / PAGE_TOKENS;
     T += P.n_query;
     n_new += P.n_query;
+    pt_entries += (T + 127) / 128 * (128 / PAGE_TOKENS);
     if (T <= 0) return PERCACHE_E_INVAL;
     if (T > h->cfg.max_prompt_tokens) return PERCACHE_E_CAPACITY;
     if (results[b].out_capacity_rows < n_new || (n_new > 0 && !results[b].out_hidden)) return PERCACHE_E_CAPACITY;
@@ -1252,6 +1284,19 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     plan.cu_ctx.push_back(static_cast<int32_t>(ctx_total));
     plan.cu_new.push_back(static_cast<int32_t>(new_total));
   }
+  // Gather-free form (paper Section 3.2.2 loads and concatenates the matched tensors; here the attention reads them
+  // where they are): K and V of every slot stay in 16-token pages, the attention walks the prompt's page table and
+  // rotates K on load, and the fetch -- a read, a write and a re-read of every cached K and V byte -- disappears.
+  // Taken when the cached part dominates (the fetch would move more bytes than the attention reads), or on request;
+  // possible when every stretch of slots is page-aligned, nothing is to be decoded afterwards (that needs the
+  // contiguous context) and the tcgen05 attention runs.  The rows of the call that are not chunk content to be
+  // stored then need pages of their own while the call lasts.
+  const bool gather_free =
+      page_aligned && hit_tokens > 0 && new_total > 0 && h->decode_reserve == 0 &&
+      !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION | PERCACHE_FLAG_ALWAYS_GATHER)) &&
+      static_cast<size_t>(pt_entries) <= 4 * static_cast<size_t>(h->ctx_cap) &&
+      ((h->flags & PERCACHE_FLAG_GATHER_FREE) || hit_tokens >= GATHER_FREE_MIN_RATIO * new_total);
+  if (gather_free) pages_needed += scratch_pages;
   // every argument check has passed: choose what would have to be evicted so that the new pages fit (never a chunk
   // this batch hits).  The store itself changes only when the device work is about to start (PageTxn::apply).
   PageTxn txn(h);
@@ -1262,6 +1307,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     txn.set_victims(victims);
   }
   const int evicted = static_cast<int>(txn.victims.size());
+  std::vector<int32_t> scratch;                   // gather-free form: pages that only live for this call
 
   // ---------------------------------------------------------------- pages for the chunks that will be stored
   std::vector<std::pair<uint64_t, ChunkEntry>> pending;
@@ -1304,6 +1350,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   AttnMerge* merges = reinterpret_cast<AttnMerge*>(cta_first + h->n_sms + 1);
   std::vector<AttnBaseTile> base_tiles;
   int n_items = 0, n_attn_ctas = 0, n_merges = 0;
+  int32_t* page_table = reinterpret_cast<int32_t*>(items);     // gather-free form: in place of the gather items
+  int32_t pt_next = 0;
   plan.slot_chunk.resize(static_cast<size_t>(ctx_total));
   plan.slot_offset.resize(static_cast<size_t>(ctx_total));
   plan.slot_is_new.resize(static_cast<size_t>(ctx_total));
@@ -1313,6 +1361,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     const percache_prompt_t& P = prompts[b];
     const int32_t pbase = plan.cu_ctx[b];                              // index into the plan's per-slot arrays
     const int32_t ctx0 = pbase + b * h->decode_reserve;                // slot in the device context
+    const int32_t pt0 = pt_next;                                       // gather-free form: first entry of its page table
     plan.ctx0.push_back(ctx0);
     plan.dec_len.push_back(0);
     int32_t t = 0;
@@ -1331,12 +1380,16 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       }
       if (reuse_len > 0) {
         const ChunkEntry& ent = h->table.find(keys[b][i])->second;
-        for (int o = 0; o < reuse_len; o += PAGE_TOKENS) {
-          GatherItem& g = items[n_items++];
-          g.dst_slot = ctx0 + t + o;
-          g.src_page = ent.pages[o / PAGE_TOKENS];
-          g.n_tok = std::min(PAGE_TOKENS, reuse_len - o);
-          g.pos = t + o;
+        if (gather_free) {
+          for (int o = 0; o < reuse_len; o += PAGE_TOKENS) page_table[pt_next++] = ent.pages[o / PAGE_TOKENS];
+        } else {
+          for (int o = 0; o < reuse_len; o += PAGE_TOKENS) {
+            GatherItem& g = items[n_items++];
+            g.dst_slot = ctx0 + t + o;
+            g.src_page = ent.pages[o / PAGE_TOKENS];
+            g.n_tok = std::min(PAGE_TOKENS, reuse_len - o);
+            g.pos = t + o;
+          }
         }
       }
       if (reuse_len < len) {
@@ -1346,13 +1399,25 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
           if (fm != first_miss.end() && fm->second.first == b && fm->second.second == i)
             ent = &pending[pending_of[keys[b][i]]].second;
         }
+        // gather-free form: rows that will not be stored still need page slots while the call lasts
+        std::vector<int32_t> tmp_pages;
+        if (gather_free && !ent) {
+          if (txn.take((len - reuse_len + PAGE_TOKENS - 1) / PAGE_TOKENS, &tmp_pages) != PERCACHE_OK)
+            return fail(PERCACHE_E_NOSPACE);
+          scratch.insert(scratch.end(), tmp_pages.begin(), tmp_pages.end());
+        }
+        if (gather_free)
+          for (int o = reuse_len; o < len; o += PAGE_TOKENS)
+            page_table[pt_next++] = ent ? ent->pages[o / PAGE_TOKENS] : tmp_pages[(o - reuse_len) / PAGE_TOKENS];
         const char* src = static_cast<const char*>(is_query ? P.query_hidden : P.chunk_hidden[i]);
         segs.push_back(Seg{src + static_cast<size_t>(reuse_len) * d * 2, P.hidden_on_device, static_cast<int>(r),
                            len - reuse_len});
         for (int o = reuse_len; o < len; ++o, ++r) {
           row_slot[r] = ctx0 + t + o;
           row_pos[r] = t + o;
-          row_pool[r] = ent ? ent->pages[o / PAGE_TOKENS] * PAGE_TOKENS + (o % PAGE_TOKENS) : -1;
+          row_pool[r] = ent ? ent->pages[o / PAGE_TOKENS] * PAGE_TOKENS + (o % PAGE_TOKENS)
+                            : (gather_free ? tmp_pages[(o - reuse_len) / PAGE_TOKENS] * PAGE_TOKENS + ((o - reuse_len) % PAGE_TOKENS)
+                                           : -1);
           row_ctx0[r] = ctx0;
           plan.row_slot[r] = t + o;
           visible_pairs += t + o + 1;
@@ -1360,11 +1425,15 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       }
       t += len;
     }
+    if (gather_free && pt_next > pt0) {     // pad the table to whole 128-slot blocks (those slots are never visible)
+      const int32_t last_page = page_table[pt_next - 1];
+      while ((pt_next - pt0) % (128 / PAGE_TOKENS) != 0) page_table[pt_next++] = last_page;
+    }
     for (int32_t r0 = plan.cu_new[b]; r0 < plan.cu_new[b + 1]; r0 += 128) {
       AttnBaseTile a{};
       a.row0 = r0;
       a.n_rows = std::min(128, plan.cu_new[b + 1] - r0);
-      a.ctx0 = ctx0;
+      a.ctx0 = gather_free ? pt0 : ctx0;           // the paged attention reads ctx0 as its page-table offset
       a.n_blocks = (row_pos[r0 + a.n_rows - 1] + 1 + 127) / 128;     // context blocks its last row can see
       base_tiles.push_back(a);
     }
@@ -1440,7 +1509,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
                          h->ctx_cap, D.kv_dim, h->rope, s);
     timer.end();
   }
-  ok = ok && (Mi <= 0 || run_layers(h, Mi, dix, n_attn_ctas, n_merges, overlap_gather, use_ref, timer, s));
+  ok = ok && (Mi <= 0 || run_layers(h, Mi, dix, n_attn_ctas, n_merges, overlap_gather, use_ref, timer, s, 0,
+                                    gather_free ? reinterpret_cast<const int32_t*>(dix.items) : nullptr));
   cudaEventRecord(h->ev_end, s);
   timer.begin(PERCACHE_PH_IO);
   for (int b = 0; b < n_prompts && ok; ++b) {
@@ -1460,6 +1530,8 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   // ---------------------------------------------------------------- commit
   for (auto& pe : pending) h->table.emplace(pe.first, std::move(pe.second));
   for (const auto& hu : hit_uses) h->table[hu.first].retrievals += hu.second;
+  release_pages(h, scratch);
+  plan.ctx_assembled = !gather_free;
   st.evictions = evicted;
   for (int b = 0; b < n_prompts; ++b) {
     results[b].n_new = plan.cu_new[b + 1] - plan.cu_new[b];
@@ -1477,6 +1549,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   refresh_page_stats(h);
   st.host_plan_us = plan_us;
   st.attn_visible_pairs = visible_pairs;
+  st.gather_free = gather_free ? 1 : 0;
   float ms = 0.f;
   cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
   st.device_us = 1000.0 * ms;
@@ -1502,6 +1575,7 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   if (!h || !hidden || !out_hidden || n_prompts <= 0 || h->paper_mode) return PERCACHE_E_INVAL;
   Plan& plan = h->plan;
   if (static_cast<size_t>(n_prompts) + 1 != plan.cu_ctx.size()) return PERCACHE_E_INVAL;   // not the last call's batch
+  if (!plan.ctx_assembled) return PERCACHE_E_INVAL;      // the last prefill ran gather-free: no context to append to
   if (n_prompts > h->m_cap) return PERCACHE_E_CAPACITY;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   const auto t_host0 = std::chrono::steady_clock::now();
@@ -1622,6 +1696,7 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   st.host_plan_us = plan_us;
   st.attn_visible_pairs = visible_pairs;
   st.evictions = 0;
+  st.gather_free = 0;
   float ms = 0.f;
   cudaEventElapsedTime(&ms, h->ev_begin, h->ev_end);
   st.device_us = 1000.0 * ms;
@@ -1684,7 +1759,7 @@ int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int
 
 int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host) {
   if (!h || !k_host || !v_host || layer < 0 || layer >= h->dims.n_layers || prompt < 0 ||
-      prompt + 1 >= static_cast<int32_t>(h->plan.cu_ctx.size()))
+      prompt + 1 >= static_cast<int32_t>(h->plan.cu_ctx.size()) || !h->plan.ctx_assembled || h->paper_mode)
     return PERCACHE_E_INVAL;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * h->dims.kv_dim;

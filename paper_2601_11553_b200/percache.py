@@ -28,6 +28,7 @@ FLAG_REFERENCE_KERNELS, FLAG_PHASE_TIMING, FLAG_REFERENCE_ATTENTION, FLAG_EVICT_
 FLAG_SINGLE_CTA_GEMM = 16
 FLAG_NO_SMALL_ROW_KERNELS = 32
 FLAG_PAPER_MODE = 64
+FLAG_GATHER_FREE, FLAG_ALWAYS_GATHER = 128, 256
 PAGE_TOKENS = 16
 PHASES = ("gather", "norm", "qkv", "attn", "oproj", "gateup", "down", "io")
 EXPORTS = ("percache_create", "percache_destroy", "percache_put_chunk_kv", "percache_prefill",
@@ -71,7 +72,8 @@ class StatsStruct(C.Structure):
                 ("ctx_tokens", C.c_int64), ("hit_tokens", C.c_int64), ("new_rows", C.c_int64),
                 ("pages_used", C.c_int64), ("pages_free", C.c_int64), ("host_plan_us", C.c_double),
                 ("device_us", C.c_double), ("phase_us", C.c_double * len(PHASES)),
-                ("phase_launches", C.c_int32 * len(PHASES)), ("attn_visible_pairs", C.c_int64), ("evictions", C.c_int64)]
+                ("phase_launches", C.c_int32 * len(PHASES)), ("attn_visible_pairs", C.c_int64), ("evictions", C.c_int64),
+                ("gather_free", C.c_int32), ("reserved0", C.c_int32)]
 
 
 _lib = None

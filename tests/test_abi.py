@@ -44,7 +44,7 @@ def test_struct_sizes_match_header():
     assert C.sizeof(pcb.LayerWeights) == 72
     assert C.sizeof(pcb.PromptStruct) == 64
     assert C.sizeof(pcb.ResultStruct) == 40
-    assert C.sizeof(pcb.StatsStruct) == 184
+    assert C.sizeof(pcb.StatsStruct) == 192
 
 
 def test_argument_validation_needs_no_gpu(lib):

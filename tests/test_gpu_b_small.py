@@ -19,7 +19,8 @@ def run_case(w: wl.Workload, flags: int, check_store: bool = True):
     store = G.oracle_store_alone(model, w.seed, [(c, ids_lens[c]) for c in w.cached_ids])
     want = orc.reuse_prefill(model, store, [H.oracle_prompt(p, [i for i, c in enumerate(p.chunk_ids) if c in w.cached_ids])
                                             for p in w.prompts], keep_ctx=True)
-    with G.make_handle(w.shape, weights, w.prompts, flags=flags) as h:
+    # the assembled context is checked bit for bit below, so this pass must assemble one
+    with G.make_handle(w.shape, weights, w.prompts, flags=flags | pcb.FLAG_ALWAYS_GATHER) as h:
         # the oracle committed the misses: push only what was cached before the call
         G.push_store(h, store, w.cached_ids)
         got = h.prefill(G.specs_for(w.prompts, w.cached_ids))

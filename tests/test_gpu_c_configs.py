@@ -32,7 +32,9 @@ def run_workload(w: wl.Workload, ctx_layers=None, random_gains=False):
     want = orc.reuse_prefill(model, store, [H.oracle_prompt(p, [i for i, c in enumerate(p.chunk_ids) if c in cached])
                                             for p in w.prompts], keep_ctx=True, commit=False)
     layers = list(range(w.shape.n_layers)) if ctx_layers is None else ctx_layers
-    with G.make_handle(w.shape, weights, w.prompts) as h:
+    # the assembled context is compared bit for bit, so the contiguous context must be built here; the gather-free
+    # form of the same workloads is checked in test_gpu_l_gather_free.py and, at full size, by the teacher-forced tests
+    with G.make_handle(w.shape, weights, w.prompts, flags=pcb.FLAG_ALWAYS_GATHER) as h:
         if w.cache_source == "integer_pool":
             for c in w.cached_ids:
                 h.put_chunk_synthetic(c, ids_lens[c], w.seed)

@@ -71,7 +71,7 @@ def test_tail_of_the_final_matched_chunk_is_recomputed(drop):
     store = orc.Store()
     h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
                      n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
-                     pool_pages=64, max_prompt_tokens=400, max_batch_prompts=1)
+                     pool_pages=64, max_prompt_tokens=400, max_batch_prompts=1, flags=pcb.FLAG_ALWAYS_GATHER)
     with h:
         warm = [1, 5]
         orc.reuse_prefill(model, store, [orc.Prompt(warm, [lens[c] for c in warm], [f64(hid[c]) for c in warm],
