@@ -506,7 +506,8 @@ class Bench:
 def table_row(r, world, steps):
     """Compact record of one workload for the per-workload table."""
     w = r["w"]
-    row = {"workload": w.name, "ms_per_step": r["total_ms"] / steps,
+    row = {"workload": w.name, "form": "gather-free" if r["st"].get("gather_free") else "gather",
+           "ms_per_step": r["total_ms"] / steps,
            "tokens_per_s": aggregate_tokens_per_s(world, w.total_tokens, steps, r["total_ms"]),
            "new_rows": r["new_rows"], "hit_tokens": int(r["st"]["hit_tokens"]), "steps": steps,
            "tensor_peak": {"tflops": r["tensor_peak"], "which": r["which_peak"]},
@@ -578,6 +579,14 @@ def run_gpu(args):
                 if not args.no_cpu_baseline:
                     row["cpu_baseline"] = cpu_baseline_for(w)
                 rows.append(row)
+            # a workload the library serves in its gather-free form is also timed in the form that assembles the
+            # context, so that the fetch kernel's bandwidth is on record for it
+            if r["st"].get("gather_free") and not w.paper_mode and not (args.flags & pcb.FLAG_ALWAYS_GATHER) and not args.no_table:
+                r2 = b.measure(w, max(3, min(steps, 10)), args.warmup, args.flags | pcb.FLAG_ALWAYS_GATHER, False, barrier, dist)
+                if rank == 0:
+                    row2 = table_row(r2, world, max(3, min(steps, 10)))
+                    row2["workload"] = w.name + " (gather form)"
+                    rows.append(row2)
         b.close()
         del b
         torch.cuda.empty_cache()
@@ -621,7 +630,8 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": r["total_ms"] / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f16", "data": "synthetic",
-        "config": {"workload": w.name, "reduced_depth": args.layers > 0, "description": w.description,
+        "config": {"workload": w.name, "form": "gather-free" if st.get("gather_free") else "gather",
+                   "reduced_depth": args.layers > 0, "description": w.description,
                    "tokens_per_step": tokens, "new_rows_per_step": new_rows, "hit_tokens_per_step": int(st["hit_tokens"]),
                    "prompts_per_step": len(w.prompts), "ms_per_prompt": r["total_ms"] / args.steps / len(w.prompts),
                    "computed_rows_per_s": world * new_rows * args.steps / (r["total_ms"] / 1000.0),

@@ -179,8 +179,8 @@ typedef struct {
  * (K rotated to its position there) and lets the attention read that.  The gather-free one leaves them in their
  * pages: the attention walks the prompt's page table, rotates K as it loads it and reads V where it is, so the fetch
  * and its traffic disappear; there P and V enter the second attention product as bf16 (the store's format) instead
- * of fp16.  It is taken when the batch has at least 8 cached tokens per new row (or PERCACHE_FLAG_GATHER_FREE is
- * set), every chunk length and reuse_tail_drop is a multiple of 16, no decode reserve is set and
+ * of fp16.  It is taken when the batch has at least 8 cached tokens per new row and no prompt more than 256 new rows
+ * (or PERCACHE_FLAG_GATHER_FREE is set), every chunk length and reuse_tail_drop is a multiple of 16, no decode reserve is set and
  * PERCACHE_FLAG_ALWAYS_GATHER is not; rows that are not stored (query tokens) then occupy pages of the store for the
  * duration of the call (they count against the store limit).  After a gather-free call there is no assembled
  * context: percache_decode and percache_debug_read_ctx return PERCACHE_E_INVAL. */

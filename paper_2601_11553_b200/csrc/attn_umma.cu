@@ -32,6 +32,10 @@ constexpr int HALF_TILE_BYTES = BLK * 64 * 2;  // 16 KB: 128 rows x 64 fp16 (one
 constexpr int TILE_BYTES = 2 * HALF_TILE_BYTES;
 constexpr int KV_STAGES = 2;
 constexpr int ATT_SMEM_BYTES = 2 * TILE_BYTES + 2 * KV_STAGES * TILE_BYTES + 1024;
+// MODE 2 stages the unrotated K pages of half a block (64 slots) at a time in a ring of two slots: 2 x 16 KB more
+constexpr int KRAW_ROWS = 64;
+constexpr int KRAW_SLOT_BYTES = 2 * KRAW_ROWS * 128;       // two 64-column halves of 64 rows
+constexpr int ATT_SMEM_BYTES_ROT = ATT_SMEM_BYTES + 2 * KRAW_SLOT_BYTES;
 constexpr uint32_t TMEM_S0 = 0, TMEM_O0 = 256;
 constexpr float RESCALE_THRESHOLD = 8.0f;
 
@@ -40,7 +44,6 @@ struct AttnArgs {
   const int32_t* cta_first;
   const int32_t* row_pos;
   const int32_t* page_table;      // paged forms: one page id per 16 context slots; an item's ctx0 indexes its prompt's first entry
-  const __nv_bfloat16* kpool;     // MODE 2: this layer's K pages [pool_pages * 16][kv_dim], unrotated bf16
   const float2* rope;             // MODE 2: (cos, sin)[position][64]
   int32_t rope_rows;              // MODE 2: positions the table covers
   __half* out;
@@ -86,6 +89,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   __shared__ __align__(8) uint64_t q_full, q_empty;
   __shared__ __align__(8) uint64_t k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ __align__(8) uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+  __shared__ __align__(8) uint64_t kraw_full[2], kraw_empty[2];      // MODE 2: the ring of staged, unrotated K pages
   __shared__ uint32_t tmem_base_slot;
   __shared__ int cta_failed;       // set by any role whose bounded wait ran out (or saw another role's error)
 
@@ -95,6 +99,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
   uint8_t* q_smem = base;                                   // [2 heads][2 halves][128][64]
   uint8_t* k_smem = base + 2 * TILE_BYTES;                  // [stages][2 halves][128][64]
   uint8_t* v_smem = k_smem + KV_STAGES * TILE_BYTES;
+  uint8_t* kraw_smem = v_smem + KV_STAGES * TILE_BYTES;     // MODE 2: [2 slots][2 halves][64][64] bf16
 
   // The work list and the row positions are written by the host before the first kernel of the call, not by the
   // kernel this one depends on: they are read ahead of the dependency wait, while the prologue runs.
@@ -118,6 +123,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     for (int i = 0; i < 2; ++i) {
       mbar_init(&s_full[i], 1); mbar_init(&p_full[i], 4);
       mbar_init(&o_done[i], 1); mbar_init(&o_free[i], 4);
+      mbar_init(&kraw_full[i], 1); mbar_init(&kraw_empty[i], 2);
     }
     fence_mbar_init();
   }
@@ -183,8 +189,9 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
     }
   } else if (warp == 8 && MODE == 2) {
     // ---------------------------------------------------------------- TMA producer, MODE 2: Q tiles from the query
-    // buffer (lanes 0-3, one 128-row box each), V blocks from the pages (lanes 0-15, one page each)
-    uint32_t unit_it = 0, kvit = 0;
+    // buffer (lanes 0-3, one 128-row box each); per context block the unrotated K pages into the staging ring, half a
+    // block (four pages x two 64-column halves = lanes 16-23) at a time, and the V pages into the V ring (lanes 0-15).
+    uint32_t unit_it = 0, kvit = 0, rawit = 0;
     bool ok = true;
     const int pg = lane & 7, hf = (lane >> 3) & 1;
     for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
@@ -201,10 +208,24 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       if (lane < 4)
         tma_load_2d(q_smem + (lane >> 1) * TILE_BYTES + (lane & 1) * HALF_TILE_BYTES, &tmQ, &q_full,
                     (h0 + (lane >> 1)) * HEAD_DIM + (lane & 1) * 64, t.row0);
-      for (int j = 0; j < nb; ++j, ++kvit) {
+      for (int j = 0; j < nb && ok; ++j, ++kvit) {
         const int st = kvit & 1;
         const uint32_t ph = (kvit >> 1) & 1u;
-        const int v_page = __ldg(pt + (t.blk_begin + j) * (BLK / PAGE_TOKENS) + pg);
+        const int page = __ldg(pt + (t.blk_begin + j) * (BLK / PAGE_TOKENS) + pg);     // page of rows 16 pg .. 16 pg + 15
+        for (int half = 0; half < 2 && ok; ++half, ++rawit) {
+          const int slot = rawit & 1;
+          ok = mbar_wait(&kraw_empty[slot], ((rawit >> 1) & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+          ok = __all_sync(0xffffffffu, ok);
+          if (!ok) { cta_failed = 1; break; }
+          if (lane == 0) mbar_arrive_expect_tx(&kraw_full[slot], KRAW_SLOT_BYTES);
+          __syncwarp();
+          // lane 16 + 4 hf + q copies page (4 half + q) of the block: its 64-column half hf, into rows 16 q .. of the slot
+          const int src_page = __shfl_sync(0xffffffffu, page, 4 * half + (lane & 3));
+          if (lane >= 16 && lane < 24)
+            tma_load_2d(kraw_smem + slot * KRAW_SLOT_BYTES + ((lane >> 2) & 1) * (KRAW_ROWS * 128) + (lane & 3) * (PAGE_TOKENS * 128),
+                        &tmK, &kraw_full[slot], g * HEAD_DIM + ((lane >> 2) & 1) * 64, src_page * PAGE_TOKENS);
+        }
+        if (!ok) break;
         ok = mbar_wait(&v_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) { cta_failed = 1; break; }
@@ -212,59 +233,95 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         __syncwarp();
         if (lane < 16)
           tma_load_2d(v_smem + st * TILE_BYTES + hf * HALF_TILE_BYTES + pg * (PAGE_TOKENS * 128), &tmV, &v_full[st],
-                      g * HEAD_DIM + hf * 64, v_page * PAGE_TOKENS);
+                      g * HEAD_DIM + hf * 64, page * PAGE_TOKENS);
       }
     }
   } else if (warp >= 10) {
-    // ---------------------------------------------------------------- K from the pages, rotated on load (MODE 2 only:
+    // ---------------------------------------------------------------- K rotated on its way to the S MMA (MODE 2 only:
     // the other forms are launched without these warps).  64 threads: thread (r0 = tid / 8, j = tid % 8) takes rows
-    // r0, r0 + 8, ... of the block and, in each, the 16-byte vector j of the head's low half and the one of its high
-    // half (elements 8j..8j+7 and 64 + 8j..): together they are eight rotation pairs.  The results go to the place
-    // the 128-byte swizzle gives vector j of that row (j ^ (row & 7)), in both 64-column halves of the tile.
+    // r0, r0 + 8, ... and, in each, the 16-byte vector j of the head's low half and the one of its high half (elements
+    // 8j..8j+7 and 64 + 8j..): together eight rotation pairs.  It reads them from the staged pages, rotates in fp32 and
+    // writes fp16 to the place the 128-byte swizzle gives vector j of that row (j ^ (row & 7)) in both 64-column halves
+    // of the K tile.  The (cos, sin) of a block's first eight rows come from the table (requested one block ahead);
+    // every further row group is eight positions on, i.e. one more complex multiplication by the table's row 8 --
+    // sixteen steps at most before the table is read again.
     if constexpr (MODE == 2) {
       const int tid = (warp - 10) * 32 + lane;
       const int j = tid & 7, r0 = tid >> 3;
-      const int kv_dim = args.n_kv_heads * HEAD_DIM;
-      uint32_t kvit = 0;
+      uint32_t kvit = 0, rawit = 0;
       bool ok = true;
+      float step[16];                                      // (cos, sin) of 8 positions for this thread's eight pairs
+      {
+        const float4* sp = reinterpret_cast<const float4*>(args.rope + static_cast<size_t>(min(8, args.rope_rows - 1)) * ROPE_HALF + j * 8);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 v = __ldg(sp + q);
+          step[4 * q] = v.x; step[4 * q + 1] = v.y; step[4 * q + 2] = v.z; step[4 * q + 3] = v.w;
+        }
+      }
+      auto load_cs = [&](int pos, float (&cs)[16]) {
+        const float4* csp = reinterpret_cast<const float4*>(args.rope + static_cast<size_t>(min(pos, args.rope_rows - 1)) * ROPE_HALF + j * 8);
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          const float4 v = __ldg(csp + q);
+          cs[4 * q] = v.x; cs[4 * q + 1] = v.y; cs[4 * q + 2] = v.z; cs[4 * q + 3] = v.w;
+        }
+      };
+      float cs_next[16];
+      if (w_begin < w_end) load_cs(first_item.blk_begin * BLK + r0, cs_next);
       for (int w = w_begin; w < w_end && ok; ++w) {
         const AttnItem t = w == w_begin ? first_item : args.items[w];
-        const int g = t.unit / pairs;
         const int nb = t.blk_end - t.blk_begin;
-        const int32_t* pt = args.page_table + t.ctx0;
-        for (int jb = 0; jb < nb; ++jb, ++kvit) {
+        for (int jb = 0; jb < nb && ok; ++jb, ++kvit) {
           const int st = kvit & 1;
           const uint32_t ph = (kvit >> 1) & 1u;
-          const int blk = t.blk_begin + jb;
+          float cs[16];
+#pragma unroll
+          for (int q = 0; q < 16; ++q) cs[q] = cs_next[q];
+          // the table row the next block starts from (the next item's first block when this one ends)
+          if (jb + 1 < nb) load_cs((t.blk_begin + jb + 1) * BLK + r0, cs_next);
+          else if (w + 1 < w_end) load_cs(args.items[w + 1].blk_begin * BLK + r0, cs_next);
           ok = mbar_wait(&k_empty[st], ph ^ 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
           ok = __all_sync(0xffffffffu, ok);
           if (!ok) { cta_failed = 1; break; }
           uint8_t* tile = k_smem + st * TILE_BYTES;
-#pragma unroll 4
-          for (int rr = 0; rr < BLK / 8; ++rr) {
-            const int row = r0 + 8 * rr;
-            const int page = __ldg(pt + blk * (BLK / PAGE_TOKENS) + (row >> 4));
-            const int pos = min(blk * BLK + row, args.rope_rows - 1);     // slots past the prompt are masked anyway
-            const __nv_bfloat16* src = args.kpool + (static_cast<size_t>(page) * PAGE_TOKENS + (row & 15)) * kv_dim +
-                                       g * HEAD_DIM + j * 8;
-            const uint4 vlo = ld_dep_v4(src), vhi = ld_dep_v4(src + ROPE_HALF);
-            const float4* csp = reinterpret_cast<const float4*>(args.rope + static_cast<size_t>(pos) * ROPE_HALF + j * 8);
-            const float4 c0 = __ldg(csp), c1 = __ldg(csp + 1), c2 = __ldg(csp + 2), c3 = __ldg(csp + 3);
-            const float cs[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
-            const uint32_t wl[4] = {vlo.x, vlo.y, vlo.z, vlo.w}, wh[4] = {vhi.x, vhi.y, vhi.z, vhi.w};
-            uint32_t ol[4], oh[4];
+          for (int half = 0; half < 2 && ok; ++half, ++rawit) {
+            const int slot = rawit & 1;
+            ok = mbar_wait(&kraw_full[slot], (rawit >> 1) & 1u, args.err_word, DEV_ERR_ATTN_PRODUCER);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) { cta_failed = 1; break; }
+            const uint8_t* raw = kraw_smem + slot * KRAW_SLOT_BYTES;
+#pragma unroll 2
+            for (int rr = 0; rr < KRAW_ROWS / 8; ++rr) {
+              const int rl = r0 + 8 * rr;                      // row inside the staged half block
+              const int row = half * KRAW_ROWS + rl;           // row inside the K tile
+              const int off = rl * 128 + ((j ^ (rl & 7)) << 4);
+              const uint4 vlo = *reinterpret_cast<const uint4*>(raw + off);
+              const uint4 vhi = *reinterpret_cast<const uint4*>(raw + KRAW_ROWS * 128 + off);
+              const uint32_t wl[4] = {vlo.x, vlo.y, vlo.z, vlo.w}, wh[4] = {vhi.x, vhi.y, vhi.z, vhi.w};
+              uint32_t ol[4], oh[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {          // two bf16 elements per 32-bit word
-              const float l0 = __uint_as_float(wl[q] << 16), l1 = __uint_as_float(wl[q] & 0xffff0000u);
-              const float h0 = __uint_as_float(wh[q] << 16), h1 = __uint_as_float(wh[q] & 0xffff0000u);
-              const float ca = cs[4 * q], sa = cs[4 * q + 1], cb = cs[4 * q + 2], sb = cs[4 * q + 3];
-              ol[q] = pack_half2(l0 * ca - h0 * sa, l1 * cb - h1 * sb);
-              oh[q] = pack_half2(h0 * ca + l0 * sa, h1 * cb + l1 * sb);
+              for (int q = 0; q < 4; ++q) {          // two bf16 elements per 32-bit word
+                const float l0 = __uint_as_float(wl[q] << 16), l1 = __uint_as_float(wl[q] & 0xffff0000u);
+                const float h0 = __uint_as_float(wh[q] << 16), h1 = __uint_as_float(wh[q] & 0xffff0000u);
+                const float ca = cs[4 * q], sa = cs[4 * q + 1], cb = cs[4 * q + 2], sb = cs[4 * q + 3];
+                ol[q] = pack_half2(l0 * ca - h0 * sa, l1 * cb - h1 * sb);
+                oh[q] = pack_half2(h0 * ca + l0 * sa, h1 * cb + l1 * sb);
+              }
+              uint8_t* dst = tile + row * 128 + ((j ^ (row & 7)) << 4);
+              *reinterpret_cast<uint4*>(dst) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
+              *reinterpret_cast<uint4*>(dst + HALF_TILE_BYTES) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+#pragma unroll
+              for (int q = 0; q < 8; ++q) {          // eight positions on: (c, s) <- (c, s) * (c8, s8)
+                const float c = cs[2 * q], sn = cs[2 * q + 1];
+                cs[2 * q] = c * step[2 * q] - sn * step[2 * q + 1];
+                cs[2 * q + 1] = sn * step[2 * q] + c * step[2 * q + 1];
+              }
             }
-            uint8_t* dst = tile + row * 128 + ((j ^ (row & 7)) << 4);
-            *reinterpret_cast<uint4*>(dst) = make_uint4(ol[0], ol[1], ol[2], ol[3]);
-            *reinterpret_cast<uint4*>(dst + HALF_TILE_BYTES) = make_uint4(oh[0], oh[1], oh[2], oh[3]);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&kraw_empty[slot]);     // both warps have read the slot: it may be refilled
           }
+          if (!ok) break;
           fence_proxy_async_smem();            // the MMA reads the tile through the async proxy
           __syncwarp();
           if (lane == 0) mbar_arrive(&k_full[st]);
@@ -642,25 +699,25 @@ int make_paged_attn_maps(AttnMaps* out, const __nv_bfloat16* qpool_layer, const 
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
                           int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table, int mode,
-                          const __nv_bfloat16* kpool_layer, const float2* rope, int rope_rows) {
+                          const float2* rope, int rope_rows) {
   if (n_ctas <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   if (group < 2 || group % 2 != 0 || mode < 0 || mode > 2) return -1;
   if (mode != 0 && page_table == nullptr) return -1;
-  if (mode == 2 && (kpool_layer == nullptr || rope == nullptr || rope_rows <= 0)) return -1;
+  if (mode == 2 && (rope == nullptr || rope_rows <= 8)) return -1;
   static bool smem_set[3][MAX_DEVICES] = {};   // once per device: the call costs host time on every launch otherwise
   const int dev = current_device_slot();
   if (!smem_set[mode][dev]) {
     const cudaError_t e =
         mode == 0 ? cudaFuncSetAttribute(umma_attention_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
         : mode == 1 ? cudaFuncSetAttribute(umma_attention_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES)
-                    : cudaFuncSetAttribute(umma_attention_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES);
+                    : cudaFuncSetAttribute(umma_attention_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, ATT_SMEM_BYTES_ROT);
     if (e != cudaSuccess) return -1;
     smem_set[mode][dev] = true;
   }
   AttnArgs a{};
   a.items = items; a.cta_first = cta_first; a.row_pos = row_pos; a.out = out; a.page_table = page_table;
-  a.kpool = kpool_layer; a.rope = rope; a.rope_rows = rope_rows;
+  a.rope = rope; a.rope_rows = rope_rows;
   a.partial_o = partial_o; a.partial_ml = partial_ml;
   a.n_q_heads = n_q_heads; a.n_kv_heads = n_kv_heads;
   a.scale_log2 = 1.4426950408889634f * 0.08838834764831845f;
@@ -669,7 +726,7 @@ int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int
   if (mode == 1)
     rc = launch_pdl(umma_attention_kernel<1>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
   else if (mode == 2)
-    rc = launch_pdl(umma_attention_kernel<2>, dim3(n_ctas), dim3(ATT_THREADS_ROT), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
+    rc = launch_pdl(umma_attention_kernel<2>, dim3(n_ctas), dim3(ATT_THREADS_ROT), ATT_SMEM_BYTES_ROT, s, maps.q, maps.k, maps.v, a);
   else
     rc = launch_pdl(umma_attention_kernel<0>, dim3(n_ctas), dim3(ATT_THREADS), ATT_SMEM_BYTES, s, maps.q, maps.k, maps.v, a);
   return rc == cudaSuccess ? 0 : -1;

@@ -174,14 +174,13 @@ int make_attn_maps(AttnMaps* out, const __half* q, int64_t m_cap, int q_dim, con
 // CTA c (of n_ctas) runs items [cta_first[c], cta_first[c + 1]).
 // mode 0: Q from the query buffer, K/V from the assembled context (maps over those buffers).
 // mode 1: Q, K, V from the pages (maps from make_paged_attn_maps; paper-faithful mode).
-// mode 2: Q from the query buffer (maps.q), V from the pages (maps.v), K loaded from kpool_layer through the page
-//         table and rotated on load with the (cos, sin) table `rope` of rope_rows positions; maps.k is unused.
+// mode 2: Q from the query buffer (maps.q), K and V from the pages (maps.k, maps.v: one 16-row page per copy); K is
+//         staged unrotated and rotated on its way to the MMA with the (cos, sin) table `rope` of rope_rows positions.
 // In modes 1 and 2 an item's ctx0 is the index of its prompt's first entry in page_table.
 int launch_umma_attention(const AttnMaps& maps, const AttnItem* items, const int32_t* cta_first, int n_ctas,
                           const int32_t* row_pos, __half* out, float* partial_o, float* partial_ml, int n_q_heads,
                           int n_kv_heads, int* err_word, cudaStream_t s, const int32_t* page_table = nullptr,
-                          int mode = 0, const __nv_bfloat16* kpool_layer = nullptr, const float2* rope = nullptr,
-                          int rope_rows = 0);
+                          int mode = 0, const float2* rope = nullptr, int rope_rows = 0);
 // Maps for the paged form of the attention (paper-faithful mode): Q, K and V are read straight from the bf16 pages
 // of one layer, 16 rows (one page) per bulk copy; an item's ctx0 then is the index of its prompt's first entry in
 // page_table (one page id per 16 context slots, padded to whole 128-slot blocks).

@@ -42,7 +42,8 @@ struct Plan {   // integer description of the last successful call (host)
 
 constexpr int MAX_EVENTS = 1024;
 constexpr int64_t GATHER_OVERLAP_MIN_BYTES = 512ll << 20;   // below this the per-layer waits cost more than they hide
-constexpr int64_t GATHER_FREE_MIN_RATIO = 8;                // cached tokens per new row from which the fetch is skipped
+constexpr int64_t GATHER_FREE_MIN_RATIO = 8;                // cached tokens per new row from which the fetch is skipped...
+constexpr int64_t GATHER_FREE_MAX_NEW_ROWS = 256;           // ...if no prompt has more new rows than two attention tiles
 
 // Key of a path of chunk ids (prefix mode): fold the ids with a 64-bit mixer (the SplitMix64 output function).
 constexpr uint64_t PATH_KEY_SEED = 0x70657263616368ull;
@@ -384,7 +385,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
       // K and V straight from the pages (K rotated on load): no assembled context
       ok = ok && launch_umma_attention(W.gf_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
                                        h->partial_o, h->partial_ml, D.n_q_heads, D.n_kv_heads, h->d_err, s,
-                                       gather_free_page_table, 2, qe.kpool, h->rope, h->cfg.max_prompt_tokens) == 0;
+                                       gather_free_page_table, 2, h->rope, h->cfg.max_prompt_tokens) == 0;
       launch_attention_merge(d_merges, n_merges, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads, s);
     } else {
       ok = ok && launch_umma_attention(W.attn_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
@@ -955,13 +956,14 @@ int percache_create(const percache_config_t* cfg, const percache_layer_weights_t
     cuda_ok = cuda_ok && make_attn_maps(&W.attn_maps, h->qbuf, h->m_cap, D.q_dim, h->kctx + l * ctx_layer,
                                         h->vctx + l * ctx_layer, h->ctx_cap, D.kv_dim) == 0;
     {
-      // gather-free form of the default mode: Q as above, V one page (16 rows) of a 64-column half per copy
+      // gather-free form of the default mode: Q as above, K and V one page (16 rows) of a 64-column half per copy
       const size_t pl = static_cast<size_t>(cfg->pool_pages) * PAGE_TOKENS;
       W.gf_maps = W.attn_maps;
       const uint32_t box[2] = {64u, static_cast<uint32_t>(PAGE_TOKENS)};
       const uint64_t vd[2] = {static_cast<uint64_t>(D.kv_dim), static_cast<uint64_t>(pl)};
       const uint64_t vs[1] = {static_cast<uint64_t>(D.kv_dim) * 2};
-      cuda_ok = cuda_ok && encode_f16_map(&W.gf_maps.v, h->vpool + l * pl * D.kv_dim, 2, vd, vs, box) == 0;
+      cuda_ok = cuda_ok && encode_f16_map(&W.gf_maps.v, h->vpool + l * pl * D.kv_dim, 2, vd, vs, box) == 0 &&
+                encode_f16_map(&W.gf_maps.k, h->kpool + l * pl * D.kv_dim, 2, vd, vs, box) == 0;
     }
     if (h->paper_mode) {
       const size_t pl = static_cast<size_t>(cfg->pool_pages) * PAGE_TOKENS;
@@ -1218,7 +1220,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   // for the gather-free form: whether every stretch of slots starts on a page boundary, how many pages the rows that
   // are not chunk content to be stored would need for the duration of the call, and the size of the page tables
   bool page_aligned = true;
-  int64_t scratch_pages = 0, pt_entries = 0;
+  int64_t scratch_pages = 0, pt_entries = 0, max_new_per_prompt = 0;
   for (int b = 0; b < n_prompts; ++b) {
     const percache_prompt_t& P = prompts[b];
     if (P.n_query < 0 || (P.n_chunks > 0 && !P.chunk_len) || (P.n_query > 0 && !P.query_hidden))
@@ -1274,6 +1276,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     T += P.n_query;
     n_new += P.n_query;
     pt_entries += (T + 127) / 128 * (128 / PAGE_TOKENS);
+    max_new_per_prompt = std::max(max_new_per_prompt, n_new);
     if (T <= 0) return PERCACHE_E_INVAL;
     if (T > h->cfg.max_prompt_tokens) return PERCACHE_E_CAPACITY;
     if (results[b].out_capacity_rows < n_new || (n_new > 0 && !results[b].out_hidden)) return PERCACHE_E_CAPACITY;
@@ -1287,15 +1290,18 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   // Gather-free form (paper Section 3.2.2 loads and concatenates the matched tensors; here the attention reads them
   // where they are): K and V of every slot stay in 16-token pages, the attention walks the prompt's page table and
   // rotates K on load, and the fetch -- a read, a write and a re-read of every cached K and V byte -- disappears.
-  // Taken when the cached part dominates (the fetch would move more bytes than the attention reads), or on request;
-  // possible when every stretch of slots is page-aligned, nothing is to be decoded afterwards (that needs the
-  // contiguous context) and the tcgen05 attention runs.  The rows of the call that are not chunk content to be
-  // stored then need pages of their own while the call lasts.
+  // Taken when the cached part dominates and every prompt has at most two tiles of new rows, or on request: every
+  // tile of rows rotates the K blocks it reads, so the form pays off when a context block is read once or twice
+  // (the fetch would move more bytes than the attention reads), not when many tiles share it.  Possible when every
+  // stretch of slots is page-aligned, nothing is to be decoded afterwards (that needs the contiguous context) and the
+  // tcgen05 attention runs.  The rows of the call that are not chunk content to be stored then need pages of their
+  // own while the call lasts.
   const bool gather_free =
       page_aligned && hit_tokens > 0 && new_total > 0 && h->decode_reserve == 0 &&
       !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION | PERCACHE_FLAG_ALWAYS_GATHER)) &&
       static_cast<size_t>(pt_entries) <= 4 * static_cast<size_t>(h->ctx_cap) &&
-      ((h->flags & PERCACHE_FLAG_GATHER_FREE) || hit_tokens >= GATHER_FREE_MIN_RATIO * new_total);
+      ((h->flags & PERCACHE_FLAG_GATHER_FREE) ||
+       (hit_tokens >= GATHER_FREE_MIN_RATIO * new_total && max_new_per_prompt <= GATHER_FREE_MAX_NEW_ROWS));
   if (gather_free) pages_needed += scratch_pages;
   // every argument check has passed: choose what would have to be evicted so that the new pages fit (never a chunk
   // this batch hits).  The store itself changes only when the device work is about to start (PageTxn::apply).

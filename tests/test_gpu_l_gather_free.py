@@ -86,8 +86,8 @@ def test_batch_of_prompts_with_shared_chunks():
 
 
 def test_selection_rule():
-    """Without either flag the form follows the batch: at least 8 cached tokens per new row, page-aligned chunks, no
-    decode reserve."""
+    """Without either flag the form follows the batch: at least 8 cached tokens per new row, no prompt with more
+    than 256 new rows, page-aligned chunks, no decode reserve."""
     def form_of(chunk_lens, n_query, hit_idx, reserve=0, flags=0):
         w = wl.small_workload(seed=106, n_layers=1, chunk_lens=chunk_lens, n_query=n_query, hit_idx=hit_idx)
         weights = wl.make_weights(w.shape, w.seed)
@@ -106,6 +106,7 @@ def test_selection_rule():
     assert form_of([120, 136], 16, [0, 1]) == 0                      # not page-aligned
     assert form_of([128, 128], 16, [0, 1], reserve=4) == 0           # a decode will follow: it needs the context
     assert form_of([128, 128], 16, []) == 0                          # nothing cached
+    assert form_of([1024, 1024, 1024], 300, [0, 1, 2]) == 0          # 3072 : 300, but three tiles of new rows
 
 
 def test_prefix_matching_with_tail_drop_gather_free():
