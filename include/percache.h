@@ -180,10 +180,14 @@ typedef struct {
  * pages: the attention walks the prompt's page table, rotates K as it loads it and reads V where it is, so the fetch
  * and its traffic disappear; there P and V enter the second attention product as bf16 (the store's format) instead
  * of fp16.  It is taken when the batch has at least 8 cached tokens per new row and no prompt more than 256 new rows
- * (or PERCACHE_FLAG_GATHER_FREE is set), every chunk length and reuse_tail_drop is a multiple of 16, no decode reserve is set and
- * PERCACHE_FLAG_ALWAYS_GATHER is not; rows that are not stored (query tokens) then occupy pages of the store for the
- * duration of the call (they count against the store limit).  After a gather-free call there is no assembled
- * context: percache_decode and percache_debug_read_ctx return PERCACHE_E_INVAL. */
+ * (or PERCACHE_FLAG_GATHER_FREE is set), every chunk length and reuse_tail_drop is a multiple of 16 and
+ * PERCACHE_FLAG_ALWAYS_GATHER is not set; rows that are not stored (query tokens) then occupy pages of the store for
+ * the duration of the call (they count against the store limit).  After a gather-free call there is no assembled
+ * context and percache_debug_read_ctx returns PERCACHE_E_INVAL.  If a decode reserve is set, those pages stay
+ * occupied after the call and the first percache_decode step runs the skipped fetch over all slots, which builds the
+ * context and gives the pages back; any later percache_prefill call, successful or not, gives them back too and ends
+ * that batch's decode steps.  Without a decode reserve percache_decode after a gather-free call returns
+ * PERCACHE_E_INVAL. */
 PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
 
@@ -317,8 +321,11 @@ PERCACHE_API int percache_debug_attn_plan(const int32_t* n_blocks, int32_t n_til
 PERCACHE_API int percache_debug_capture_layers(percache_t* h, float* host_buf, int64_t capacity_floats);
 
 /* Assembled context of the last call: rotated K and V of one prompt and layer as fp16
- * [n_total + tokens decoded since][n_kv_heads][head_dim], copied to host buffers. */
-PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host);
+ * [n_total + tokens decoded since][n_kv_heads][head_dim], copied to host buffers that hold capacity_tokens tokens
+ * each (fewer than needed -> PERCACHE_E_CAPACITY, nothing is written).  PERCACHE_E_INVAL when the last call left no
+ * assembled context (gather-free form, paper-faithful mode). */
+PERCACHE_API int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host,
+                                         int64_t capacity_tokens);
 
 /* Failure-path check that is safe to run: one tiny kernel waits, through the very wait function every tcgen05
  * kernel of this library uses, on a shared-memory barrier nobody arrives at.  The first waiter's limit is limit_us

@@ -38,6 +38,9 @@ struct Plan {   // integer description of the last successful call (host)
   std::vector<int32_t> ctx0;      // device context slot of every prompt's slot 0 (prompts are decode_reserve apart)
   std::vector<int32_t> dec_len;   // tokens appended to every prompt by percache_decode since the prefill
   bool ctx_assembled = true;      // false after a gather-free call: there is no contiguous context to read or extend
+  // gather-free call with a decode reserve: the prompts' page tables (8-entry padded) and where each starts, kept so
+  // that the first decode step can assemble the context after all
+  std::vector<int32_t> page_table, pt0;
 };
 
 constexpr int MAX_EVENTS = 1024;
@@ -94,6 +97,7 @@ struct percache {
   uint64_t next_serial = 0;
 
   Plan plan;
+  std::vector<int32_t> retained_scratch;   // pages of rows that are not stored, kept for that late assembly
   float* capture_host = nullptr;   // debugging aid: layer inputs of the next calls are copied here (see header)
   int64_t capture_capacity = 0;    // floats
   int32_t decode_reserve = 0;     // context slots kept free behind every prompt for percache_decode
@@ -1186,6 +1190,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   if (!h || !prompts || !results || n_prompts <= 0) return PERCACHE_E_INVAL;
   if (n_prompts > h->cfg.max_batch_prompts) return PERCACHE_E_CAPACITY;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
+  if (!h->retained_scratch.empty()) {      // a new batch begins: the previous one can no longer be decoded on
+    release_pages(h, h->retained_scratch);
+    h->retained_scratch.clear();
+    if (!h->plan.ctx_assembled) h->plan = Plan();
+  }
   if (h->paper_mode) return prefill_paper(h, prompts, n_prompts, results);
   const auto t_host0 = std::chrono::steady_clock::now();
   const ModelDims& D = h->dims;
@@ -1293,11 +1302,11 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   // Taken when the cached part dominates and every prompt has at most two tiles of new rows, or on request: every
   // tile of rows rotates the K blocks it reads, so the form pays off when a context block is read once or twice
   // (the fetch would move more bytes than the attention reads), not when many tiles share it.  Possible when every
-  // stretch of slots is page-aligned, nothing is to be decoded afterwards (that needs the contiguous context) and the
-  // tcgen05 attention runs.  The rows of the call that are not chunk content to be stored then need pages of their
-  // own while the call lasts.
+  // stretch of slots is page-aligned and the tcgen05 attention runs.  The rows of the call that are not chunk
+  // content to be stored then need pages of their own while the call lasts -- and beyond it when a decode reserve is
+  // set: percache_decode needs the contiguous context, which its first step then assembles from the pages.
   const bool gather_free =
-      page_aligned && hit_tokens > 0 && new_total > 0 && h->decode_reserve == 0 &&
+      page_aligned && hit_tokens > 0 && new_total > 0 &&
       !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION | PERCACHE_FLAG_ALWAYS_GATHER)) &&
       static_cast<size_t>(pt_entries) <= 4 * static_cast<size_t>(h->ctx_cap) &&
       ((h->flags & PERCACHE_FLAG_GATHER_FREE) ||
@@ -1536,7 +1545,17 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   // ---------------------------------------------------------------- commit
   for (auto& pe : pending) h->table.emplace(pe.first, std::move(pe.second));
   for (const auto& hu : hit_uses) h->table[hu.first].retrievals += hu.second;
-  release_pages(h, scratch);
+  if (gather_free && h->decode_reserve > 0) {       // decode steps may follow: keep what their late assembly needs
+    h->retained_scratch = scratch;
+    plan.page_table.assign(page_table, page_table + pt_next);
+    int32_t at = 0;
+    for (int b = 0; b < n_prompts; ++b) {
+      plan.pt0.push_back(at);
+      at += (plan.cu_ctx[b + 1] - plan.cu_ctx[b] + 127) / 128 * (128 / PAGE_TOKENS);
+    }
+  } else {
+    release_pages(h, scratch);
+  }
   plan.ctx_assembled = !gather_free;
   st.evictions = evicted;
   for (int b = 0; b < n_prompts; ++b) {
@@ -1581,7 +1600,8 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   if (!h || !hidden || !out_hidden || n_prompts <= 0 || h->paper_mode) return PERCACHE_E_INVAL;
   Plan& plan = h->plan;
   if (static_cast<size_t>(n_prompts) + 1 != plan.cu_ctx.size()) return PERCACHE_E_INVAL;   // not the last call's batch
-  if (!plan.ctx_assembled) return PERCACHE_E_INVAL;      // the last prefill ran gather-free: no context to append to
+  // the last prefill ran gather-free: without a decode reserve nothing was kept to build the context from
+  if (!plan.ctx_assembled && plan.page_table.empty()) return PERCACHE_E_INVAL;
   if (n_prompts > h->m_cap) return PERCACHE_E_CAPACITY;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   const auto t_host0 = std::chrono::steady_clock::now();
@@ -1673,6 +1693,30 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
     if (!dev_alloc(h, &h->cref, static_cast<size_t>(h->m_cap) * wide)) return PERCACHE_E_NOMEM;
   }
   bool ok = true;
+  bool assembled_now = false;
+  if (!plan.ctx_assembled) {
+    // First decode step after a gather-free prefill: every slot of every prompt still sits in a page (cached chunks
+    // in theirs, the rows that prefill computed in the pages lent to them), so the fetch that prefill skipped runs
+    // now, over all slots, and builds the contiguous context the decode kernels read and append to.
+    int n_items = 0;
+    for (int b = 0; b < n_prompts; ++b) {
+      const int32_t T = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+      for (int32_t o = 0; o < T; o += PAGE_TOKENS) {
+        GatherItem& g = items[n_items++];
+        g.dst_slot = plan.ctx0[b] + o;
+        g.src_page = plan.page_table[static_cast<size_t>(plan.pt0[b] + o / PAGE_TOKENS)];
+        g.n_tok = std::min<int32_t>(PAGE_TOKENS, T - o);
+        g.pos = o;
+      }
+    }
+    ok = ok && cudaMemcpyAsync(reinterpret_cast<int32_t*>(const_cast<GatherItem*>(dev_index(h).items)), items,
+                               static_cast<size_t>(n_items) * sizeof(GatherItem), cudaMemcpyHostToDevice, s) == cudaSuccess;
+    timer.begin(PERCACHE_PH_GATHER);
+    launch_gather_rerope(dev_index(h).items, n_items, D.n_layers, h->kpool, h->vpool, h->cfg.pool_pages, h->kctx, h->vctx,
+                         h->ctx_cap, D.kv_dim, h->rope, s);
+    timer.end();
+    assembled_now = true;
+  }
   const size_t used_ints = static_cast<size_t>(reinterpret_cast<int32_t*>(merges + n_merges) - h->h_index);
   ok = ok && cudaMemcpyAsync(h->d_index, h->h_index, used_ints * sizeof(int32_t), cudaMemcpyHostToDevice, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(h->d_err, 0, sizeof(int), s) == cudaSuccess;
@@ -1692,6 +1736,14 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   const cudaError_t sync_rc = cudaStreamSynchronize(s);
   if (!ok || sync_rc != cudaSuccess || cudaGetLastError() != cudaSuccess) return PERCACHE_E_CUDA;
   if (*h->h_err != 0) return PERCACHE_E_DEVICE_TIMEOUT;
+  if (assembled_now) {         // the context exists now: the lent pages go back
+    plan.ctx_assembled = true;
+    plan.page_table.clear();
+    plan.pt0.clear();
+    release_pages(h, h->retained_scratch);
+    h->retained_scratch.clear();
+    refresh_page_stats(h);
+  }
   for (int b = 0; b < n_prompts; ++b) plan.dec_len[b] += 1;      // the token's K/V now is part of the context
   st.n_prompts = n_prompts;
   st.chunks_hit = st.chunks_missed = 0;
@@ -1763,15 +1815,17 @@ int64_t percache_debug_read_plan(percache_t* h, int32_t which, int32_t* out, int
   return static_cast<int64_t>(v->size());
 }
 
-int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host) {
+int percache_debug_read_ctx(percache_t* h, int32_t prompt, int32_t layer, void* k_host, void* v_host,
+                            int64_t capacity_tokens) {
   if (!h || !k_host || !v_host || layer < 0 || layer >= h->dims.n_layers || prompt < 0 ||
       prompt + 1 >= static_cast<int32_t>(h->plan.cu_ctx.size()) || !h->plan.ctx_assembled || h->paper_mode)
     return PERCACHE_E_INVAL;
   if (cudaSetDevice(h->cfg.device) != cudaSuccess) return PERCACHE_E_CUDA;
   const size_t ctx_layer = static_cast<size_t>(h->ctx_cap) * h->dims.kv_dim;
   const size_t off = layer * ctx_layer + static_cast<size_t>(h->plan.ctx0[prompt]) * h->dims.kv_dim;
-  const size_t bytes = static_cast<size_t>(h->plan.cu_ctx[prompt + 1] - h->plan.cu_ctx[prompt] + h->plan.dec_len[prompt]) *
-                       h->dims.kv_dim * 2;
+  const int64_t tokens = h->plan.cu_ctx[prompt + 1] - h->plan.cu_ctx[prompt] + h->plan.dec_len[prompt];
+  if (capacity_tokens < tokens) return PERCACHE_E_CAPACITY;
+  const size_t bytes = static_cast<size_t>(tokens) * h->dims.kv_dim * 2;
   if (cudaMemcpy(k_host, h->kctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess ||
       cudaMemcpy(v_host, h->vctx + off, bytes, cudaMemcpyDeviceToHost) != cudaSuccess)
     return PERCACHE_E_CUDA;

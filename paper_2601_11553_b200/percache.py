@@ -105,7 +105,7 @@ def load_library() -> C.CDLL:
     lib.percache_chunk_info.argtypes = [vp, u64, C.POINTER(i32), C.POINTER(i64)]
     lib.percache_debug_read_plan.argtypes = [vp, i32, C.POINTER(i32), i64]
     lib.percache_debug_read_plan.restype = i64
-    lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp]
+    lib.percache_debug_read_ctx.argtypes = [vp, i32, i32, vp, vp, i64]
     lib.percache_debug_attn_plan.argtypes = [vp, i32, i32, i32, i32, vp, i64, vp]
     lib.percache_debug_gemm.argtypes = [i32, i32, i32, i32, vp, vp, vp, i32]
     lib.percache_debug_gemm_noalloc.argtypes = [i32, i32, i32, i32, vp, vp, vp]
@@ -374,7 +374,8 @@ class PerCache:
         """Assembled (rotated K, V) of one prompt and layer: two float16 arrays [n_total, kv_dim]."""
         k = np.empty((n_total, self.kv_dim), dtype=np.float16)
         v = np.empty_like(k)
-        _check(self._lib.percache_debug_read_ctx(self._h, prompt, layer, _ptr(k), _ptr(v)), "percache_debug_read_ctx")
+        _check(self._lib.percache_debug_read_ctx(self._h, prompt, layer, _ptr(k), _ptr(v), n_total),
+               "percache_debug_read_ctx")
         return k, v
 
 

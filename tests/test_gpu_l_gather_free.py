@@ -42,7 +42,7 @@ def _both_forms(w: wl.Workload, match_prefix=False, tail_drop=0, extra_prompts=(
             outs[form] = [g.out_hidden.copy() for g in got]
             missed = [c for c in ids_lens if c not in cached]
             kvs[form] = [h.get_chunk_kv(c) for c in missed]
-            if form == "gather_free":      # no contiguous context exists: reading it, or decoding on it, is refused
+            if form == "gather_free":      # no contiguous context exists (and no decode reserve was set): refused
                 with pytest.raises(pcb.PerCacheError) as e:
                     h.read_ctx(0, 0, want[0].layout.n_total)
                 assert e.value.code == pcb.E_INVAL
@@ -87,7 +87,7 @@ def test_batch_of_prompts_with_shared_chunks():
 
 def test_selection_rule():
     """Without either flag the form follows the batch: at least 8 cached tokens per new row, no prompt with more
-    than 256 new rows, page-aligned chunks, no decode reserve."""
+    than 256 new rows, page-aligned chunks."""
     def form_of(chunk_lens, n_query, hit_idx, reserve=0, flags=0):
         w = wl.small_workload(seed=106, n_layers=1, chunk_lens=chunk_lens, n_query=n_query, hit_idx=hit_idx)
         weights = wl.make_weights(w.shape, w.seed)
@@ -104,7 +104,7 @@ def test_selection_rule():
     assert form_of([128, 128], 40, [0, 1], flags=pcb.FLAG_GATHER_FREE) == 1
     assert form_of([128, 128], 16, [0, 1], flags=pcb.FLAG_ALWAYS_GATHER) == 0
     assert form_of([120, 136], 16, [0, 1]) == 0                      # not page-aligned
-    assert form_of([128, 128], 16, [0, 1], reserve=4) == 0           # a decode will follow: it needs the context
+    assert form_of([128, 128], 16, [0, 1], reserve=4) == 1           # a decode reserve does not change the choice
     assert form_of([128, 128], 16, []) == 0                          # nothing cached
     assert form_of([1024, 1024, 1024], 300, [0, 1, 2]) == 0          # 3072 : 300, but three tiles of new rows
 
@@ -139,3 +139,53 @@ def test_prefix_matching_with_tail_drop_gather_free():
         for ref in (want.out_hidden, full[want.layout.new_slots]):
             c = G.compare_hidden(got.out_hidden, ref)
             assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
+
+
+def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
+    """With a decode reserve the gather-free prefill keeps the pages it lent to the query rows; the first decode step
+    runs the fetch it skipped, over every slot, then decoding goes on as after any prefill."""
+    from oracle import decode as dec
+    seed, reserve, n_steps = 108, 3, 3
+    ws = [wl.small_workload(seed=seed, n_layers=2, chunk_lens=cl, n_query=nq, hit_idx=hi, id_base=100 + 50 * b)
+          for b, (cl, nq, hi) in enumerate([([128, 64], 9, [0, 1]), ([256], 20, [0])])]
+    shape = ws[0].shape
+    weights = wl.make_weights(shape, seed, random_gains=True)
+    model = H.oracle_model(shape, weights)
+    prompts = [w.prompts[0] for w in ws]
+    cached = [c for w in ws for c in w.cached_ids]
+    lens = {c: l for p in prompts for c, l in zip(p.chunk_ids, p.chunk_len)}
+    store = G.oracle_store_alone(model, seed, [(c, lens[c]) for c in cached])
+    want = orc.reuse_prefill(model, store, [H.oracle_prompt(p, list(range(len(p.chunk_ids)))) for p in prompts],
+                             keep_ctx=True, commit=False)
+    states = [dec.begin_decode(r) for r in want]
+    toks = [wl.make_hidden(seed, (9, j), len(prompts), shape.d_model) for j in range(n_steps)]
+    with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=pcb.FLAG_GATHER_FREE) as h:
+        h.set_decode_reserve(reserve)
+        G.push_store(h, store, cached)
+        free_before = h.stats()["pages_free"]
+        got = h.prefill(G.specs_for(prompts, cached))
+        assert h.stats()["gather_free"] == 1
+        assert h.stats()["pages_free"] == free_before - 1 - 2        # the query rows' pages are still lent out
+        for g, r in zip(got, want):
+            c = G.compare_hidden(g.out_hidden, r.out_hidden)
+            assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
+        for j in range(n_steps):
+            out = h.decode(np.ascontiguousarray(toks[j]))
+            ref = np.stack([dec.decode_step(model, states[b], orc.bf16_bits_to_f64(toks[j][b])) for b in range(len(prompts))])
+            c = G.compare_hidden(out, ref)
+            assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, (j, c)
+            assert h.stats()["pages_free"] == free_before            # given back by the first step
+        # the context the first step assembled is the one the gather form builds: gathered V bit for bit (the read
+        # returns the decoded tokens' slots as well)
+        for b, r in enumerate(want):
+            n_total = r.layout.n_total
+            hit = r.layout.slot_is_new == 0
+            for l in range(shape.n_layers):
+                k, v = h.read_ctx(b, l, n_total + n_steps)
+                want_v = r.v_ctx[l].reshape(n_total, -1)
+                assert np.array_equal(v[:n_total][hit].view(np.uint16), want_v[hit].astype(np.float16).view(np.uint16))
+                want_k = r.k_ctx[l].reshape(n_total, -1)
+                assert np.max(np.abs(k[:n_total].astype(np.float64) - want_k)) < 3e-2
+        with pytest.raises(pcb.PerCacheError) as e:                  # the reserve is used up
+            h.decode(np.ascontiguousarray(toks[0]))
+        assert e.value.code == pcb.E_CAPACITY
