@@ -29,17 +29,41 @@ __device__ __forceinline__ void half8_to_f32(const uint4& v, float (&f)[8]) {
   }
 }
 
+__device__ __forceinline__ void bf16x8_to_f32(const uint4& v, float (&f)[8]) {
+  const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    f[2 * i] = __uint_as_float(w[i] << 16);
+    f[2 * i + 1] = __uint_as_float(w[i] & 0xffff0000u);
+  }
+}
+
+// Where a paged decode step finds K and V: the bf16 pages of one layer, the prompts' page tables (one page id per 16
+// slots; an item's ctx0 then is the index of its prompt's first entry) and the (cos, sin) table for rotating K.
+struct DecodePages {
+  const __nv_bfloat16* kpool;
+  const __nv_bfloat16* vpool;
+  const int32_t* page_table;
+  const float2* rope;
+};
+
 // partial_o: [item][group][128] fp32; partial_ml: [item][group][2] (reference maximum in log2 units, sum)
-template <int GROUP>
+// PAGED = false: K (rotated) and V from the assembled fp16 context; a lane holds 16 consecutive dimensions.
+// PAGED = true (after a gather-free prefill): K and V straight from the bf16 pages through the page table, K rotated
+// to the slot's position as it is loaded; a lane then holds the 16-byte vector l8 of the head's low half and the one
+// of its high half (dimensions 8 l8 .. 8 l8 + 7 and 64 + 8 l8 ..), i.e. eight whole rotation pairs.
+template <int GROUP, bool PAGED>
 __global__ void __launch_bounds__(DEC_THREADS)
 decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* q, const __half* kctx,
-                        const __half* vctx, float* __restrict__ partial_o,
+                        const __half* vctx, DecodePages pages, float* __restrict__ partial_o,
                         float* __restrict__ partial_ml, int n_q_heads, int n_kv_heads, float scale_log2) {
   __shared__ float sm_o[DEC_WARPS][GROUP][HEAD_DIM];
   __shared__ float sm_ml[DEC_WARPS][GROUP][2];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const int l8 = lane & 7;                  // which 16 of the 128 dimensions this lane holds
   const int grp = lane >> 3;                // which of the warp's four slots per step
+  // first dimension of the lane's two 8-element vectors
+  const int d_lo = PAGED ? l8 * 8 : l8 * 16, d_hi = PAGED ? ROPE_HALF + l8 * 8 : l8 * 16 + 8;
   pdl_launch_dependents();
   const DecodeAttnItem it = items[blockIdx.x];     // host-written before the step's first kernel: read ahead of the wait
   pdl_wait();
@@ -49,12 +73,12 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
   float qv[GROUP][16];
 #pragma unroll
   for (int h = 0; h < GROUP; ++h) {
-    const __half* qp = q + (static_cast<size_t>(it.row) * n_q_heads + g * GROUP + h) * HEAD_DIM + l8 * 16;
+    const __half* qp = q + (static_cast<size_t>(it.row) * n_q_heads + g * GROUP + h) * HEAD_DIM;
     float f[8];
-    half8_to_f32(ld_dep_v4(qp), f);
+    half8_to_f32(ld_dep_v4(qp + d_lo), f);
 #pragma unroll
     for (int e = 0; e < 8; ++e) qv[h][e] = f[e] * scale_log2;
-    half8_to_f32(ld_dep_v4(qp + 8), f);
+    half8_to_f32(ld_dep_v4(qp + d_hi), f);
 #pragma unroll
     for (int e = 0; e < 8; ++e) qv[h][8 + e] = f[e] * scale_log2;
   }
@@ -67,25 +91,52 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
     for (int e = 0; e < 16; ++e) o[h][e] = 0.f;
   }
   const size_t base = static_cast<size_t>(it.ctx0) * kv_dim + g * HEAD_DIM + l8 * 16;
-  // Loads run three steps ahead of the arithmetic (three register buffers), so that every warp keeps 6 KB in flight.
+  // Loads run three steps ahead of the arithmetic (three register buffers), so that every warp keeps 6 KB in flight
+  // (paged: K, V and the slot's eight (cos, sin) pairs).
   constexpr int STEP = DEC_WARPS * 4;
-  auto fetch = [&](int s0, uint4 (&r)[4]) {
+  constexpr int NR = PAGED ? 8 : 4;
+  auto fetch = [&](int s0, uint4 (&r)[NR]) {
     const int slot = s0 + grp;
     if (slot < it.slot_end) {
-      const size_t off = base + static_cast<size_t>(slot) * kv_dim;
-      r[0] = ld_dep_v4(kctx + off);          // the newest slot was written by the kernel before this one
-      r[1] = ld_dep_v4(kctx + off + 8);
-      r[2] = ld_dep_v4(vctx + off);
-      r[3] = ld_dep_v4(vctx + off + 8);
+      if constexpr (PAGED) {
+        const int page = __ldg(pages.page_table + it.ctx0 + (slot >> 4));
+        const size_t off = (static_cast<size_t>(page) * PAGE_TOKENS + (slot & 15)) * kv_dim + g * HEAD_DIM;
+        r[0] = ld_dep_v4(pages.kpool + off + d_lo);     // the newest slot was written by the kernel before this one
+        r[1] = ld_dep_v4(pages.kpool + off + d_hi);
+        r[2] = ld_dep_v4(pages.vpool + off + d_lo);
+        r[3] = ld_dep_v4(pages.vpool + off + d_hi);
+        const uint4* cs = reinterpret_cast<const uint4*>(pages.rope + static_cast<size_t>(slot) * ROPE_HALF + l8 * 8);
+        r[4] = __ldg(cs); r[5] = __ldg(cs + 1); r[6] = __ldg(cs + 2); r[7] = __ldg(cs + 3);
+      } else {
+        const size_t off = base + static_cast<size_t>(slot) * kv_dim;
+        r[0] = ld_dep_v4(kctx + off);          // the newest slot was written by the kernel before this one
+        r[1] = ld_dep_v4(kctx + off + 8);
+        r[2] = ld_dep_v4(vctx + off);
+        r[3] = ld_dep_v4(vctx + off + 8);
+      }
     }
   };
-  auto consume = [&](int s0, const uint4 (&r)[4]) {
+  auto consume = [&](int s0, const uint4 (&r)[NR]) {
     const bool live = s0 + grp < it.slot_end;
     float kf[16], vf[16];
-    half8_to_f32(r[0], *reinterpret_cast<float(*)[8]>(&kf[0]));
-    half8_to_f32(r[1], *reinterpret_cast<float(*)[8]>(&kf[8]));
-    half8_to_f32(r[2], *reinterpret_cast<float(*)[8]>(&vf[0]));
-    half8_to_f32(r[3], *reinterpret_cast<float(*)[8]>(&vf[8]));
+    if constexpr (PAGED) {
+      float lo[8], hi[8];
+      bf16x8_to_f32(r[0], lo);
+      bf16x8_to_f32(r[1], hi);
+      bf16x8_to_f32(r[2], *reinterpret_cast<float(*)[8]>(&vf[0]));
+      bf16x8_to_f32(r[3], *reinterpret_cast<float(*)[8]>(&vf[8]));
+      const float* cs = reinterpret_cast<const float*>(&r[4]);      // (cos, sin) of the lane's eight pairs
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        kf[e] = lo[e] * cs[2 * e] - hi[e] * cs[2 * e + 1];
+        kf[8 + e] = hi[e] * cs[2 * e] + lo[e] * cs[2 * e + 1];
+      }
+    } else {
+      half8_to_f32(r[0], *reinterpret_cast<float(*)[8]>(&kf[0]));
+      half8_to_f32(r[1], *reinterpret_cast<float(*)[8]>(&kf[8]));
+      half8_to_f32(r[2], *reinterpret_cast<float(*)[8]>(&vf[0]));
+      half8_to_f32(r[3], *reinterpret_cast<float(*)[8]>(&vf[8]));
+    }
 #pragma unroll
     for (int h = 0; h < GROUP; ++h) {
       float sc = 0.f;
@@ -106,28 +157,34 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
       }
     }
   };
-  uint4 ra[4] = {}, rb[4] = {}, rc[4] = {};
+  uint4 ra[NR] = {}, rb[NR] = {}, rc[NR] = {};
   int s0 = it.slot_begin + warp * 4;
   fetch(s0, ra);
   fetch(s0 + STEP, rb);
   fetch(s0 + 2 * STEP, rc);
   while (s0 < it.slot_end) {
     {
-      const uint4 c[4] = {ra[0], ra[1], ra[2], ra[3]};
+      uint4 c[NR];
+#pragma unroll
+      for (int x = 0; x < NR; ++x) c[x] = ra[x];
       fetch(s0 + 3 * STEP, ra);
       consume(s0, c);
     }
     s0 += STEP;
     if (s0 >= it.slot_end) break;
     {
-      const uint4 c[4] = {rb[0], rb[1], rb[2], rb[3]};
+      uint4 c[NR];
+#pragma unroll
+      for (int x = 0; x < NR; ++x) c[x] = rb[x];
       fetch(s0 + 3 * STEP, rb);
       consume(s0, c);
     }
     s0 += STEP;
     if (s0 >= it.slot_end) break;
     {
-      const uint4 c[4] = {rc[0], rc[1], rc[2], rc[3]};
+      uint4 c[NR];
+#pragma unroll
+      for (int x = 0; x < NR; ++x) c[x] = rc[x];
       fetch(s0 + 3 * STEP, rc);
       consume(s0, c);
     }
@@ -153,7 +210,7 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
     }
     if (grp == 0) {
 #pragma unroll
-      for (int e = 0; e < 16; ++e) sm_o[warp][h][l8 * 16 + e] = o[h][e];
+      for (int e = 0; e < 16; ++e) sm_o[warp][h][(e < 8 ? d_lo + e : d_hi + e - 8)] = o[h][e];
       if (l8 == 0) { sm_ml[warp][h][0] = m[h]; sm_ml[warp][h][1] = l[h]; }
     }
   }
@@ -223,20 +280,29 @@ decode_merge_kernel(const DecodeAttnMerge* __restrict__ merges, const float* par
 
 int launch_decode_attention(const DecodeAttnItem* items, int n_items, const DecodeAttnMerge* merges, int n_merges,
                             const __half* q, const __half* kctx_layer, const __half* vctx_layer, float* partial_o,
-                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s) {
+                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s,
+                            const __nv_bfloat16* kpool_layer, const __nv_bfloat16* vpool_layer,
+                            const int32_t* page_table, const float2* rope) {
   if (n_items <= 0) return 0;
   const int group = n_q_heads / n_kv_heads;
   const float scale_log2 = 1.4426950408889634f * 0.08838834764831845f;      // log2(e) / sqrt(128)
+  const bool paged = page_table != nullptr;
+  if (paged && (!kpool_layer || !vpool_layer || !rope)) return -1;
+  const DecodePages pages{kpool_layer, vpool_layer, page_table, rope};
   cudaError_t rc;
   if (group == 2) {
-    rc = launch_pdl(decode_attention_kernel<2>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer, vctx_layer,
-                    partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
+    rc = paged ? launch_pdl(decode_attention_kernel<2, true>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer,
+                            vctx_layer, pages, partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2)
+               : launch_pdl(decode_attention_kernel<2, false>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer,
+                            vctx_layer, pages, partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
     if (rc == cudaSuccess)
       rc = launch_pdl(decode_merge_kernel<2>, dim3(n_merges, 2), dim3(HEAD_DIM), 0, s, merges, partial_o, partial_ml, out,
                       n_q_heads);
   } else if (group == 4) {
-    rc = launch_pdl(decode_attention_kernel<4>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer, vctx_layer,
-                    partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
+    rc = paged ? launch_pdl(decode_attention_kernel<4, true>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer,
+                            vctx_layer, pages, partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2)
+               : launch_pdl(decode_attention_kernel<4, false>, dim3(n_items), dim3(DEC_THREADS), 0, s, items, q, kctx_layer,
+                            vctx_layer, pages, partial_o, partial_ml, n_q_heads, n_kv_heads, scale_log2);
     if (rc == cudaSuccess)
       rc = launch_pdl(decode_merge_kernel<4>, dim3(n_merges, 4), dim3(HEAD_DIM), 0, s, merges, partial_o, partial_ml, out,
                       n_q_heads);

@@ -66,6 +66,7 @@ __device__ __forceinline__ void qkv_store1(const QkvEpilogue& e, int row, const 
     p[0] = bl;
     p[ROPE_HALF] = bh;
   }
+  if (e.skip_ctx) return;                 // a paged decode step reads the pages: nothing goes to the context
   const float l = __bfloat162float(bl), h = __bfloat162float(bh);
   __half* dst = (is_k ? e.kctx : e.vctx) + static_cast<size_t>(rw.slot) * kv_dim + kvh * HEAD_DIM + c;
   dst[0] = to_half_sat(is_k ? l * cs.x - h * cs.y : l);

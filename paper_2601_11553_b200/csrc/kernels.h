@@ -70,9 +70,14 @@ struct DecodeAttnMerge {   // the chunks of one (row, KV head) are in slots part
 };
 // partial_o: fp32 [items][query heads per KV head][128]; partial_ml: fp32 [items][query heads per KV head][2].
 // Query heads per KV head must be 2 or 4.
+// page_table != nullptr: the paged form (after a gather-free prefill): K and V are read from the bf16 pages of the
+// layer through the page table, K rotated on load with the (cos, sin) table; an item's ctx0 then indexes its prompt's
+// first page-table entry and kctx_layer / vctx_layer are unused.
 int launch_decode_attention(const DecodeAttnItem* items, int n_items, const DecodeAttnMerge* merges, int n_merges,
                             const __half* q, const __half* kctx_layer, const __half* vctx_layer, float* partial_o,
-                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s);
+                            float* partial_ml, __half* out, int n_q_heads, int n_kv_heads, cudaStream_t s,
+                            const __nv_bfloat16* kpool_layer = nullptr, const __nv_bfloat16* vpool_layer = nullptr,
+                            const int32_t* page_table = nullptr, const float2* rope = nullptr);
 
 // A tile before scheduling: its rows and the number of 128-slot context blocks its last row can see.
 struct AttnBaseTile { int32_t row0, n_rows, ctx0, n_blocks; };

@@ -330,7 +330,7 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
   // A handful of rows (decode) is a matter of reading the weights once: CUDA-core kernels bound by HBM, with the
   // RMSNorm folded into the QKV and gate/up projections
   const bool small_rows = !use_ref && !(h->flags & PERCACHE_FLAG_NO_SMALL_ROW_KERNELS) && Mi <= SMALL_GEMM_MAX_ROWS &&
-                          gather_free_page_table == nullptr &&
+                          (gather_free_page_table == nullptr || n_decode_items > 0) &&
                           d % 256 == 0 && D.q_dim % 256 == 0 && D.d_ffn % 256 == 0;
   bool ok = true;
   // debugging aid: the residual stream as it enters layer l goes to capture_host[l] (stream order does the rest)
@@ -384,7 +384,9 @@ bool run_layers(percache* h, int Mi, const DevIndex& ix, int n_attn_ctas, int n_
       ok = ok && launch_decode_attention(reinterpret_cast<const DecodeAttnItem*>(d_attn_items), n_decode_items,
                                          reinterpret_cast<const DecodeAttnMerge*>(d_merges), n_merges, h->qbuf, qe.kctx,
                                          qe.vctx, h->partial_o, h->partial_ml, h->attn_out, D.n_q_heads, D.n_kv_heads,
-                                         s) == 0;
+                                         s, gather_free_page_table ? qe.kpool : nullptr,
+                                         gather_free_page_table ? qe.vpool : nullptr, gather_free_page_table,
+                                         h->rope) == 0;
     } else if (gather_free_page_table != nullptr) {
       // K and V straight from the pages (K rotated on load): no assembled context
       ok = ok && launch_umma_attention(W.gf_maps, d_attn_items, d_cta_first, n_attn_ctas, d_row_pos, h->attn_out,
@@ -1311,7 +1313,10 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
       static_cast<size_t>(pt_entries) <= 4 * static_cast<size_t>(h->ctx_cap) &&
       ((h->flags & PERCACHE_FLAG_GATHER_FREE) ||
        (hit_tokens >= GATHER_FREE_MIN_RATIO * new_total && max_new_per_prompt <= GATHER_FREE_MAX_NEW_ROWS));
-  if (gather_free) pages_needed += scratch_pages;
+  // with a decode reserve the decoded tokens get page slots behind every prompt's last one, so that decode steps can
+  // read pages as well (an upper bound: the last page of the prompt may have room left)
+  const int64_t decode_pages_per_prompt = (h->decode_reserve + PAGE_TOKENS - 1) / PAGE_TOKENS + (h->decode_reserve > 0 ? 1 : 0);
+  if (gather_free) pages_needed += scratch_pages + (h->decode_reserve > 0 ? decode_pages_per_prompt * n_prompts : 0);
   // every argument check has passed: choose what would have to be evicted so that the new pages fit (never a chunk
   // this batch hits).  The store itself changes only when the device work is about to start (PageTxn::apply).
   PageTxn txn(h);
@@ -1367,6 +1372,7 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   int n_items = 0, n_attn_ctas = 0, n_merges = 0;
   int32_t* page_table = reinterpret_cast<int32_t*>(items);     // gather-free form: in place of the gather items
   int32_t pt_next = 0;
+  std::vector<std::vector<int32_t>> decode_pages;              // per prompt: pages for tokens decoded later
   plan.slot_chunk.resize(static_cast<size_t>(ctx_total));
   plan.slot_offset.resize(static_cast<size_t>(ctx_total));
   plan.slot_is_new.resize(static_cast<size_t>(ctx_total));
@@ -1443,6 +1449,16 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
     if (gather_free && pt_next > pt0) {     // pad the table to whole 128-slot blocks (those slots are never visible)
       const int32_t last_page = page_table[pt_next - 1];
       while ((pt_next - pt0) % (128 / PAGE_TOKENS) != 0) page_table[pt_next++] = last_page;
+      if (h->decode_reserve > 0) {
+        // page slots for the tokens decode steps will append: slots n_total .. n_total + reserve - 1 (the first of them
+        // may still fit the prompt's last page)
+        const int32_t T = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+        const int32_t have = (T + PAGE_TOKENS - 1) / PAGE_TOKENS, want = (T + h->decode_reserve + PAGE_TOKENS - 1) / PAGE_TOKENS;
+        std::vector<int32_t> more;
+        if (want > have && txn.take(want - have, &more) != PERCACHE_OK) return fail(PERCACHE_E_NOSPACE);
+        scratch.insert(scratch.end(), more.begin(), more.end());
+        decode_pages.push_back(more);
+      }
     }
     for (int32_t r0 = plan.cu_new[b]; r0 < plan.cu_new[b + 1]; r0 += 128) {
       AttnBaseTile a{};
@@ -1547,11 +1563,14 @@ int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_
   for (const auto& hu : hit_uses) h->table[hu.first].retrievals += hu.second;
   if (gather_free && h->decode_reserve > 0) {       // decode steps may follow: keep what their late assembly needs
     h->retained_scratch = scratch;
-    plan.page_table.assign(page_table, page_table + pt_next);
+    // per prompt: the pages of its slots, then the pages for decoded tokens (the padding of the prefill table is dropped)
     int32_t at = 0;
     for (int b = 0; b < n_prompts; ++b) {
-      plan.pt0.push_back(at);
-      at += (plan.cu_ctx[b + 1] - plan.cu_ctx[b] + 127) / 128 * (128 / PAGE_TOKENS);
+      const int32_t T = plan.cu_ctx[b + 1] - plan.cu_ctx[b];
+      plan.pt0.push_back(static_cast<int32_t>(plan.page_table.size()));
+      plan.page_table.insert(plan.page_table.end(), page_table + at, page_table + at + (T + PAGE_TOKENS - 1) / PAGE_TOKENS);
+      plan.page_table.insert(plan.page_table.end(), decode_pages[b].begin(), decode_pages[b].end());
+      at += (T + 127) / 128 * (128 / PAGE_TOKENS);
     }
   } else {
     release_pages(h, scratch);
@@ -1623,6 +1642,8 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
     row_slot[b] = plan.ctx0[b] + T;
     row_pos[b] = T;
     row_pool[b] = -1;                       // decoded tokens are not chunk content: nothing goes to the store
+    if (!plan.ctx_assembled)                // ... but after a gather-free prefill they get a page slot lent to the batch
+      row_pool[b] = plan.page_table[static_cast<size_t>(plan.pt0[b] + T / PAGE_TOKENS)] * PAGE_TOKENS + T % PAGE_TOKENS;
     row_ctx0[b] = plan.ctx0[b];
     base_tiles.push_back(AttnBaseTile{b, 1, plan.ctx0[b], (T + 1 + 127) / 128});
     visible_pairs += T + 1;
@@ -1633,6 +1654,9 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   const int group = D.n_q_heads / D.n_kv_heads;
   const bool stream_attention = !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION |
                                               PERCACHE_FLAG_NO_SMALL_ROW_KERNELS)) && (group == 2 || group == 4);
+  // After a gather-free prefill the streaming kernel reads the pages themselves (K rotated on load): no context is
+  // ever assembled for this batch.  Where that kernel cannot run, the first step assembles the context instead.
+  const bool paged_decode = !plan.ctx_assembled && stream_attention;
   int n_attn_ctas = 0, n_merges = 0, n_decode_items = 0;
   if (stream_attention) {
     int64_t total_slots = 0;
@@ -1659,8 +1683,8 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
         dmerges[n_merges++] = DecodeAttnMerge{b, g, next_slot + g * n_chunks, n_chunks, 0, 0, 0, 0};
       for (int c = 0; c < n_chunks; ++c)
         for (int g = 0; g < D.n_kv_heads; ++g)
-          ditems[n_decode_items++] = DecodeAttnItem{b, plan.ctx0[b], c * chunk, std::min(n_slots, (c + 1) * chunk), g,
-                                                    next_slot + g * n_chunks + c, 0, 0};
+          ditems[n_decode_items++] = DecodeAttnItem{b, paged_decode ? plan.pt0[b] : plan.ctx0[b], c * chunk,
+                                                    std::min(n_slots, (c + 1) * chunk), g, next_slot + g * n_chunks + c, 0, 0};
       next_slot += n_chunks * D.n_kv_heads;
     }
   } else {
@@ -1694,7 +1718,10 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   }
   bool ok = true;
   bool assembled_now = false;
-  if (!plan.ctx_assembled) {
+  if (paged_decode) {       // the prompts' page tables (with the decoded tokens' pages) in place of the gather items
+    if (plan.page_table.size() > 4 * static_cast<size_t>(h->ctx_cap)) return PERCACHE_E_CAPACITY;
+    std::memcpy(items, plan.page_table.data(), plan.page_table.size() * sizeof(int32_t));
+  } else if (!plan.ctx_assembled) {
     // First decode step after a gather-free prefill: every slot of every prompt still sits in a page (cached chunks
     // in theirs, the rows that prefill computed in the pages lent to them), so the fetch that prefill skipped runs
     // now, over all slots, and builds the contiguous context the decode kernels read and append to.
@@ -1726,7 +1753,8 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   cudaEventRecord(h->ev_begin, s);
   launch_bf16_to_f32(h->xin, h->resid, static_cast<int64_t>(n_prompts) * d, s);
   timer.end();
-  ok = ok && run_layers(h, n_prompts, dev_index(h), n_attn_ctas, n_merges, false, use_ref, timer, s, n_decode_items);
+  ok = ok && run_layers(h, n_prompts, dev_index(h), n_attn_ctas, n_merges, false, use_ref, timer, s, n_decode_items,
+                        paged_decode ? reinterpret_cast<const int32_t*>(dev_index(h).items) : nullptr);
   cudaEventRecord(h->ev_end, s);
   timer.begin(PERCACHE_PH_IO);
   ok = ok && cudaMemcpyAsync(out_hidden, h->resid, static_cast<size_t>(n_prompts) * d * sizeof(float),

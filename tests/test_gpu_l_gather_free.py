@@ -141,11 +141,8 @@ def test_prefix_matching_with_tail_drop_gather_free():
             assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
 
 
-def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
-    """With a decode reserve the gather-free prefill keeps the pages it lent to the query rows; the first decode step
-    runs the fetch it skipped, over every slot, then decoding goes on as after any prefill."""
+def _decode_setup(seed, reserve, n_steps):
     from oracle import decode as dec
-    seed, reserve, n_steps = 108, 3, 3
     ws = [wl.small_workload(seed=seed, n_layers=2, chunk_lens=cl, n_query=nq, hit_idx=hi, id_base=100 + 50 * b)
           for b, (cl, nq, hi) in enumerate([([128, 64], 9, [0, 1]), ([256], 20, [0])])]
     shape = ws[0].shape
@@ -159,13 +156,23 @@ def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
                              keep_ctx=True, commit=False)
     states = [dec.begin_decode(r) for r in want]
     toks = [wl.make_hidden(seed, (9, j), len(prompts), shape.d_model) for j in range(n_steps)]
+    return dec, shape, weights, model, prompts, cached, store, want, states, toks
+
+
+@pytest.mark.parametrize("reserve,n_steps", [(3, 3), (40, 20)])
+def test_decode_after_a_gather_free_prefill_reads_the_pages(reserve, n_steps):
+    """With a decode reserve the gather-free prefill keeps the pages it lent to the query rows and adds page slots for
+    the tokens to come; decode steps then read K and V from the pages as well (K rotated on load) and no context is
+    ever assembled for the batch.  The second case decodes across page and 128-slot block boundaries."""
+    dec, shape, weights, model, prompts, cached, store, want, states, toks = _decode_setup(108, reserve, n_steps)
     with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=pcb.FLAG_GATHER_FREE) as h:
         h.set_decode_reserve(reserve)
         G.push_store(h, store, cached)
         free_before = h.stats()["pages_free"]
         got = h.prefill(G.specs_for(prompts, cached))
         assert h.stats()["gather_free"] == 1
-        assert h.stats()["pages_free"] == free_before - 1 - 2        # the query rows' pages are still lent out
+        lent = sum((p.n_total + reserve + 15) // 16 - sum(p.chunk_len) // 16 for p in prompts)
+        assert h.stats()["pages_free"] == free_before - lent          # query rows' pages + slots for decoded tokens
         for g, r in zip(got, want):
             c = G.compare_hidden(g.out_hidden, r.out_hidden)
             assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, c
@@ -174,9 +181,37 @@ def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
             ref = np.stack([dec.decode_step(model, states[b], orc.bf16_bits_to_f64(toks[j][b])) for b in range(len(prompts))])
             c = G.compare_hidden(out, ref)
             assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, (j, c)
-            assert h.stats()["pages_free"] == free_before            # given back by the first step
-        # the context the first step assembled is the one the gather form builds: gathered V bit for bit (the read
-        # returns the decoded tokens' slots as well)
+        with pytest.raises(pcb.PerCacheError) as e:                   # still no contiguous context
+            h.read_ctx(0, 0, want[0].layout.n_total + n_steps)
+        assert e.value.code == pcb.E_INVAL
+        if n_steps == reserve:
+            with pytest.raises(pcb.PerCacheError) as e:               # the reserve is used up
+                h.decode(np.ascontiguousarray(toks[0]))
+            assert e.value.code == pcb.E_CAPACITY
+        # the next prefill gives the lent pages back
+        h.prefill(G.specs_for(prompts[:1], cached))
+        assert h.stats()["pages_free"] == free_before - ((prompts[0].n_total + reserve + 15) // 16 - sum(prompts[0].chunk_len) // 16)
+
+
+def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
+    """Where the streaming decode kernels are switched off, the first decode step runs the fetch the prefill skipped,
+    over every slot, which builds the context the gather form builds; the lent pages then go back."""
+    reserve, n_steps = 3, 3
+    dec, shape, weights, model, prompts, cached, store, want, states, toks = _decode_setup(109, reserve, n_steps)
+    with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=pcb.FLAG_GATHER_FREE) as h:
+        h.set_decode_reserve(reserve)
+        G.push_store(h, store, cached)
+        free_before = h.stats()["pages_free"]
+        got = h.prefill(G.specs_for(prompts, cached))
+        assert h.stats()["gather_free"] == 1 and h.stats()["pages_free"] < free_before
+        h.set_flags(pcb.FLAG_GATHER_FREE | pcb.FLAG_NO_SMALL_ROW_KERNELS)
+        for j in range(n_steps):
+            out = h.decode(np.ascontiguousarray(toks[j]))
+            ref = np.stack([dec.decode_step(model, states[b], orc.bf16_bits_to_f64(toks[j][b])) for b in range(len(prompts))])
+            c = G.compare_hidden(out, ref)
+            assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, (j, c)
+            assert h.stats()["pages_free"] == free_before             # given back by the first step
+        # gathered V bit for bit (the read returns the decoded tokens' slots as well)
         for b, r in enumerate(want):
             n_total = r.layout.n_total
             hit = r.layout.slot_is_new == 0
@@ -186,6 +221,3 @@ def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
                 assert np.array_equal(v[:n_total][hit].view(np.uint16), want_v[hit].astype(np.float16).view(np.uint16))
                 want_k = r.k_ctx[l].reshape(n_total, -1)
                 assert np.max(np.abs(k[:n_total].astype(np.float64) - want_k)) < 3e-2
-        with pytest.raises(pcb.PerCacheError) as e:                  # the reserve is used up
-            h.decode(np.ascontiguousarray(toks[0]))
-        assert e.value.code == pcb.E_CAPACITY
