@@ -711,7 +711,9 @@ def run_decode(args):
     stream = torch.cuda.current_stream(dev)
     h = pcb.PerCache(n_layers=shape.n_layers, d_model=shape.d_model, n_q_heads=shape.n_q_heads,
                      n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim, d_ffn=shape.d_ffn, weights=weights,
-                     pool_pages=sum((l + 15) // 16 for l in ids_lens.values()) + 64,
+                     # + pages lent to the query rows and to the decoded tokens when the prefill runs gather-free
+                     pool_pages=sum((l + 15) // 16 for l in ids_lens.values()) + 64
+                     + sum((p.n_query + reserve + 15) // 16 + 2 for p in w.prompts),
                      max_prompt_tokens=max(p.n_total for p in w.prompts) + reserve, max_batch_prompts=B,
                      max_batch_ctx_tokens=w.total_tokens + B * reserve, max_batch_new_rows=w.total_tokens, device=local,
                      stream=stream.cuda_stream)

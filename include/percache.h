@@ -183,11 +183,13 @@ typedef struct {
  * (or PERCACHE_FLAG_GATHER_FREE is set), every chunk length and reuse_tail_drop is a multiple of 16 and
  * PERCACHE_FLAG_ALWAYS_GATHER is not set; rows that are not stored (query tokens) then occupy pages of the store for
  * the duration of the call (they count against the store limit).  After a gather-free call there is no assembled
- * context and percache_debug_read_ctx returns PERCACHE_E_INVAL.  If a decode reserve is set, those pages stay
- * occupied after the call and the first percache_decode step runs the skipped fetch over all slots, which builds the
- * context and gives the pages back; any later percache_prefill call, successful or not, gives them back too and ends
- * that batch's decode steps.  Without a decode reserve percache_decode after a gather-free call returns
- * PERCACHE_E_INVAL. */
+ * context and percache_debug_read_ctx returns PERCACHE_E_INVAL.  If a decode reserve is set, those pages (and page
+ * slots for the tokens to be decoded) stay occupied after the call and the first percache_decode step runs the
+ * skipped fetch over all slots, which builds the context and gives the pages back; with PERCACHE_FLAG_GATHER_FREE
+ * set at that time the decode steps instead read the pages themselves (K rotated on load; each step's attention is
+ * about 40 % slower, no context is ever built, the pages stay occupied).  Any later percache_prefill call, successful
+ * or not, gives the pages back and ends that batch's decode steps.  Without a decode reserve percache_decode after a
+ * gather-free call returns PERCACHE_E_INVAL. */
 PERCACHE_API int percache_prefill(percache_t* h, const percache_prompt_t* prompts, int32_t n_prompts,
                      percache_result_t* results /*[n_prompts]*/);
 

@@ -91,22 +91,51 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
     for (int e = 0; e < 16; ++e) o[h][e] = 0.f;
   }
   const size_t base = static_cast<size_t>(it.ctx0) * kv_dim + g * HEAD_DIM + l8 * 16;
-  // Loads run three steps ahead of the arithmetic (three register buffers), so that every warp keeps 6 KB in flight
-  // (paged: K, V and the slot's eight (cos, sin) pairs).
+  // Loads run three steps ahead of the arithmetic (three register buffers), so that every warp keeps 6 KB in flight.
   constexpr int STEP = DEC_WARPS * 4;
-  constexpr int NR = PAGED ? 8 : 4;
+  constexpr int NR = 4;
+  // Paged form: (cos, sin) of the lane's eight pairs at the slot it works on.  A lane's slots are STEP = 16 apart, so
+  // the first comes from the table and every next one is a complex multiplication by the table's row 16 on (a chunk
+  // has at most 64 such steps: the error stays near 1e-6 relative).
+  float cs[16], cs_step[16];
+  if constexpr (PAGED) {
+    const float4* c0 = reinterpret_cast<const float4*>(pages.rope + static_cast<size_t>(it.slot_begin + warp * 4 + grp) * ROPE_HALF + l8 * 8);
+    const float4* c1 = reinterpret_cast<const float4*>(pages.rope + static_cast<size_t>(STEP) * ROPE_HALF + l8 * 8);
+#pragma unroll
+    for (int x = 0; x < 4; ++x) {
+      const float4 a = __ldg(c0 + x), b = __ldg(c1 + x);
+      cs[4 * x] = a.x; cs[4 * x + 1] = a.y; cs[4 * x + 2] = a.z; cs[4 * x + 3] = a.w;
+      cs_step[4 * x] = b.x; cs_step[4 * x + 1] = b.y; cs_step[4 * x + 2] = b.z; cs_step[4 * x + 3] = b.w;
+    }
+  }
+  // Paged form: a lane's slots are 16 apart, i.e. one page-table entry per step; the entries are requested three
+  // steps ahead of the loads that need them so that the K/V loads never wait for a table entry.
+  int pq0 = 0, pq1 = 0, pq2 = 0;
+  int pq_slot = it.slot_begin + warp * 4 + grp;             // slot whose page id pq0 holds
+  if constexpr (PAGED) {
+    const int32_t* pt = pages.page_table + it.ctx0;
+    const int last = (it.slot_end - 1) >> 4;
+    pq0 = __ldg(pt + min(pq_slot >> 4, last));
+    pq1 = __ldg(pt + min((pq_slot + STEP) >> 4, last));
+    pq2 = __ldg(pt + min((pq_slot + 2 * STEP) >> 4, last));
+  }
   auto fetch = [&](int s0, uint4 (&r)[NR]) {
     const int slot = s0 + grp;
+    int page = 0;
+    if constexpr (PAGED) {       // fetches come in slot order, one step apart: pop the queue, request one more entry
+      page = pq0;
+      pq0 = pq1;
+      pq1 = pq2;
+      pq_slot += STEP;
+      pq2 = __ldg(pages.page_table + it.ctx0 + min((pq_slot + 2 * STEP) >> 4, (it.slot_end - 1) >> 4));
+    }
     if (slot < it.slot_end) {
       if constexpr (PAGED) {
-        const int page = __ldg(pages.page_table + it.ctx0 + (slot >> 4));
         const size_t off = (static_cast<size_t>(page) * PAGE_TOKENS + (slot & 15)) * kv_dim + g * HEAD_DIM;
         r[0] = ld_dep_v4(pages.kpool + off + d_lo);     // the newest slot was written by the kernel before this one
         r[1] = ld_dep_v4(pages.kpool + off + d_hi);
         r[2] = ld_dep_v4(pages.vpool + off + d_lo);
         r[3] = ld_dep_v4(pages.vpool + off + d_hi);
-        const uint4* cs = reinterpret_cast<const uint4*>(pages.rope + static_cast<size_t>(slot) * ROPE_HALF + l8 * 8);
-        r[4] = __ldg(cs); r[5] = __ldg(cs + 1); r[6] = __ldg(cs + 2); r[7] = __ldg(cs + 3);
       } else {
         const size_t off = base + static_cast<size_t>(slot) * kv_dim;
         r[0] = ld_dep_v4(kctx + off);          // the newest slot was written by the kernel before this one
@@ -125,11 +154,13 @@ decode_attention_kernel(const DecodeAttnItem* __restrict__ items, const __half* 
       bf16x8_to_f32(r[1], hi);
       bf16x8_to_f32(r[2], *reinterpret_cast<float(*)[8]>(&vf[0]));
       bf16x8_to_f32(r[3], *reinterpret_cast<float(*)[8]>(&vf[8]));
-      const float* cs = reinterpret_cast<const float*>(&r[4]);      // (cos, sin) of the lane's eight pairs
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
-        kf[e] = lo[e] * cs[2 * e] - hi[e] * cs[2 * e + 1];
-        kf[8 + e] = hi[e] * cs[2 * e] + lo[e] * cs[2 * e + 1];
+        const float c = cs[2 * e], sn = cs[2 * e + 1];
+        kf[e] = lo[e] * c - hi[e] * sn;
+        kf[8 + e] = hi[e] * c + lo[e] * sn;
+        cs[2 * e] = c * cs_step[2 * e] - sn * cs_step[2 * e + 1];          // on to the lane's next slot
+        cs[2 * e + 1] = sn * cs_step[2 * e] + c * cs_step[2 * e + 1];
       }
     } else {
       half8_to_f32(r[0], *reinterpret_cast<float(*)[8]>(&kf[0]));

@@ -1654,9 +1654,11 @@ int percache_decode(percache_t* h, int32_t n_prompts, const void* hidden, int32_
   const int group = D.n_q_heads / D.n_kv_heads;
   const bool stream_attention = !(h->flags & (PERCACHE_FLAG_REFERENCE_KERNELS | PERCACHE_FLAG_REFERENCE_ATTENTION |
                                               PERCACHE_FLAG_NO_SMALL_ROW_KERNELS)) && (group == 2 || group == 4);
-  // After a gather-free prefill the streaming kernel reads the pages themselves (K rotated on load): no context is
-  // ever assembled for this batch.  Where that kernel cannot run, the first step assembles the context instead.
-  const bool paged_decode = !plan.ctx_assembled && stream_attention;
+  // After a gather-free prefill the first decode step assembles the context (the fetch the prefill skipped, over every
+  // slot) and decoding goes on as usual.  With PERCACHE_FLAG_GATHER_FREE set, the streaming kernel reads the pages
+  // themselves instead (K rotated on load) and no context is ever assembled for this batch: every step's attention is
+  // then about 40 % slower (measured), so this pays only for a handful of decoded tokens.
+  const bool paged_decode = !plan.ctx_assembled && stream_attention && (h->flags & PERCACHE_FLAG_GATHER_FREE);
   int n_attn_ctas = 0, n_merges = 0, n_decode_items = 0;
   if (stream_attention) {
     int64_t total_slots = 0;

@@ -162,8 +162,9 @@ def _decode_setup(seed, reserve, n_steps):
 @pytest.mark.parametrize("reserve,n_steps", [(3, 3), (40, 20)])
 def test_decode_after_a_gather_free_prefill_reads_the_pages(reserve, n_steps):
     """With a decode reserve the gather-free prefill keeps the pages it lent to the query rows and adds page slots for
-    the tokens to come; decode steps then read K and V from the pages as well (K rotated on load) and no context is
-    ever assembled for the batch.  The second case decodes across page and 128-slot block boundaries."""
+    the tokens to come; with PERCACHE_FLAG_GATHER_FREE still set, decode steps read K and V from the pages as well (K
+    rotated on load) and no context is ever assembled for the batch.  The second case decodes across page and
+    128-slot block boundaries."""
     dec, shape, weights, model, prompts, cached, store, want, states, toks = _decode_setup(108, reserve, n_steps)
     with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=pcb.FLAG_GATHER_FREE) as h:
         h.set_decode_reserve(reserve)
@@ -193,9 +194,11 @@ def test_decode_after_a_gather_free_prefill_reads_the_pages(reserve, n_steps):
         assert h.stats()["pages_free"] == free_before - ((prompts[0].n_total + reserve + 15) // 16 - sum(prompts[0].chunk_len) // 16)
 
 
-def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
-    """Where the streaming decode kernels are switched off, the first decode step runs the fetch the prefill skipped,
-    over every slot, which builds the context the gather form builds; the lent pages then go back."""
+@pytest.mark.parametrize("reserve_case", [0, 1], ids=["streaming-kernels", "tensor-core-kernels"])
+def test_decode_after_a_gather_free_prefill_assembles_the_context_late(reserve_case):
+    """Without the flag at decode time (here also with the streaming decode kernels switched off), the first decode step
+    runs the fetch the prefill skipped, over every slot, which builds the context the gather form builds; the lent
+    pages then go back."""
     reserve, n_steps = 3, 3
     dec, shape, weights, model, prompts, cached, store, want, states, toks = _decode_setup(109, reserve, n_steps)
     with G.make_handle(shape, weights, prompts, decode_reserve=reserve, flags=pcb.FLAG_GATHER_FREE) as h:
@@ -204,7 +207,7 @@ def test_decode_after_a_gather_free_prefill_assembles_the_context_late():
         free_before = h.stats()["pages_free"]
         got = h.prefill(G.specs_for(prompts, cached))
         assert h.stats()["gather_free"] == 1 and h.stats()["pages_free"] < free_before
-        h.set_flags(pcb.FLAG_GATHER_FREE | pcb.FLAG_NO_SMALL_ROW_KERNELS)
+        h.set_flags(pcb.FLAG_NO_SMALL_ROW_KERNELS if reserve_case else 0)
         for j in range(n_steps):
             out = h.decode(np.ascontiguousarray(toks[j]))
             ref = np.stack([dec.decode_step(model, states[b], orc.bf16_bits_to_f64(toks[j][b])) for b in range(len(prompts))])
