@@ -6,15 +6,20 @@
 // The host cuts the units' context ranges into items and deals them to the CTAs so that every CTA gets
 // the same number of context blocks; CTA c runs items [cta_first[c], cta_first[c + 1]) in order.
 //
-// One persistent CTA per SM, 320 threads:
+// One persistent CTA per SM, 384 threads:
 //   warps 0-3  softmax group of query head 2g      (thread = row; TMEM lanes by warp quarter)
 //   warps 4-7  softmax group of query head 2g + 1
 //   warp 8     TMA producer: Q tiles of both heads, then K and V blocks of 128 context slots into
 //              two-stage rings (each block = two 64-column halves in the 128-byte swizzle)
-//   warp 9     MMA issuer: S_i = Q_i K^T into TMEM, O_i += P_i V with P_i read from TMEM
-// TMEM (512 columns): S_0 [0,128) S_1 [128,256) O_0 [256,384) O_1 [384,512); P_i (fp16, two per
-// column) overwrites the first 64 columns of S_i.  Per head the chain S -> softmax -> PV -> next S is
-// serial; the two heads alternate so the tensor core works on one while the other is in softmax.
+//   warp 9     MMA issuer: S_i = Q_i K^T into TMEM (and, in MODE 2, O_i += P_i V with P_i read from TMEM)
+//   warp 10    MODE 0, 1: issuer of O_i += P_i V;  MODE 2: warps 10-11 rotate K (see below)
+// TMEM (512 columns), MODE 0 and 1: O_0 [0,128) O_1 [128,256); one S buffer [256,384) that both heads
+// take turns with; P_0 [384,448) P_1 [448,512) (16-bit, two per column).  A softmax group copies its S
+// block into registers at once and hands the buffer back, so the next S block is computed while the
+// exponentials of the current ones run, and a PV product never stands between a group and its next S
+// block: S blocks and PV products are issued by two different threads (see the issuers).
+// MODE 2 (no warp to spare): S_0 [256,384) S_1 [384,512), P_i over the first 64 columns of S_i, one
+// issuer; per head the chain S -> softmax -> PV -> next S is serial and the two heads alternate.
 // The running maximum is only raised when the block maximum exceeds it by more than 8 (in log2
 // units), which keeps P below 2^8 and makes rescaling of O in TMEM rare.
 // A row at position p sees context slots 0..p of its prompt (hit or freshly computed alike).
@@ -25,8 +30,8 @@ namespace pc {
 
 namespace {
 
-constexpr int ATT_THREADS = 320;
-constexpr int ATT_THREADS_ROT = 384;          // + two warps that rotate K on its way from the pages (MODE 2)
+constexpr int ATT_THREADS = 384;               // registers are handed out per four warps: warps 10-11 cost nothing more
+constexpr int ATT_THREADS_ROT = 384;
 constexpr int BLK = 128;                       // rows per tile and context slots per block
 constexpr int HALF_TILE_BYTES = BLK * 64 * 2;  // 16 KB: 128 rows x 64 fp16 (one swizzled half)
 constexpr int TILE_BYTES = 2 * HALF_TILE_BYTES;
@@ -36,7 +41,7 @@ constexpr int ATT_SMEM_BYTES = 2 * TILE_BYTES + 2 * KV_STAGES * TILE_BYTES + 102
 constexpr int KRAW_ROWS = 64;
 constexpr int KRAW_SLOT_BYTES = 2 * KRAW_ROWS * 128;       // two 64-column halves of 64 rows
 constexpr int ATT_SMEM_BYTES_ROT = ATT_SMEM_BYTES + 2 * KRAW_SLOT_BYTES;
-constexpr uint32_t TMEM_S0 = 0, TMEM_O0 = 256;
+constexpr uint32_t TMEM_O0 = 0, TMEM_SX = 256, TMEM_P0 = 384;
 constexpr float RESCALE_THRESHOLD = 8.0f;
 
 struct AttnArgs {
@@ -80,15 +85,17 @@ __device__ __forceinline__ float fmax3(float a, float b, float c) {
 // context: the page gather and its write + re-read of every cached K and V byte disappear.
 // Everything else is the same kernel.
 template <int MODE>
-__global__ void __launch_bounds__(MODE == 2 ? ATT_THREADS_ROT : ATT_THREADS, 1)
+__global__ void __launch_bounds__(ATT_THREADS, 1)
 umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
                       const __grid_constant__ CUtensorMap tmV, AttnArgs args) {
   constexpr bool PAGED = MODE == 1;                  // Q, K, V all by page copies
   constexpr bool PV_BF16 = MODE != 0;                // V comes from the bf16 pages
+  constexpr bool SPLIT = MODE != 2;                  // two MMA issuers and the shared S buffer (see the header)
   extern __shared__ uint8_t smem_raw[];
   __shared__ __align__(8) uint64_t q_full, q_empty;
   __shared__ __align__(8) uint64_t k_full[KV_STAGES], k_empty[KV_STAGES], v_full[KV_STAGES], v_empty[KV_STAGES];
   __shared__ __align__(8) uint64_t s_full[2], p_full[2], o_done[2], o_free[2];
+  __shared__ __align__(8) uint64_t sx_free;          // the S buffer has been read into registers (4 warps arrive)
   __shared__ __align__(8) uint64_t kraw_full[2], kraw_empty[2];      // MODE 2: the ring of staged, unrotated K pages
   __shared__ uint32_t tmem_base_slot;
   __shared__ int cta_failed;       // set by any role whose bounded wait ran out (or saw another role's error)
@@ -125,6 +132,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       mbar_init(&o_done[i], 1); mbar_init(&o_free[i], 4);
       mbar_init(&kraw_full[i], 1); mbar_init(&kraw_empty[i], 2);
     }
+    mbar_init(&sx_free, 4);
     fence_mbar_init();
   }
   if (warp == 9) {
@@ -236,7 +244,7 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
                       g * HEAD_DIM + hf * 64, page * PAGE_TOKENS);
       }
     }
-  } else if (warp >= 10) {
+  } else if (warp >= 10 && MODE == 2) {
     // ---------------------------------------------------------------- K rotated on its way to the S MMA (MODE 2 only:
     // the other forms are launched without these warps).  64 threads: thread (r0 = tid / 8, j = tid % 8) takes rows
     // r0, r0 + 8, ... and, in each, the 16-byte vector j of the head's low half and the one of its high half (elements
@@ -361,61 +369,102 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
       }
       (void)ok;
     }
-  } else if (warp == 9) {
-    // ---------------------------------------------------------------- MMA issuer
+  } else if (warp == 9 || (warp == 10 && MODE != 2)) {
+    // ---------------------------------------------------------------- MMA issuers
+    // Issuing a tcgen05.mma holds the thread until the tensor pipe takes it, so a single thread that also polls the
+    // barriers between groups leaves the pipe idle for that long after every group.  Where a warp is free (MODE 0
+    // and 1) the S blocks are issued by warp 9 and the PV products by warp 10, each in its own order
+    // (S_0(j), S_1(j), S_0(j+1), ... and PV_0(j), PV_1(j), ...): every dependency between them goes through a
+    // barrier (S buffer free, P written, PV complete), none through the order in the pipe.  In MODE 2 warps 10-11
+    // rotate K and warp 9 issues both, in the order  PV_0(j), S_0(j+1), PV_1(j), S_1(j+1).
     if (lane == 0) {
       // operand type of each MMA: 0 fp16, 1 bf16 (both operands of one MMA always have the same type)
       constexpr uint32_t idesc_qk = make_idesc_f16(BLK, BLK, PAGED ? 1 : 0, 0, 0);          // A, B K-major
       constexpr uint32_t idesc_pv = make_idesc_f16(BLK, HEAD_DIM, PV_BF16 ? 1 : 0, 0, 1);   // B (V) MN-major
-      uint32_t unit_it = 0, kvit = 0;
+      uint32_t unit_it = 0, kvit = 0, s_it = 0;      // s_it: S blocks issued so far, all into the one S buffer
       bool ok = true;
-      // S_i(kvidx) = Q_i K(kvidx)^T
+      auto fail = [&]() { ok = false; cta_failed = 1; };
+      // S_i(kvidx) = Q_i K(kvidx)^T, once the previous S block (of the other head) has been read out of the buffer
       auto issue_s = [&](int i, uint32_t kvidx) {
+        if (SPLIT) {
+          if (s_it != 0 && !mbar_wait(&sx_free, (s_it - 1u) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { fail(); return; }
+          tc_fence_after_sync();
+        }
         const int st = kvidx & 1;
         const uint32_t qa = smem_u32(q_smem + i * TILE_BYTES), ka = smem_u32(k_smem + st * TILE_BYTES);
 #pragma unroll
         for (int kk = 0; kk < HEAD_DIM / 16; ++kk) {
           const uint32_t off = (kk >> 2) * HALF_TILE_BYTES + (kk & 3) * 32;
-          umma_ss(tmem_base + TMEM_S0 + i * BLK, make_smem_desc_sw128(qa + off, 16, 1024),
+          umma_ss(tmem_base + TMEM_SX + (SPLIT ? 0 : i * BLK), make_smem_desc_sw128(qa + off, 16, 1024),
                   make_smem_desc_sw128(ka + off, 16, 1024), idesc_qk, kk != 0 ? 1u : 0u);
         }
         umma_commit(&s_full[i]);
+        ++s_it;
+      };
+      // O_i += P_i(kvidx) V(kvidx)
+      auto issue_pv = [&](int i, uint32_t kvidx, bool first) {
+        const int st = kvidx & 1;
+        if (!mbar_wait(&p_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { fail(); return; }
+        if (first && !mbar_wait(&o_free[i], (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_MMA)) { fail(); return; }
+        if (i == 0 && !mbar_wait(&v_full[st], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { fail(); return; }
+        tc_fence_after_sync();
+        const uint32_t va = smem_u32(v_smem + st * TILE_BYTES);
+#pragma unroll
+        for (int kk = 0; kk < BLK / 16; ++kk) {
+          // 16 context slots = 16 rows of 128 bytes in each 64-column half; halves are 16 KB apart
+          umma_ts(tmem_base + TMEM_O0 + i * HEAD_DIM, tmem_base + (SPLIT ? TMEM_P0 + i * (BLK / 2) : TMEM_SX + i * BLK) + kk * 8,
+                  make_smem_desc_sw128(va + kk * 2048, HALF_TILE_BYTES, 1024), idesc_pv, (!first || kk != 0) ? 1u : 0u);
+        }
+        umma_commit(&o_done[i]);
+        if (i == 1) umma_commit(&v_empty[st]);
+      };
+      auto wait_k = [&](uint32_t kvidx) {
+        if (!mbar_wait(&k_full[kvidx & 1], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) fail();
       };
       for (int w = w_begin; w < w_end && ok; ++w, ++unit_it) {
         const AttnItem t = w == w_begin ? first_item : args.items[w];
         const int nb = t.blk_end - t.blk_begin;
         const uint32_t kv0 = kvit;
-        if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-        if (!mbar_wait(&k_full[kv0 & 1], (kv0 >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-        tc_fence_after_sync();
+        if (SPLIT && warp == 10) {
+          for (int j = 0; j < nb && ok; ++j) {
+            issue_pv(0, kv0 + j, j == 0);
+            if (ok) issue_pv(1, kv0 + j, j == 0);
+          }
+          kvit += nb;
+          continue;
+        }
+        if (!mbar_wait(&q_full, unit_it & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { fail(); break; }
+        if (SPLIT) {
+          for (int j = 0; j < nb && ok; ++j) {
+            wait_k(kv0 + j);
+            if (ok) issue_s(0, kv0 + j);
+            if (ok) issue_s(1, kv0 + j);
+            if (!ok) break;
+            umma_commit(&k_empty[(kv0 + j) & 1]);
+            if (j + 1 == nb) umma_commit(&q_empty);
+          }
+          kvit += nb;
+          continue;
+        }
+        // one issuer, one S buffer per head: per head the chain S -> softmax -> PV -> next S is serial (P lies over
+        // the first half of S), the two heads alternate
+        wait_k(kv0);
+        if (!ok) break;
         issue_s(0, kv0);
         issue_s(1, kv0);
         umma_commit(&k_empty[kv0 & 1]);
         if (nb == 1) umma_commit(&q_empty);
         for (int j = 0; j < nb && ok; ++j) {
           const uint32_t kvidx = kv0 + j;
-          const int st = kvidx & 1;
-          for (int i = 0; i < 2; ++i) {
-            if (!mbar_wait(&p_full[i], kvidx & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-            if (j == 0 && !mbar_wait(&o_free[i], (unit_it & 1u) ^ 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-            if (i == 0 && !mbar_wait(&v_full[st], (kvidx >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-            tc_fence_after_sync();
-            const uint32_t va = smem_u32(v_smem + st * TILE_BYTES);
-#pragma unroll
-            for (int kk = 0; kk < BLK / 16; ++kk) {
-              // 16 context slots = 16 rows of 128 bytes in each 64-column half; halves are 16 KB apart
-              umma_ts(tmem_base + TMEM_O0 + i * HEAD_DIM, tmem_base + TMEM_S0 + i * BLK + kk * 8,
-                      make_smem_desc_sw128(va + kk * 2048, HALF_TILE_BYTES, 1024), idesc_pv, (j | kk) != 0 ? 1u : 0u);
-            }
-            umma_commit(&o_done[i]);
-            if (i == 1) umma_commit(&v_empty[st]);
+          for (int i = 0; i < 2 && ok; ++i) {
+            issue_pv(i, kvidx, j == 0);
+            if (!ok) break;
             if (j + 1 < nb) {
-              const uint32_t nxt = kvidx + 1;
-              if (i == 0 && !mbar_wait(&k_full[nxt & 1], (nxt >> 1) & 1u, args.err_word, DEV_ERR_ATTN_MMA)) { ok = false; cta_failed = 1; break; }
-              tc_fence_after_sync();
-              issue_s(i, nxt);
+              if (i == 0) wait_k(kvidx + 1);
+              if (!ok) break;
+              issue_s(i, kvidx + 1);
               if (i == 1) {
-                umma_commit(&k_empty[nxt & 1]);
+                umma_commit(&k_empty[(kvidx + 1) & 1]);
                 if (j + 2 == nb) umma_commit(&q_empty);
               }
             }
@@ -424,13 +473,14 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         kvit += nb;
       }
     }
-  } else {
+  } else if (warp < 8) {
     // ---------------------------------------------------------------- softmax groups (warps 0..7)
     const int i = warp >> 2;                      // which query head of the pair
     const int quarter = warp & 3;
     const int r_in_tile = quarter * 32 + lane;
     const uint32_t lane_base = static_cast<uint32_t>(quarter * 32) << 16;
-    const uint32_t t_s = tmem_base + lane_base + TMEM_S0 + i * BLK;
+    const uint32_t t_s = tmem_base + lane_base + TMEM_SX + (SPLIT ? 0 : i * BLK);
+    const uint32_t t_p = SPLIT ? tmem_base + lane_base + TMEM_P0 + i * (BLK / 2) : t_s;
     const uint32_t t_o = tmem_base + lane_base + TMEM_O0 + i * HEAD_DIM;
     uint32_t unit_it = 0, kvit = 0;
     bool ok = true;
@@ -454,6 +504,11 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
 #pragma unroll
         for (int c = 0; c < 4; ++c) tmem_ld_32x32(t_s + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
         tmem_wait_ld();
+        if (SPLIT) {
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&sx_free);              // the block is in registers: the buffer may take the next
+        }
         const int limit = pos - (t.blk_begin + j) * BLK;     // columns 0..limit are visible
         // maximum of the raw scores (the scale is positive, so it commutes with the maximum)
         // four independent chains: the reduction is bound by instruction latency, not by issue
@@ -516,8 +571,13 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
         }
         const float sum = sum0 + sum1;
         l += sum;
-        tmem_st_32x32(t_s, *reinterpret_cast<uint32_t(*)[32]>(&p[0]));
-        tmem_st_32x32(t_s + 32, *reinterpret_cast<uint32_t(*)[32]>(&p[32]));
+        // P_i of the previous block must have been consumed (PV complete) before it is overwritten
+        ok = mbar_wait(&o_done[i], (kvidx - 1u) & 1u, args.err_word, DEV_ERR_ATTN_CORR);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) { cta_failed = 1; break; }
+        tc_fence_after_sync();
+        tmem_st_32x32(t_p, *reinterpret_cast<uint32_t(*)[32]>(&p[0]));
+        tmem_st_32x32(t_p + 32, *reinterpret_cast<uint32_t(*)[32]>(&p[32]));
         tmem_wait_st();
         tc_fence_before_sync();
         __syncwarp();
