@@ -65,6 +65,26 @@ __device__ __forceinline__ float fast_exp2(float x) {
   return y;
 }
 
+// two fp32 lanes per instruction (packed in a 64-bit register pair)
+__device__ __forceinline__ uint64_t pack_f32x2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack_f32x2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma_f32x2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c));
+  return r;
+}
+__device__ __forceinline__ uint64_t add_f32x2(uint64_t a, uint64_t b) {
+  uint64_t r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b));
+  return r;
+}
+
 // max(a, b, c) in one instruction (three-input form of max.f32)
 __device__ __forceinline__ float fmax3(float a, float b, float c) {
   float y;
@@ -553,14 +573,17 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
           }
         }
         uint32_t p[64];
-        float sum0 = 0.f, sum1 = 0.f;
         const float neg_m = -m;
+        const uint64_t scale2 = pack_f32x2(args.scale_log2, args.scale_log2), negm2 = pack_f32x2(neg_m, neg_m);
+        uint64_t sum2a = pack_f32x2(0.f, 0.f), sum2b = sum2a;
 #pragma unroll
         for (int c = 0; c < 64; ++c) {
-          const float p0 = fast_exp2(fmaf(__uint_as_float(s[2 * c]), args.scale_log2, neg_m));
-          const float p1 = fast_exp2(fmaf(__uint_as_float(s[2 * c + 1]), args.scale_log2, neg_m));
-          sum0 += p0;
-          sum1 += p1;
+          float x0, x1;
+          unpack_f32x2(fma_f32x2(pack_f32x2(__uint_as_float(s[2 * c]), __uint_as_float(s[2 * c + 1])), scale2, negm2), x0, x1);
+          const float p0 = fast_exp2(x0);
+          const float p1 = fast_exp2(x1);
+          if (c & 1) sum2b = add_f32x2(sum2b, pack_f32x2(p0, p1));
+          else sum2a = add_f32x2(sum2a, pack_f32x2(p0, p1));
           if constexpr (PV_BF16) {          // P in the operand type of V
             __nv_bfloat162 bb = __floats2bfloat162_rn(p0, p1);
             p[c] = *reinterpret_cast<uint32_t*>(&bb);
@@ -569,6 +592,8 @@ umma_attention_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_cons
             p[c] = *reinterpret_cast<uint32_t*>(&hh);
           }
         }
+        float sum0, sum1;
+        unpack_f32x2(add_f32x2(sum2a, sum2b), sum0, sum1);
         const float sum = sum0 + sum1;
         l += sum;
         // P_i of the previous block must have been consumed (PV complete) before it is overwritten
