@@ -121,6 +121,35 @@ def test_batch_of_ragged_prompts_and_first_miss_wins():
         assert np.max(np.abs(again[0].out_hidden - got[0].out_hidden[-17:])) < 2e-2
 
 
+def test_many_units_of_every_length_in_one_call():
+    """One call whose attention work list holds units of one block and of many, tiles of one row and of 128, several
+    items per CTA and units cut along the context: what the two MMA-issuing threads of the attention kernel hand to
+    each other (S buffer, P, PV completion) is exercised across every kind of unit boundary."""
+    shape = wl.small_workload(seed=47, n_layers=2, chunk_lens=[8], n_query=1, hit_idx=[]).shape
+    weights = wl.make_weights(shape, 47, random_gains=True)
+    model = H.oracle_model(shape, weights)
+    lens = {200 + c: int(n) for c, n in enumerate([5, 16, 33, 64, 100, 128, 129, 200, 257, 400, 48, 7])}
+    mk = lambda cid: wl.chunk_hidden_for(47, cid, lens[cid], shape.d_model)
+    cached = [201, 204, 207, 209]
+    prompts = []
+    for b, (ids, nq) in enumerate([([200], 1), ([201, 202], 3), ([209, 203], 128), ([204, 205, 206], 40),
+                                   ([207], 300), ([208, 210], 17), ([209, 207, 204], 1), ([211, 201], 129),
+                                   ([205], 64), ([206, 209, 208], 2)]):
+        prompts.append(wl.Prompt(ids, [lens[c] for c in ids], nq, [mk(c) for c in ids],
+                                 wl.make_hidden(47, (2, b), nq, shape.d_model)))
+    store = G.oracle_store_alone(model, 47, [(c, lens[c]) for c in cached])
+    want = orc.reuse_prefill(model, store, [H.oracle_prompt(p, [i for i, c in enumerate(p.chunk_ids) if c in cached])
+                                            for p in prompts], commit=False)
+    with G.make_handle(shape, weights, prompts) as h:
+        G.push_store(h, store, cached)
+        got = h.prefill(G.specs_for(prompts, cached))
+        G.check_plan(h.read_plan(), [r.layout for r in want])
+        for b, (g, r) in enumerate(zip(got, want)):
+            assert g.n_new == len(r.layout.new_slots)
+            c = G.compare_hidden(g.out_hidden, r.out_hidden)
+            assert c["max_abs"] <= G.TOL_MAX_ABS and c["mean_abs"] <= G.TOL_MEAN_ABS, (b, c)
+
+
 def test_host_side_errors_leave_store_unchanged():
     w = wl.small_workload(seed=47, n_layers=1, chunk_lens=[32, 32], n_query=4, hit_idx=[])
     weights = wl.make_weights(w.shape, w.seed)
